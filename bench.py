@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the CLSA decode hot path: index scores + top-k + L sparse-attention layers per step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+A step is one `clsa_decode_step` call (through the C ABI) over one batch of seeded synthetic input
+that is already resident in HBM. Each timed step is bracketed by its own CUDA events on the launch
+stream; between steps a 512 MiB buffer is rewritten so every step starts with a cold L2 (the reuse
+of gathered rows between the layers of one step is part of the method and is kept).
+`value` = algorithmic bytes per step (indexer-key bytes + L * selected rows * Hkv * D * 2 B * {K,V})
+divided by the mean step time, summed over ranks. With --gpus N > 1 (launched by torchrun) every rank
+runs an independent replica of the workload: the path has no exchange step, so there is no collective
+on the data path ("replicas only").
+
+--impl reference times the CPU oracle on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode step HBM GB/s (index+top-k+L-layer sparse attn)"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="headline128k")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--no-breakdown", action="store_true", help="skip the per-kernel instrumented loop")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Polls NVML (read-only) for SM clock and clock-event reasons while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        med = sorted(self.samples)[len(self.samples) // 2] if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# --------------------------------------------------------------------------------------- oracle legs
+def oracle_sample(w, seqs, layers):
+    """Time the oracle, as it stands, on sequences `seqs` and `layers` layers of workload `w`.
+    Returns (seconds, algorithmic bytes of the sample, threads). Input synthesis is not timed."""
+    import numpy as np
+
+    import oracle
+    from workloads import Workload
+
+    c = w.cfg
+    sub = Workload(c.replace(num_seqs=len(seqs), num_layers=layers))
+    # the sample reuses the parent's per-sequence contents: same lengths, same keys, same queries
+    sub.seq_len = w.seq_len[seqs].copy()
+    sub.max_seq_len = int(sub.seq_len.max())
+    starts, acc = [], 0
+    for n in sub.seq_len:
+        starts.append(acc)
+        acc += int(n)
+    sub.seq_start = np.array(starts, dtype=np.int64)
+    sub.total_rows = acc
+    kidx = np.concatenate([w.kidx_bits(int(b)) for b in seqs])
+    q_idx = w.q_idx_bits()[seqs]
+    prob = oracle.problem_from_workload(sub, idx_k_cache=kidx)
+    t0 = time.perf_counter()
+    scores = prob.index_scores(q_idx)
+    idx, cnt = prob.topk(scores)
+    t_route = time.perf_counter() - t0
+    # K/V rows the selection touches (synthesised outside the timed region)
+    kc = np.zeros((sub.total_rows, c.num_kv_heads, c.head_dim), dtype=np.uint16)
+    vc = np.zeros_like(kc)
+    for i, b in enumerate(seqs):
+        for t in range(c.q_per_seq):
+            loc = idx[i, t, : cnt[i, t]].astype(np.int64)
+            kc[sub.seq_start[i] + loc] = w.kv_rows_bits("k", int(w.seq_start[b]) + loc).reshape(-1, c.num_kv_heads, c.head_dim)
+            vc[sub.seq_start[i] + loc] = w.kv_rows_bits("v", int(w.seq_start[b]) + loc).reshape(-1, c.num_kv_heads, c.head_dim)
+    prob2 = oracle.problem_from_workload(sub, k_cache=kc, v_cache=vc, idx_k_cache=kidx)
+    qs = [w.q_layer_bits(l)[seqs] for l in range(layers)]
+    t0 = time.perf_counter()
+    for l in range(layers):
+        prob2.sparse_attn(qs[l], idx, cnt)
+    t_attn = time.perf_counter() - t0
+    nbytes = int(sub.seq_len.astype(np.int64).sum()) * c.idx_dim * 2 + layers * int(cnt.sum()) * c.num_kv_heads * c.head_dim * 4
+    return t_route + t_attn, nbytes, oracle.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from workloads import CONFIGS, Workload
+
+    oracle.build()
+    w = Workload(CONFIGS[args.config])
+    c = w.cfg
+    seqs = [0]
+    sample = f"sequence 0 of {c.num_seqs}, all {c.num_layers} layers, whole context, per step"
+    for _ in range(max(1, min(args.warmup, 1))):
+        oracle_sample(w, seqs, c.num_layers)
+    tot_s, tot_b, threads = 0.0, 0, 1
+    for _ in range(args.steps):
+        s, b, threads = oracle_sample(w, seqs, c.num_layers)
+        tot_s += s
+        tot_b += b
+    val = tot_b / tot_s / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": tot_s / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": c.name, "num_seqs": c.num_seqs, "context": c.ctx, "top_k": c.top_k,
+                   "layers": c.num_layers, "q_heads": c.num_q_heads, "kv_heads": c.num_kv_heads, "idx_dim": c.idx_dim},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------- CUDA arm
+def run_ours(args):
+    import torch
+
+    import __graft_entry__ as entry
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank == 0:
+        entry._load_build_module().build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    else:
+        torch.cuda.set_device(local)
+    import paper_2606_06467_b200 as clsa
+    from workloads import CONFIGS, Workload
+
+    dev = torch.device("cuda", local)
+    w = Workload(CONFIGS[args.config])
+    c = w.cfg
+    if c.q_per_seq != 1:
+        raise SystemExit("bench.py times decode workloads (q_per_seq == 1)")
+    t = w.to_device(dev)
+    L = c.num_layers
+    p = clsa.make_params(num_seqs=c.num_seqs, num_q_heads=c.num_q_heads, num_kv_heads=c.num_kv_heads,
+                         head_dim=c.head_dim, idx_dim=c.idx_dim, top_k=c.top_k, num_layers=L, max_seq_len=w.max_seq_len,
+                         sm_scale=c.sm_scale, seq_start=t["seq_start"], seq_len=t["seq_len"], k_cache=t["k_cache"],
+                         v_cache=t["v_cache"], idx_k_cache=t["idx_k_cache"])
+    ws = torch.zeros(clsa.clsa_workspace_bytes(p), dtype=torch.uint8, device=dev)
+    idx = torch.empty((c.num_seqs, 1, c.top_k), dtype=torch.int32, device=dev)
+    cnt = torch.empty((c.num_seqs, 1), dtype=torch.int32, device=dev)
+    q_layers = [t["q_layers"][l] for l in range(L)]
+    outs = [torch.empty((c.num_seqs, 1, c.num_q_heads, c.head_dim), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    alg_bytes = w.algorithmic_bytes()
+    stream = torch.cuda.current_stream()
+
+    def step():
+        clsa.clsa_decode_step(p, t["q_idx"], q_layers, outs, idx, cnt, ws, stream=stream)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        flush.zero_()
+        step()
+    sync_all()
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    K = args.steps
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for i in range(K):
+        flush.zero_()
+        ev[i][0].record(stream)
+        step()
+        ev[i][1].record(stream)
+    sync_all()
+    clocks = sampler.stop()
+    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    assert clsa.clsa_device_status(ws) == 0, "device status word is not clean"
+    if dist is not None:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / K
+    value = world * alg_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: per-step inputs from pinned host memory, per-step results back to the host --------
+    h_qidx = t["q_idx"].cpu().pin_memory()
+    h_q = [q.cpu().pin_memory() for q in q_layers]
+    h_out = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs]
+    d_qidx = torch.empty_like(t["q_idx"])
+    d_q = [torch.empty_like(q) for q in q_layers]
+
+    def e2e_step():
+        d_qidx.copy_(h_qidx, non_blocking=True)
+        for l in range(L):
+            d_q[l].copy_(h_q[l], non_blocking=True)
+        clsa.clsa_decode_step(p, d_qidx, d_q, outs, idx, cnt, ws, stream=stream)
+        for l in range(L):
+            h_out[l].copy_(outs[l], non_blocking=True)
+
+    for _ in range(3):
+        flush.zero_()
+        e2e_step()
+    sync_all()
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for i in range(K):
+        flush.zero_()
+        ev2[i][0].record(stream)
+        e2e_step()
+        ev2[i][1].record(stream)
+    sync_all()
+    e2e_ms = sum(a.elapsed_time(b) for a, b in ev2)
+    if dist is not None:
+        tt = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_value = world * alg_bytes / (e2e_ms / K * 1e-3) / 1e9
+    h2d = (h_qidx.numel() + sum(q.numel() for q in h_q)) * 2
+    d2h = sum(o.numel() for o in h_out) * 2
+
+    # ---- per-kernel durations: the same launches issued as separate ABI calls with events between -------
+    breakdown = None
+    attn_us = None
+    if not args.no_breakdown:
+        scores = ws  # decode_step keeps its scores in the workspace; the separate calls get their own buffer
+        stride = (w.max_seq_len + 63) // 64 * 64
+        scores = torch.empty((c.num_seqs, 1, stride), dtype=torch.float32, device=dev)
+        nb = min(K, 20)
+        acc = {"index_scores": 0.0, "topk": 0.0, "sparse_attn": 0.0}
+        for i in range(nb + 2):
+            flush.zero_()
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(L + 3)]
+            marks[0].record(stream)
+            clsa.clsa_index_scores(p, t["q_idx"], scores, stride, ws, stream=stream)
+            marks[1].record(stream)
+            clsa.clsa_topk(p, scores, stride, idx, cnt, ws, stream=stream)
+            marks[2].record(stream)
+            for l in range(L):
+                p.sweep = l & 1
+                clsa.clsa_sparse_attn(p, q_layers[l], idx, cnt, outs[l], None, ws, stream=stream)
+                marks[3 + l].record(stream)
+            p.sweep = 0
+            torch.cuda.synchronize()
+            if i >= 2:
+                acc["index_scores"] += marks[0].elapsed_time(marks[1])
+                acc["topk"] += marks[1].elapsed_time(marks[2])
+                acc["sparse_attn"] += marks[2].elapsed_time(marks[2 + L])
+        breakdown = {k: v / nb * 1e3 for k, v in acc.items()}  # microseconds per step
+        attn_us = breakdown["sparse_attn"] / L
+        breakdown["sparse_attn_per_layer"] = attn_us
+
+    peak, peak_kind = measured_peaks()
+    gathered_per_layer = int(w.selected_counts().sum()) * c.num_kv_heads * c.head_dim * 4
+    roofline = {
+        "bound": "hbm", "kernel": "sparse_attn_kernel (+ merge), one layer",
+        "achieved": (gathered_per_layer / (attn_us * 1e-6) / 1e9) if attn_us else None,
+        "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+        "frac": (gathered_per_layer / (attn_us * 1e-6) / 1e9 / peak) if attn_us else None,
+        "traffic": None,
+        "algorithmic_bytes_per_launch": gathered_per_layer,
+        "step_frac": value / world / peak,
+    }
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        try:
+            with open(prof) as f:
+                roofline["traffic"] = json.load(f).get(c.name, {}).get("sparse_attn_kernel")
+        except Exception:
+            pass
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+
+        oracle.build()
+        seqs = list(range(c.num_seqs)) if c.num_seqs <= 16 else list(range(0, c.num_seqs, c.num_seqs // 16))[:16]
+        secs, nbytes, threads = oracle_sample(w, seqs, L)
+        cpu_baseline = {"value": nbytes / secs / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+                        "sample": f"{len(seqs)} of {c.num_seqs} sequences, all {L} layers, one pass ({secs:.2f} s)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
+            "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": c.name, "num_seqs": c.num_seqs, "context": c.ctx, "top_k": c.top_k, "layers": L,
+                       "q_heads": c.num_q_heads, "kv_heads": c.num_kv_heads, "idx_dim": c.idx_dim,
+                       "algorithmic_bytes_per_step": alg_bytes, "l2": "flushed between steps (512 MiB rewrite)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "roofline": roofline, "breakdown_us": breakdown, "cpu_baseline": cpu_baseline,
+            "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms / K,
+                    "note": "per-step inputs (q_idx, L query tensors) from pinned host memory and all L outputs back; "
+                            "the KV and indexer-key caches are decoder state and stay resident"},
+            "gpu_launches": K * (2 + 2 * L),
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

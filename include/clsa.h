@@ -1,0 +1,150 @@
+/*
+ * clsa.h -- C ABI of the CLSA decoding hot path for NVIDIA B200 (sm_100a).
+ *
+ * Cross-layer sparse attention shares one routing index between all cross-decoder layers that read
+ * the same KV cache. The path behind this boundary is the part of a decode (or prefill-chunk) step
+ * that touches the caches:
+ *
+ *   1. index scores   I = Q_idx K_idx^T                      (Eq. 3; single indexer head, Eq. 2)
+ *   2. routing index  S_t = TopK(I_t, k), once per query     (Eq. 3)
+ *   3. per layer l    O_t^(l) = Attn(Q_t^(l), K_{S_t}, V_{S_t}) (Eq. 4), every layer reusing S_t
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ * Pointers: every pointer is a DEVICE pointer unless its comment says HOST. The clsa_params struct
+ *   itself lives in host memory and is read during the call only.
+ * Ownership: the caller owns every buffer (inputs, outputs, workspace). The library allocates
+ *   nothing, frees nothing, keeps no state between calls except cached device properties, and only
+ *   enqueues work on the given stream. No entry point synchronises except clsa_device_status.
+ * Errors: each call returns a clsa_status. All argument checks run on the host before anything is
+ *   enqueued: a call that returns CLSA_ERR_INVALID_ARG, CLSA_ERR_UNSUPPORTED or CLSA_ERR_WORKSPACE
+ *   has launched nothing. Unsupported shapes are refused, never routed to a slower path.
+ *   Data-dependent problems seen on the device (an index outside its sequence, a sequence longer
+ *   than max_seq_len) never trap: the offending element is skipped and a bit is set in the status
+ *   word at the start of the workspace (see clsa_device_status).
+ * Layout: bf16 = IEEE bfloat16 bit patterns. Strides are in elements. Cache rows of sequence b are
+ *   rows seq_start[b] .. seq_start[b] + seq_len[b] - 1 of one row space shared by K, V and K_idx.
+ *   The last q_per_seq tokens of a sequence are its query tokens (their own K/V/K_idx rows have
+ *   already been appended by the caller).
+ * Visibility: with causal == 0 every query sees all seq_len[b] tokens (decoding); with causal == 1
+ *   query t (0-based, of T = q_per_seq) sees positions s <= seq_len[b] - T + t.
+ * Index contract: idx holds, per (sequence, query), `count` distinct sequence-local positions in
+ *   [0, visible); entries at or beyond count are -1. clsa_topk emits them in ascending position
+ *   order; clsa_sparse_attn accepts any order.
+ */
+#ifndef CLSA_H_
+#define CLSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define CLSA_API __attribute__((visibility("default")))
+#else
+#define CLSA_API
+#endif
+
+typedef enum {
+  CLSA_OK = 0,
+  CLSA_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer or stride */
+  CLSA_ERR_UNSUPPORTED = 2, /* valid but not built: head_dim != 128, idx_dim not in {64,128}, group size > 16 ... */
+  CLSA_ERR_WORKSPACE = 3,   /* workspace null, misaligned (256 B) or smaller than clsa_workspace_bytes */
+  CLSA_ERR_CUDA = 4         /* a CUDA runtime call or launch failed; cudaGetLastError has the detail */
+} clsa_status;
+
+/* Bits of the device status word (first 4 bytes of the workspace, cleared by the host of the caller
+ * or by clsa_clear_status; kernels only ever OR into it). */
+#define CLSA_DEV_BAD_INDEX 1u   /* an idx entry < 0 or >= seq_len inside the first `count` entries: skipped */
+#define CLSA_DEV_BAD_SEQLEN 2u  /* seq_len[b] < q_per_seq or > max_seq_len: that sequence was skipped */
+#define CLSA_DEV_BAD_COUNT 4u   /* count[b,t] < 0 or > top_k: clamped */
+
+typedef void* clsa_stream; /* a cudaStream_t */
+
+typedef struct {
+  int32_t num_seqs;     /* B >= 1 */
+  int32_t q_per_seq;    /* T >= 1: 1 = decode; > 1 = prefill chunk */
+  int32_t num_q_heads;  /* Hq; Hq % Hkv == 0; group size Hq/Hkv <= 16 */
+  int32_t num_kv_heads; /* Hkv */
+  int32_t head_dim;     /* D == 128 */
+  int32_t idx_dim;      /* d_idx: 64 or 128 */
+  int32_t top_k;        /* k >= 1: the maximum number of activated tokens per query */
+  int32_t num_layers;   /* L >= 1; read by clsa_decode_step and clsa_workspace_bytes only */
+  int32_t causal;       /* 0 or 1, see "Visibility" */
+  int32_t max_seq_len;  /* host-known upper bound of seq_len[], used for grid sizing (no device read-back) */
+  float sm_scale;       /* softmax scale of Eq. 4's Attn; 1/sqrt(head_dim) in the benchmarks */
+  int32_t sweep;        /* 0 or 1: direction in which clsa_sparse_attn walks the selected set; a cache-locality
+                           hint only (results agree to rounding). clsa_decode_step uses (sweep + l) & 1 for layer l */
+  const int64_t* seq_start; /* [B] first cache row of each sequence */
+  const int32_t* seq_len;   /* [B] valid tokens n_b >= T, including the T query tokens */
+  const void* k_cache;      /* bf16 [rows][Hkv][D]; element (r,g,d) at r*kv_token_stride + g*kv_head_stride + d */
+  const void* v_cache;      /* bf16, same layout and strides as k_cache */
+  int64_t kv_token_stride;  /* multiple of 8 (16-byte rows) */
+  int64_t kv_head_stride;   /* multiple of 8 */
+  const void* idx_k_cache;  /* bf16 [rows][d_idx]; element (r,j) at r*idx_token_stride + j */
+  int64_t idx_token_stride; /* multiple of 8 */
+} clsa_params;
+
+/* Bytes of workspace that any of the calls below may need for these params (the maximum over the
+ * four; clsa_decode_step additionally keeps the fp32 score matrix there). Reads only the scalar
+ * fields. *bytes is HOST memory. The workspace must be 256-byte aligned; its first 256 bytes hold
+ * the device status word and must be zero before the first call (cudaMemset or clsa_clear_status). */
+CLSA_API clsa_status clsa_workspace_bytes(const clsa_params* p, size_t* bytes);
+
+/* Eq. 3, first half: scores[b][t][s] = sum_j q_idx[b][t][j] * K_idx[seq_start[b]+s][j] for every
+ * visible s; the bare dot product, no scale and no activation, one indexer head. bf16 products are
+ * exact in fp32; accumulation is fp32. Entries at s >= visible(b,t) are not written.
+ *   q_idx  bf16 [B][T][d_idx], 16-byte aligned
+ *   scores fp32 [B][T][score_stride], score_stride >= max_seq_len
+ * T == 1 streams the indexer-key cache once (HBM-bound); T > 1 is a tensor-core GEMM. */
+CLSA_API clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* scores, int64_t score_stride,
+                              void* workspace, size_t workspace_bytes, clsa_stream stream);
+
+/* Eq. 3, second half: per (b,t) the c = min(k, visible) positions with the largest scores, ties to
+ * the lower position, -0.0 equal to +0.0. Fewer than k visible tokens selects all of them (k is a
+ * maximum). Exact selection: no approximation, no sampling.
+ *   idx   int32 [B][T][k]  ascending positions, tail -1
+ *   count int32 [B][T]
+ * Scores must be finite; a NaN is ordered by its bit pattern and never faults. */
+CLSA_API clsa_status clsa_topk(const clsa_params* p, const float* scores, int64_t score_stride, int32_t* idx,
+                      int32_t* count, void* workspace, size_t workspace_bytes, clsa_stream stream);
+
+/* Eq. 4 for ONE layer: for each (b,t) and query head h with KV head g = h / (Hq/Hkv),
+ *   O = sum_{s in S} softmax_s(sm_scale * Q[b][t][h] . K[s][g]) V[s][g]   over the selected rows only.
+ * No positional rotation is applied (the cross-decoder's global attention is NoPE).
+ *   q   bf16 [B][T][Hq][D]           this layer's queries, 16-byte aligned
+ *   out bf16 [B][T][Hq][D]           round-to-nearest-even from fp32 accumulators
+ *   lse fp32 [B][T][Hq] or NULL      log-sum-exp of the scaled logits (natural log)
+ * A (b,t) with count 0 yields zeros and lse = -inf. */
+CLSA_API clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t* idx, const int32_t* count,
+                             void* out, float* lse, void* workspace, size_t workspace_bytes, clsa_stream stream);
+
+/* One step (Sec. 2.1: the routing index is computed once and shared by the layers): index scores, TopK, then L
+ * sparse-attention launches on `stream`, all fed the same idx/count, which are returned.
+ *   q_layers   HOST array of L device pointers, each bf16 [B][T][Hq][D]
+ *   out_layers HOST array of L device pointers, each bf16 [B][T][Hq][D]
+ * Equivalent, bit for bit, to clsa_index_scores, clsa_topk and L calls of clsa_sparse_attn made one
+ * after another with sweep = (p->sweep + l) & 1 for layer l. T > 1 is not chained here. */
+CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
+                             void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
+                             size_t workspace_bytes, clsa_stream stream);
+
+/* Zero the status word (asynchronous, on `stream`). */
+CLSA_API clsa_status clsa_clear_status(void* workspace, size_t workspace_bytes, clsa_stream stream);
+
+/* Copy the device status word to *bits (HOST). Synchronises `stream`. */
+CLSA_API clsa_status clsa_device_status(const void* workspace, uint32_t* bits, clsa_stream stream);
+
+/* Static string for a status code. */
+CLSA_API const char* clsa_status_string(clsa_status s);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+CLSA_API int clsa_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CLSA_H_ */

@@ -9,7 +9,7 @@
  *   sparse attn    O_t^(l) = Attn(Q_t^(l), K_{S_t}, V_{S_t})      (Eq. 4)
  *   dense attn     O^(l) = Attn(Q^(l), K, V)    (Eq. 1) -- an independent routine used only to
  *                                               check the k >= n limit of Eq. 4
- *   decode step    one S_t, reused by every cross-decoder layer   (Sec. 2.1, last paragraph)
+ *   decode step    one S_t, reused by every cross-decoder layer   (Sec. 2.1, closing paragraph)
  *
  * These results are plain definitions (a matrix product, an exact selection, a softmax-weighted
  * mean over a subset), so each function is that definition written out with no blocking, fusion
@@ -19,7 +19,7 @@
  * Readings where the paper is silent (all listed in the design notes of the repository):
  *   - scores are the bare dot product (no scale, no activation);
  *   - ties in TopK go to the lower token index, scores compare by value (-0.0 == +0.0);
- *   - fewer than k visible tokens: all of them are selected ("maximal activated tokens");
+ *   - fewer than k visible tokens: all of them are selected (k is stated as a maximum);
  *   - decode: every cached token is visible; causal chunk: query t of T sees s <= n - T + t;
  *   - Attn is scaled dot-product attention with an explicit sm_scale, no positional rotation
  *     (NoPE in global attention), GQA with contiguous groups: KV head = query head / group size.

@@ -1,0 +1,228 @@
+// C-ABI entry points: argument validation, workspace carving and the launch sequence.
+// Every check that can refuse a call runs here on the host before anything is enqueued.
+#include <math.h>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace clsa {
+
+bool device_info(DeviceInfo* out) {
+  static std::mutex mu;
+  static DeviceInfo cache[64];
+  static bool have[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return false; }
+  if (dev < 0 || dev >= 64) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!have[dev]) {
+    DeviceInfo d;
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    cache[dev] = d;
+    have[dev] = true;
+  }
+  *out = cache[dev];
+  return true;
+}
+
+WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& dev) {
+  WorkspaceLayout w;
+  const AttnPlan plan = make_attn_plan(p, dev);
+  auto align = [](size_t x) { return (x + 255) / 256 * 256; };
+  w.partial_off = kStatusBytes;
+  w.partial_bytes = align(plan.partial_bytes);
+  w.scores_off = w.partial_off + w.partial_bytes;
+  w.score_stride = ((int64_t)p.max_seq_len + 63) / 64 * 64;
+  w.scores_bytes = align((size_t)p.num_seqs * p.q_per_seq * w.score_stride * sizeof(float));
+  w.total = w.scores_off + w.scores_bytes;
+  return w;
+}
+
+namespace {
+
+bool aligned(const void* ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) == 0; }
+
+// Checks of the scalar fields only (shared by every entry point).
+clsa_status check_shape(const clsa_params* p) {
+  if (p == nullptr) return CLSA_ERR_INVALID_ARG;
+  if (p->num_seqs < 1 || p->q_per_seq < 1 || p->num_q_heads < 1 || p->num_kv_heads < 1 || p->head_dim < 1 ||
+      p->idx_dim < 1 || p->top_k < 1 || p->num_layers < 1)
+    return CLSA_ERR_INVALID_ARG;
+  if (p->num_q_heads % p->num_kv_heads != 0) return CLSA_ERR_INVALID_ARG;
+  if (p->causal != 0 && p->causal != 1) return CLSA_ERR_INVALID_ARG;
+  if (p->sweep != 0 && p->sweep != 1) return CLSA_ERR_INVALID_ARG;
+  if (p->max_seq_len < p->q_per_seq) return CLSA_ERR_INVALID_ARG;
+  if (!isfinite(p->sm_scale)) return CLSA_ERR_INVALID_ARG;
+  if ((int64_t)p->num_seqs * p->q_per_seq > (int64_t)1 << 30) return CLSA_ERR_INVALID_ARG;
+  if (p->head_dim != 128) return CLSA_ERR_UNSUPPORTED;
+  if (p->idx_dim != 64 && p->idx_dim != 128) return CLSA_ERR_UNSUPPORTED;
+  if (p->num_q_heads / p->num_kv_heads > 16) return CLSA_ERR_UNSUPPORTED;
+  return CLSA_OK;
+}
+
+clsa_status check_seq(const clsa_params* p) {
+  if (p->seq_start == nullptr || p->seq_len == nullptr) return CLSA_ERR_INVALID_ARG;
+  if (!aligned(p->seq_start, 8) || !aligned(p->seq_len, 4)) return CLSA_ERR_INVALID_ARG;
+  return CLSA_OK;
+}
+
+clsa_status check_idx_cache(const clsa_params* p) {
+  if (p->idx_k_cache == nullptr || !aligned(p->idx_k_cache, 16)) return CLSA_ERR_INVALID_ARG;
+  if (p->idx_token_stride < p->idx_dim || p->idx_token_stride % 8 != 0) return CLSA_ERR_INVALID_ARG;
+  return CLSA_OK;
+}
+
+clsa_status check_kv_cache(const clsa_params* p) {
+  if (p->k_cache == nullptr || p->v_cache == nullptr) return CLSA_ERR_INVALID_ARG;
+  if (!aligned(p->k_cache, 16) || !aligned(p->v_cache, 16)) return CLSA_ERR_INVALID_ARG;
+  if (p->kv_head_stride < p->head_dim || p->kv_head_stride % 8 != 0) return CLSA_ERR_INVALID_ARG;
+  if (p->kv_token_stride < p->head_dim || p->kv_token_stride % 8 != 0) return CLSA_ERR_INVALID_ARG;
+  return CLSA_OK;
+}
+
+clsa_status check_workspace(const void* ws, size_t ws_bytes, size_t need) {
+  if (ws == nullptr || !aligned(ws, 256) || ws_bytes < need) return CLSA_ERR_WORKSPACE;
+  return CLSA_OK;
+}
+
+#define CLSA_TRY(expr)                     \
+  do {                                     \
+    const clsa_status st__ = (expr);       \
+    if (st__ != CLSA_OK) return st__;      \
+  } while (0)
+
+clsa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? CLSA_OK : CLSA_ERR_CUDA; }
+
+}  // namespace
+}  // namespace clsa
+
+using namespace clsa;
+
+extern "C" {
+
+clsa_status clsa_workspace_bytes(const clsa_params* p, size_t* bytes) {
+  if (bytes == nullptr) return CLSA_ERR_INVALID_ARG;
+  CLSA_TRY(check_shape(p));
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  *bytes = make_workspace_layout(*p, dev).total;
+  return CLSA_OK;
+}
+
+clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* scores, int64_t score_stride,
+                              void* workspace, size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  CLSA_TRY(check_idx_cache(p));
+  if (q_idx == nullptr || scores == nullptr || !aligned(q_idx, 16) || !aligned(scores, 4)) return CLSA_ERR_INVALID_ARG;
+  if (score_stride < p->max_seq_len) return CLSA_ERR_INVALID_ARG;
+  if (p->q_per_seq != 1) return CLSA_ERR_UNSUPPORTED;
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  return from_cuda(launch_index_scores_decode(*p, q_idx, scores, score_stride, static_cast<uint32_t*>(workspace), dev,
+                                              static_cast<cudaStream_t>(stream)));
+}
+
+clsa_status clsa_topk(const clsa_params* p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,
+                      void* workspace, size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  if (scores == nullptr || idx == nullptr || count == nullptr) return CLSA_ERR_INVALID_ARG;
+  if (!aligned(scores, 4) || !aligned(idx, 4) || !aligned(count, 4)) return CLSA_ERR_INVALID_ARG;
+  if (score_stride < p->max_seq_len) return CLSA_ERR_INVALID_ARG;
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  return from_cuda(launch_topk(*p, scores, score_stride, idx, count, static_cast<uint32_t*>(workspace), dev,
+                               static_cast<cudaStream_t>(stream)));
+}
+
+clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t* idx, const int32_t* count, void* out,
+                             float* lse, void* workspace, size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  CLSA_TRY(check_kv_cache(p));
+  if (q == nullptr || idx == nullptr || count == nullptr || out == nullptr) return CLSA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(out, 16) || !aligned(idx, 4) || !aligned(count, 4) || !aligned(lse, 4))
+    return CLSA_ERR_INVALID_ARG;
+  if (workspace == nullptr || !aligned(workspace, 256)) return CLSA_ERR_WORKSPACE;
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  const WorkspaceLayout w = make_workspace_layout(*p, dev);
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, w.partial_off + w.partial_bytes));
+  auto base = static_cast<unsigned char*>(workspace);
+  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, reinterpret_cast<float*>(base + w.partial_off),
+                                      reinterpret_cast<uint32_t*>(base), p->sweep, dev,
+                                      static_cast<cudaStream_t>(stream)));
+}
+
+clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
+                             void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
+                             size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  CLSA_TRY(check_idx_cache(p));
+  CLSA_TRY(check_kv_cache(p));
+  if (q_idx == nullptr || q_layers == nullptr || out_layers == nullptr || idx == nullptr || count == nullptr)
+    return CLSA_ERR_INVALID_ARG;
+  if (!aligned(q_idx, 16) || !aligned(idx, 4) || !aligned(count, 4)) return CLSA_ERR_INVALID_ARG;
+  for (int l = 0; l < p->num_layers; ++l)
+    if (q_layers[l] == nullptr || out_layers[l] == nullptr || !aligned(q_layers[l], 16) || !aligned(out_layers[l], 16))
+      return CLSA_ERR_INVALID_ARG;
+  if (p->q_per_seq != 1) return CLSA_ERR_UNSUPPORTED;
+  if (workspace == nullptr || !aligned(workspace, 256)) return CLSA_ERR_WORKSPACE;
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  const WorkspaceLayout w = make_workspace_layout(*p, dev);
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, w.total));
+  auto base = static_cast<unsigned char*>(workspace);
+  auto status = reinterpret_cast<uint32_t*>(base);
+  auto scores = reinterpret_cast<float*>(base + w.scores_off);
+  auto partials = reinterpret_cast<float*>(base + w.partial_off);
+  auto s = static_cast<cudaStream_t>(stream);
+  cudaError_t err = launch_index_scores_decode(*p, q_idx, scores, w.score_stride, status, dev, s);
+  if (err != cudaSuccess) return CLSA_ERR_CUDA;
+  err = launch_topk(*p, scores, w.score_stride, idx, count, status, dev, s);
+  if (err != cudaSuccess) return CLSA_ERR_CUDA;
+  for (int l = 0; l < p->num_layers; ++l) {
+    // alternate the sweep direction so that a layer starts on the rows its predecessor touched last
+    err = launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, partials, status,
+                             (p->sweep + l) & 1, dev, s);
+    if (err != cudaSuccess) return CLSA_ERR_CUDA;
+  }
+  return CLSA_OK;
+}
+
+clsa_status clsa_clear_status(void* workspace, size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
+  return from_cuda(cudaMemsetAsync(workspace, 0, kStatusBytes, static_cast<cudaStream_t>(stream)));
+}
+
+clsa_status clsa_device_status(const void* workspace, uint32_t* bits, clsa_stream stream) {
+  if (workspace == nullptr || bits == nullptr) return CLSA_ERR_INVALID_ARG;
+  auto s = static_cast<cudaStream_t>(stream);
+  cudaError_t err = cudaMemcpyAsync(bits, workspace, sizeof(uint32_t), cudaMemcpyDeviceToHost, s);
+  if (err == cudaSuccess) err = cudaStreamSynchronize(s);
+  return from_cuda(err);
+}
+
+const char* clsa_status_string(clsa_status s) {
+  switch (s) {
+    case CLSA_OK: return "ok";
+    case CLSA_ERR_INVALID_ARG: return "invalid argument";
+    case CLSA_ERR_UNSUPPORTED: return "unsupported shape";
+    case CLSA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case CLSA_ERR_CUDA: return "CUDA runtime error";
+  }
+  return "unknown status";
+}
+
+int clsa_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,86 @@
+// Shared declarations of the CLSA CUDA library: workspace layout, launch plans, small device helpers.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "clsa.h"
+
+namespace clsa {
+
+// ---------------------------------------------------------------------------------------------
+// Host-side plans
+// ---------------------------------------------------------------------------------------------
+struct DeviceInfo {
+  int sm_count;
+  int max_smem_optin;  // bytes of dynamic shared memory a block may opt in to
+  int l2_bytes;
+};
+// Cached per device (queried once). Returns false if the CUDA runtime reports an error.
+bool device_info(DeviceInfo* out);
+
+constexpr size_t kStatusBytes = 256;   // status word + padding at the start of the workspace
+constexpr int kAttnWarps = 8;          // warps per attention block, each an autonomous worker
+constexpr int kAttnStageTokens = 16;   // tokens per pipeline stage (one PV MMA k-step)
+constexpr int kAttnStages = 3;         // cp.async ring depth per warp
+constexpr int kPartialFloats = 132;    // per (row, span, head): 128 outputs, running max, running sum, pad
+
+// Split of the flattened (query row, selected slot) space over the persistent attention warps.
+struct AttnPlan {
+  int num_blocks;       // persistent blocks (one per SM)
+  int num_spans;        // J: contiguous spans of the slot space, one per group of Hkv warps
+  int64_t span_slots;   // SP: slots per span; a multiple of 16, or of top_k when >= top_k
+  int max_parts;        // partial results per row (1 = spans hold whole rows, no merge launch)
+  size_t partial_bytes; // workspace for the partials (0 when max_parts == 1)
+};
+AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev);
+
+struct TopkPlan {
+  int cluster;      // blocks per (sequence, query) row, a thread-block cluster
+  int slice_cap;    // score slots each block keeps in shared memory (0 = re-read global memory each pass)
+  size_t smem_bytes;
+};
+TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev);
+
+struct WorkspaceLayout {
+  size_t partial_off, partial_bytes;
+  size_t scores_off, scores_bytes;  // used by clsa_decode_step only
+  int64_t score_stride;
+  size_t total;
+};
+WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& dev);
+
+// ---------------------------------------------------------------------------------------------
+// Kernel launchers (each returns the cudaError_t of its launches)
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_index_scores_decode(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
+                                       uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,
+                        uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
+                               float* lse, float* partials, uint32_t* status, int reverse, const DeviceInfo& dev,
+                               cudaStream_t stream);
+
+// ---------------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Round-to-nearest-even fp32 -> bf16 pair packed as (hi << 16) | lo.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+__device__ __forceinline__ void flag_status(uint32_t* status, uint32_t bit) {
+  if (status != nullptr) atomicOr(status, bit);
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+#endif
+
+}  // namespace clsa

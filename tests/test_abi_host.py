@@ -1,0 +1,124 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the header
+declares, the Python struct mirrors the C struct, and invalid calls are refused before any CUDA work."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "clsa.h")
+
+
+@pytest.fixture(scope="module")
+def clsa():
+    sys.path.insert(0, ROOT)
+    import __graft_entry__ as entry
+
+    entry._load_build_module().build()
+    import paper_2606_06467_b200 as mod
+
+    return mod
+
+
+def _declared_functions():
+    text = open(HEADER).read()
+    return sorted(set(re.findall(r"CLSA_API\s+[\w\s\*]+?\b(clsa_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(clsa):
+    names = _declared_functions()
+    assert len(names) == 9 and set(names) == set(clsa.EXPORTS)
+    lib = ctypes.CDLL(clsa.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert clsa.clsa_version() == 100
+    assert clsa.clsa_status_string(0) == "ok" and "unsupported" in clsa.clsa_status_string(2)
+
+
+def test_struct_layout_matches_the_header(clsa, tmp_path):
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "clsa.h"\nint main(void){printf("%zu", sizeof(clsa_params));\n'
+                   + "".join(f'printf(" %zu", offsetof(clsa_params, {f}));\n' for f, _ in clsa.clsa_params._fields_)
+                   + "return 0;}\n")
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    nums = [int(x) for x in subprocess.check_output([str(exe)]).split()]
+    assert nums[0] == ctypes.sizeof(clsa.clsa_params)
+    assert nums[1:] == [getattr(clsa.clsa_params, f).offset for f, _ in clsa.clsa_params._fields_]
+
+
+def _good(clsa, **kw):
+    base = dict(num_seqs=2, num_q_heads=32, num_kv_heads=8, head_dim=128, idx_dim=128, top_k=64, num_layers=2,
+                max_seq_len=1024, sm_scale=0.088, seq_start=0x1000, seq_len=0x2000, k_cache=0x10000, v_cache=0x20000,
+                idx_k_cache=0x30000)
+    base.update(kw)
+    return clsa.make_params(**base)
+
+
+def test_bad_arguments_are_refused_on_the_host(clsa):
+    raw = clsa.raw()
+    n = ctypes.c_size_t(0)
+    P = ctypes.byref
+    assert raw.clsa_workspace_bytes(None, P(n)) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_workspace_bytes(P(_good(clsa)), None) == clsa.CLSA_ERR_INVALID_ARG
+    for kw, want in (
+        (dict(num_seqs=0), clsa.CLSA_ERR_INVALID_ARG), (dict(top_k=0), clsa.CLSA_ERR_INVALID_ARG),
+        (dict(num_q_heads=30), clsa.CLSA_ERR_INVALID_ARG), (dict(causal=2), clsa.CLSA_ERR_INVALID_ARG),
+        (dict(sweep=3), clsa.CLSA_ERR_INVALID_ARG), (dict(max_seq_len=0), clsa.CLSA_ERR_INVALID_ARG),
+        (dict(sm_scale=float("nan")), clsa.CLSA_ERR_INVALID_ARG), (dict(num_layers=0), clsa.CLSA_ERR_INVALID_ARG),
+        (dict(head_dim=64), clsa.CLSA_ERR_UNSUPPORTED), (dict(idx_dim=96), clsa.CLSA_ERR_UNSUPPORTED),
+        (dict(num_q_heads=34, num_kv_heads=2), clsa.CLSA_ERR_UNSUPPORTED),
+    ):
+        assert raw.clsa_workspace_bytes(P(_good(clsa, **kw)), P(n)) == want, kw
+    ws, wsb, st = 0x100000, 1 << 20, None
+    good = _good(clsa)
+    # index scores
+    assert raw.clsa_index_scores(P(good), None, 0x40000, 1024, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_index_scores(P(good), 0x50008, 0x40000, 1024, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG  # q misaligned
+    assert raw.clsa_index_scores(P(good), 0x50000, 0x40000, 1000, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG  # stride < max len
+    assert raw.clsa_index_scores(P(_good(clsa, idx_k_cache=None)), 0x50000, 0x40000, 1024, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_index_scores(P(_good(clsa, idx_token_stride=100)), 0x50000, 0x40000, 1024, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_index_scores(P(_good(clsa, seq_len=None)), 0x50000, 0x40000, 1024, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_index_scores(P(good), 0x50000, 0x40000, 1024, None, wsb, st) == clsa.CLSA_ERR_WORKSPACE
+    assert raw.clsa_index_scores(P(good), 0x50000, 0x40000, 1024, ws + 16, wsb, st) == clsa.CLSA_ERR_WORKSPACE
+    assert raw.clsa_index_scores(P(good), 0x50000, 0x40000, 1024, ws, 8, st) == clsa.CLSA_ERR_WORKSPACE
+    # top-k
+    assert raw.clsa_topk(P(good), None, 1024, 0x60000, 0x70000, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_topk(P(good), 0x40000, 512, 0x60000, 0x70000, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_topk(P(good), 0x40000, 1024, 0x60002, 0x70000, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    # sparse attention
+    assert raw.clsa_sparse_attn(P(good), None, 0x60000, 0x70000, 0x80000, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_sparse_attn(P(_good(clsa, k_cache=0x10004)), 0x50000, 0x60000, 0x70000, 0x80000, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_sparse_attn(P(_good(clsa, kv_head_stride=64)), 0x50000, 0x60000, 0x70000, 0x80000, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_sparse_attn(P(good), 0x50000, 0x60000, 0x70000, 0x80000, None, None, wsb, st) == clsa.CLSA_ERR_WORKSPACE
+    # decode step
+    L = good.num_layers
+    qs = (ctypes.c_void_p * L)(0x50000, 0x51000)
+    outs = (ctypes.c_void_p * L)(0x80000, None)
+    assert raw.clsa_decode_step(P(good), 0x50000, qs, outs, 0x60000, 0x70000, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_decode_step(P(good), 0x50000, None, outs, 0x60000, 0x70000, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_clear_status(None, 0, st) == clsa.CLSA_ERR_WORKSPACE
+    assert raw.clsa_device_status(None, None, st) == clsa.CLSA_ERR_INVALID_ARG
+
+
+def test_binding_raises_with_the_status(clsa):
+    with pytest.raises(clsa.ClsaError) as e:
+        clsa.clsa_workspace_bytes(_good(clsa, head_dim=256))
+    assert e.value.status == clsa.CLSA_ERR_UNSUPPORTED
+
+
+def test_product_does_not_touch_the_oracle():
+    """Neither the binding nor the CUDA sources may import, include or link anything under oracle/."""
+    pkg = os.path.join(ROOT, "paper_2606_06467_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), os.path.join(dirpath, f)
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".c")):
+            text = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2606_06467_b200" not in text and "clsa.h" not in text
