@@ -91,7 +91,8 @@ typedef struct {
 /* Bytes of workspace that any of the calls below may need for these params (the maximum over the
  * four; clsa_decode_step additionally keeps the fp32 score matrix there). Reads only the scalar
  * fields. *bytes is HOST memory. The workspace must be 256-byte aligned; its first 256 bytes hold
- * the device status word and must be zero before the first call (cudaMemset or clsa_clear_status). */
+ * the device status word and must be zero before the first call (cudaMemset or clsa_clear_status).
+ * Calls that overlap on the GPU must not share a workspace. */
 CLSA_API clsa_status clsa_workspace_bytes(const clsa_params* p, size_t* bytes);
 
 /* Eq. 3, first half: scores[b][t][s] = sum_j q_idx[b][t][j] * K_idx[seq_start[b]+s][j] for every

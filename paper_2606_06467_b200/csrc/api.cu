@@ -31,12 +31,10 @@ bool device_info(DeviceInfo* out) {
 }
 
 WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& dev) {
+  (void)dev;
   WorkspaceLayout w;
-  const AttnPlan plan = make_attn_plan(p, dev);
   auto align = [](size_t x) { return (x + 255) / 256 * 256; };
-  w.partial_off = kStatusBytes;
-  w.partial_bytes = align(plan.partial_bytes);
-  w.scores_off = w.partial_off + w.partial_bytes;
+  w.scores_off = kStatusBytes;
   w.score_stride = ((int64_t)p.max_seq_len + 63) / 64 * 64;
   w.scores_bytes = align((size_t)p.num_seqs * p.q_per_seq * w.score_stride * sizeof(float));
   w.total = w.scores_off + w.scores_bytes;
@@ -151,14 +149,10 @@ clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t*
   if (q == nullptr || idx == nullptr || count == nullptr || out == nullptr) return CLSA_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(out, 16) || !aligned(idx, 4) || !aligned(count, 4) || !aligned(lse, 4))
     return CLSA_ERR_INVALID_ARG;
-  if (workspace == nullptr || !aligned(workspace, 256)) return CLSA_ERR_WORKSPACE;
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
-  const WorkspaceLayout w = make_workspace_layout(*p, dev);
-  CLSA_TRY(check_workspace(workspace, workspace_bytes, w.partial_off + w.partial_bytes));
-  auto base = static_cast<unsigned char*>(workspace);
-  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, reinterpret_cast<float*>(base + w.partial_off),
-                                      reinterpret_cast<uint32_t*>(base), p->sweep, dev,
+  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, dev,
                                       static_cast<cudaStream_t>(stream)));
 }
 
@@ -184,7 +178,6 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
   auto base = static_cast<unsigned char*>(workspace);
   auto status = reinterpret_cast<uint32_t*>(base);
   auto scores = reinterpret_cast<float*>(base + w.scores_off);
-  auto partials = reinterpret_cast<float*>(base + w.partial_off);
   auto s = static_cast<cudaStream_t>(stream);
   cudaError_t err = launch_index_scores_decode(*p, q_idx, scores, w.score_stride, status, dev, s);
   if (err != cudaSuccess) return CLSA_ERR_CUDA;
@@ -192,8 +185,8 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
   if (err != cudaSuccess) return CLSA_ERR_CUDA;
   for (int l = 0; l < p->num_layers; ++l) {
     // alternate the sweep direction so that a layer starts on the rows its predecessor touched last
-    err = launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, partials, status,
-                             (p->sweep + l) & 1, dev, s);
+    // alternate the sweep direction so that a layer starts on the rows its predecessor touched last
+    err = launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p->sweep + l) & 1, dev, s);
     if (err != cudaSuccess) return CLSA_ERR_CUDA;
   }
   return CLSA_OK;

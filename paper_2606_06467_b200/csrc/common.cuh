@@ -22,15 +22,14 @@ constexpr size_t kStatusBytes = 256;   // status word + padding at the start of 
 constexpr int kAttnWarps = 8;          // warps per attention block, each an autonomous worker
 constexpr int kAttnStageTokens = 16;   // tokens per pipeline stage (one PV MMA k-step)
 constexpr int kAttnStages = 3;         // cp.async ring depth per warp
-constexpr int kPartialFloats = 132;    // per (row, span, head): 128 outputs, running max, running sum, pad
 
-// Split of the flattened (query row, selected slot) space over the persistent attention warps.
+// Launch shape of the sparse-attention kernel.
 struct AttnPlan {
-  int num_blocks;       // persistent blocks (one per SM)
-  int num_spans;        // J: contiguous spans of the slot space, one per group of Hkv warps
-  int64_t span_slots;   // SP: slots per span; a multiple of 16, or of top_k when >= top_k
-  int max_parts;        // partial results per row (1 = spans hold whole rows, no merge launch)
-  size_t partial_bytes; // workspace for the partials (0 when max_parts == 1)
+  int cluster;          // C: blocks per query row (a thread-block cluster), 1/2/4/8
+  int heads_per_block;  // HC = min(Hkv, 8): KV heads served by one block, one warp each
+  int subs;             // S = 8 / HC: token ranges per block
+  int head_groups;      // ceil(Hkv / HC): grid.y
+  size_t smem_bytes;
 };
 AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev);
 
@@ -42,8 +41,7 @@ struct TopkPlan {
 TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev);
 
 struct WorkspaceLayout {
-  size_t partial_off, partial_bytes;
-  size_t scores_off, scores_bytes;  // used by clsa_decode_step only
+  size_t scores_off, scores_bytes;  // fp32 score matrix of clsa_decode_step
   int64_t score_stride;
   size_t total;
 };
@@ -57,8 +55,7 @@ cudaError_t launch_index_scores_decode(const clsa_params& p, const void* q_idx, 
 cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,
                         uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
-                               float* lse, float* partials, uint32_t* status, int reverse, const DeviceInfo& dev,
-                               cudaStream_t stream);
+                               float* lse, uint32_t* status, int reverse, const DeviceInfo& dev, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------
 // Device helpers

@@ -5,19 +5,29 @@
 // (m16n8k16, fp32 accumulate) with the query heads of one KV head packed into the 16 rows of one
 // tile, far below tensor-pipe capacity.
 //
-// Decomposition. All (query row, selected slot) pairs form one flat slot space of R * k slots
-// (R = B * T query rows). It is cut into J equal spans. A persistent grid of one 8-warp block per
-// SM runs 8 * blocks autonomous warps; warp v serves KV head v % Hkv of span v / Hkv, so the warps
-// of one block walk the same tokens for different KV heads and together fetch each token's whole
-// contiguous [Hkv][D] K row and V row. A warp streams its span in 16-token stages through a
-// private 3-deep cp.async ring (16-byte chunks, XOR-swizzled for conflict-free ldmatrix), runs
-// S = Q K^T, an online softmax in the exp2 domain, and O += P V per stage; there is no block-level
-// barrier anywhere. When spans are shorter than k (decoding) a row is split over several spans:
-// each writes an unnormalised partial (O, max, sum) and a small merge kernel combines them by
-// log-sum-exp. When spans hold whole rows (prefill) outputs are written directly.
-// `reverse` flips the order in which a warp walks its span; alternating it between consecutive
+// Decomposition. One thread-block cluster of C blocks serves one query row (sequence, query
+// token); its selected tokens are cut into C * S contiguous ranges. A block has 8 autonomous
+// warps: warp w serves KV head w % HC of token range w / HC (HC heads per block, S = 8 / HC
+// ranges per block). A warp streams
+// its range in 16-token stages through a private 3-deep cp.async ring (16-byte chunks,
+// XOR-swizzled for conflict-free ldmatrix), runs S = Q K^T, an online softmax in the exp2 domain
+// and O += P V per stage; there is no block-level barrier in the main loop. Split-K merge: every
+// warp leaves its unnormalised partial (O, running max, running sum) in its own shared memory,
+// the cluster synchronises once, and the (KV head, query head) outputs are dealt round-robin to
+// the warps of the cluster, each reading the C * S partials it needs through distributed shared
+// memory and combining them by log-sum-exp. Nothing goes through global memory, nothing spins.
+// The launch shape is chosen per call so that all blocks are resident at once where possible:
+// HC shrinks (down to one KV head per block, its 8 warps splitting the tokens) until
+// rows * Hkv / HC fits the SM count, then C grows while the clusters still fit. Decoding a batch of
+// 16 with 8 KV heads runs 128 single-block clusters whose merge never leaves the block; a prefill
+// chunk runs one block per query row with nothing to merge.
+// `reverse` flips the order in which a warp walks its range; alternating it between consecutive
 // layers makes layer l+1 start on the rows layer l touched last, which are the ones still in L2.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace clsa {
 namespace {
@@ -25,6 +35,8 @@ namespace {
 constexpr int kThreads = kAttnWarps * 32;
 constexpr int kStageBytes = kAttnStageTokens * 256 * 2;  // 16 K rows + 16 V rows of 256 bytes
 constexpr int kWarpRingBytes = kAttnStages * kStageBytes;
+constexpr int kPartialStride = 132;                      // floats per head of a partial: 128 outputs, max, sum, pad
+constexpr int kMergeBatch = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -39,10 +51,9 @@ struct AttnArgs {
   const int32_t* count;
   uint16_t* out;
   float* lse;
-  float* partials;
   uint32_t* status;
-  int64_t num_rows, span_slots;
-  int q_per_seq, num_q_heads, num_kv_heads, group, top_k, num_spans, max_parts, reverse;
+  int q_per_seq, num_q_heads, num_kv_heads, group, top_k;
+  int heads_per_block, subs, reverse;
   float scale_log2;
 };
 
@@ -64,8 +75,8 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
 }
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 // 2^x by the hardware approximation (2 ulp; -inf gives +0).
@@ -75,57 +86,46 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-__device__ __forceinline__ int clamp_count(int c, int top_k, uint32_t* status) {
-  if (c < 0 || c > top_k) {
-    flag_status(status, CLSA_DEV_BAD_COUNT);
-    c = c < 0 ? 0 : top_k;
-  }
-  return c;
-}
-
 __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = (int)cluster.num_blocks();
+  const int crank = (int)cluster.block_rank();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t vwarp = (int64_t)blockIdx.x * kAttnWarps + warp;
-  const int g = (int)(vwarp % a.num_kv_heads);
-  const int64_t span = vwarp / a.num_kv_heads;
-  if (span >= a.num_spans) return;
-  const int64_t total_slots = a.num_rows * a.top_k;
-  const int64_t slot_lo = span * a.span_slots;
-  if (slot_lo >= total_slots) return;
-  const int64_t slot_hi = min(total_slots, slot_lo + a.span_slots);
+  const int64_t r = blockIdx.x / C;                 // query row
+  const int HC = a.heads_per_block, S = a.subs, G = a.group;
+  const int g_local = warp % HC, sub = warp / HC;
+  const int g = blockIdx.y * HC + g_local;          // KV head of this warp
+  const bool active = sub < S && g < a.num_kv_heads;
+  const int nsplit = C * S;                         // token ranges of the row
 
   unsigned char* ring = smem + warp * kWarpRingBytes;
   const uint32_t ring_u32 = smem_u32(ring);
   uint32_t* stage_mask = reinterpret_cast<uint32_t*>(smem + kAttnWarps * kWarpRingBytes) + warp * kAttnStages;
 
-  const int G = a.group;
   const int qrow_a = lane >> 2;        // MMA row (query head within the group) of c0/c1; c2/c3 are row + 8
   const int qcol = (lane & 3) * 2;
+  const int h0 = g * G;                // first query head of this KV head
 
-  const int64_t row_first = slot_lo / a.top_k, row_last = (slot_hi - 1) / a.top_k;
-  const int64_t nrows = row_last - row_first + 1;
-#pragma unroll 1
-  for (int64_t ri = 0; ri < nrows; ++ri) {
-    const int64_t r = a.reverse ? row_last - ri : row_first + ri;
-    const int64_t row_slot0 = r * a.top_k;
-    const int cnt = clamp_count(a.count[r], a.top_k, lane == 0 ? a.status : nullptr);
-    const int t_lo = (int)max((int64_t)0, slot_lo - row_slot0);
-    const int t_hi = (int)min((int64_t)cnt, slot_hi - row_slot0);
-    const bool whole = (slot_lo <= row_slot0) && (slot_hi >= row_slot0 + a.top_k);
-    const int h0 = g * G;  // first query head of this KV head
-    if (t_lo >= t_hi) {
-      if (whole) {  // nothing selected for this row: zeros and lse = -inf
-        for (int e = lane; e < G * 64; e += 32)
-          reinterpret_cast<uint32_t*>(a.out + (r * a.num_q_heads + h0) * 128)[e] = 0u;
-        if (a.lse != nullptr && lane < G) a.lse[r * a.num_q_heads + h0 + lane] = -INFINITY;
-      }
-      continue;
-    }
-    const int b = (int)(r / a.q_per_seq);
-    const int64_t s0 = a.seq_start[b];
-    const int n = a.seq_len[b];
+  // independent loads first: the row's count and the sequence's placement
+  int cnt = a.count[r];
+  const int b = (int)(r / a.q_per_seq);
+  const int64_t s0 = a.seq_start[b];
+  const int n = a.seq_len[b];
+  if (cnt < 0 || cnt > a.top_k) {
+    if (threadIdx.x == 0 && crank == 0 && blockIdx.y == 0) flag_status(a.status, CLSA_DEV_BAD_COUNT);
+    cnt = cnt < 0 ? 0 : a.top_k;
+  }
+  const int per = (((cnt + nsplit - 1) / nsplit) + kAttnStageTokens - 1) / kAttnStageTokens * kAttnStageTokens;
+  const int range = crank * S + sub;
+  const int t_lo = min(cnt, range * per), t_hi = active ? min(cnt, t_lo + per) : t_lo;
 
+  float o[16][4];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) { o[j][0] = 0.f; o[j][1] = 0.f; o[j][2] = 0.f; o[j][3] = 0.f; }
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+  if (t_lo < t_hi) {
     // Query fragments (A operand, 16 x 128): rows >= G are zero padding.
     uint32_t qa[8][4];
     {
@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
     }
 
     const int nstages = (t_hi - t_lo + kAttnStageTokens - 1) / kAttnStageTokens;
-    const int32_t* row_idx = a.idx + row_slot0;
+    const int32_t* row_idx = a.idx + r * a.top_k;
     const uint16_t* kbase = a.kc + g * a.head_stride + (lane & 15) * 8;
     const uint16_t* vbase = a.vc + g * a.head_stride + (lane & 15) * 8;
 
@@ -176,11 +176,6 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
       }
       cp_async_commit();
     };
-
-    float o[16][4];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) { o[j][0] = 0.f; o[j][1] = 0.f; o[j][2] = 0.f; o[j][3] = 0.f; }
-    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
     // prologue: stages 0 .. kAttnStages-2 in flight, positions of the next one in a register
     int next_idx = load_idx(0);
@@ -236,6 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
       const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
       const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
       const float alpha0 = fast_exp2(m0 - mu0), alpha1 = fast_exp2(m1 - mu1);
+      const bool rescale = (mn0 != m0) || (mn1 != m1);
       m0 = mn0;
       m1 = mn1;
       uint32_t pa[4];
@@ -249,8 +245,10 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
         l0 = l0 * alpha0 + (bf16_lo(p00) + bf16_hi(p00)) + (bf16_lo(p10) + bf16_hi(p10));
         l1 = l1 * alpha1 + (bf16_lo(p01) + bf16_hi(p01)) + (bf16_lo(p11) + bf16_hi(p11));
       }
+      if (__any_sync(0xffffffffu, rescale)) {  // the running max moved for some head: rescale the accumulators
 #pragma unroll
-      for (int j = 0; j < 16; ++j) { o[j][0] *= alpha0; o[j][1] *= alpha0; o[j][2] *= alpha1; o[j][3] *= alpha1; }
+        for (int j = 0; j < 16; ++j) { o[j][0] *= alpha0; o[j][1] *= alpha0; o[j][2] *= alpha1; o[j][3] *= alpha1; }
+      }
       // O += P V
 #pragma unroll
       for (int jp = 0; jp < 8; ++jp) {
@@ -268,8 +266,11 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  }
 
-    if (whole) {
+  if (nsplit == 1) {
+    // the warp saw the whole row: normalise and write straight from the accumulators
+    if (active) {
       const float inv0 = l0 > 0.f ? 1.f / l0 : 0.f, inv1 = l1 > 0.f ? 1.f / l1 : 0.f;
       uint16_t* obase = a.out + (r * a.num_q_heads + h0) * 128;
 #pragma unroll
@@ -283,92 +284,136 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
         if (qrow_a < G) a.lse[r * a.num_q_heads + h0 + qrow_a] = l0 > 0.f ? (m0 + log2f(l0)) * kLn2 : -INFINITY;
         if (qrow_a + 8 < G) a.lse[r * a.num_q_heads + h0 + qrow_a + 8] = l1 > 0.f ? (m1 + log2f(l1)) * kLn2 : -INFINITY;
       }
-    } else {
-      const int part = (int)(span - row_slot0 / a.span_slots);
-      float* pbase = a.partials + ((r * a.max_parts + part) * a.num_q_heads + h0) * kPartialFloats;
+    }
+    return;  // uniform over the cluster (a cluster of one block)
+  }
+
+  // ---- split-K merge through distributed shared memory ---------------------------------------------
+  // Each warp parks its partial in its own (now idle) staging ring: [G][kPartialStride] floats.
+  float* mypart = reinterpret_cast<float*>(ring);
+  if (active) {
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        if (qrow_a < G)
-          *reinterpret_cast<float2*>(pbase + qrow_a * kPartialFloats + j * 8 + qcol) = make_float2(o[j][0], o[j][1]);
-        if (qrow_a + 8 < G)
-          *reinterpret_cast<float2*>(pbase + (qrow_a + 8) * kPartialFloats + j * 8 + qcol) = make_float2(o[j][2], o[j][3]);
-      }
-      if ((lane & 3) == 0) {
-        if (qrow_a < G) *reinterpret_cast<float2*>(pbase + qrow_a * kPartialFloats + 128) = make_float2(m0, l0);
-        if (qrow_a + 8 < G) *reinterpret_cast<float2*>(pbase + (qrow_a + 8) * kPartialFloats + 128) = make_float2(m1, l1);
-      }
+    for (int j = 0; j < 16; ++j) {
+      if (qrow_a < G)
+        *reinterpret_cast<float2*>(mypart + qrow_a * kPartialStride + j * 8 + qcol) = make_float2(o[j][0], o[j][1]);
+      if (qrow_a + 8 < G)
+        *reinterpret_cast<float2*>(mypart + (qrow_a + 8) * kPartialStride + j * 8 + qcol) = make_float2(o[j][2], o[j][3]);
+    }
+    if ((lane & 3) == 0) {
+      if (qrow_a < G) *reinterpret_cast<float2*>(mypart + qrow_a * kPartialStride + 128) = make_float2(m0, l0);
+      if (qrow_a + 8 < G) *reinterpret_cast<float2*>(mypart + (qrow_a + 8) * kPartialStride + 128) = make_float2(m1, l1);
     }
   }
+  cluster.sync();
+
+  // Output jobs (KV head of this block's group, query head of the group) dealt over the cluster's warps.
+  const int heads_here = min(HC, a.num_kv_heads - (int)blockIdx.y * HC);
+  const int njobs = heads_here * G;
+  for (int job = crank + C * warp; job < njobs; job += C * kAttnWarps) {
+    const int jg = job / G, hh = job - jg * G;   // local KV head, query head within the group
+    // partial p = (block p / S, range p % S) was left by warp (p % S) * HC + jg of block p / S
+    auto part_ptr = [&](int p) -> const float* {
+      const int c2 = p / S, sub2 = p - c2 * S;
+      return cluster.map_shared_rank(reinterpret_cast<float*>(smem + (sub2 * HC + jg) * kWarpRingBytes), c2) +
+             hh * kPartialStride;
+    };
+    float M = -INFINITY;
+    for (int p = lane; p < nsplit; p += 32) M = fmaxf(M, part_ptr(p)[128]);
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, d));
+    const float mu = M == -INFINITY ? 0.f : M;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    for (int p0 = 0; p0 < nsplit; p0 += 32) {
+      float wl = 0.f;
+      if (p0 + lane < nsplit) {
+        const float2 ml = *reinterpret_cast<const float2*>(part_ptr(p0 + lane) + 128);
+        wl = fast_exp2(ml.x - mu);
+        L += wl * ml.y;
+      }
+      const int chunk_n = min(32, nsplit - p0);
+      for (int q0 = 0; q0 < chunk_n; q0 += kMergeBatch) {
+        float4 v[kMergeBatch];
+#pragma unroll
+        for (int qq = 0; qq < kMergeBatch; ++qq)
+          v[qq] = q0 + qq < chunk_n ? *reinterpret_cast<const float4*>(part_ptr(p0 + q0 + qq) + lane * 4)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int qq = 0; qq < kMergeBatch; ++qq) {
+          const float w = __shfl_sync(0xffffffffu, wl, (q0 + qq) & 31);
+          const float wq = q0 + qq < chunk_n ? w : 0.f;
+          acc.x = fmaf(wq, v[qq].x, acc.x); acc.y = fmaf(wq, v[qq].y, acc.y);
+          acc.z = fmaf(wq, v[qq].z, acc.z); acc.w = fmaf(wq, v[qq].w, acc.w);
+        }
+      }
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) L += __shfl_xor_sync(0xffffffffu, L, d);
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    const int64_t item = r * a.num_q_heads + (int64_t)(blockIdx.y * HC + jg) * G + hh;
+    uint2 packed;
+    packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+    packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2*>(a.out + item * 128 + lane * 4) = packed;
+    if (a.lse != nullptr && lane == 0) a.lse[item] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+  }
+  cluster.sync();  // no block may exit while a neighbour can still read its shared memory
 }
 
-// Log-sum-exp merge of the partials of one (query row, head): one warp each, 4 output values per lane.
-__global__ void __launch_bounds__(256) attn_merge_kernel(const float* __restrict__ partials, const int32_t* __restrict__ count,
-                                                         uint16_t* __restrict__ out, float* __restrict__ lse,
-                                                         int64_t num_rows, int num_q_heads, int top_k, int64_t span_slots,
-                                                         int max_parts) {
-  const int lane = threadIdx.x & 31;
-  const int64_t item = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (item >= num_rows * num_q_heads) return;
-  const int64_t r = item / num_q_heads;
-  const int h = (int)(item % num_q_heads);
-  int cnt = count[r];
-  cnt = cnt < 0 ? 0 : (cnt > top_k ? top_k : cnt);
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  float L = 0.f, M = -INFINITY;
-  if (cnt > 0) {
-    const int64_t slot0 = r * top_k;
-    const int nparts = (int)((slot0 + cnt - 1) / span_slots - slot0 / span_slots) + 1;
-    const float* base = partials + ((r * max_parts) * num_q_heads + h) * kPartialFloats;
-    const int64_t pstride = (int64_t)num_q_heads * kPartialFloats;
-    for (int p = 0; p < nparts; ++p) M = fmaxf(M, base[p * pstride + 128]);
-    const float mu = M == -INFINITY ? 0.f : M;
-    for (int p = 0; p < nparts; ++p) {
-      const float* pp = base + p * pstride;
-      const float w = fast_exp2(pp[128] - mu);
-      const float4 ov = *reinterpret_cast<const float4*>(pp + lane * 4);
-      acc[0] += w * ov.x; acc[1] += w * ov.y; acc[2] += w * ov.z; acc[3] += w * ov.w;
-      L += w * pp[129];
-    }
-  }
-  const float inv = L > 0.f ? 1.f / L : 0.f;
-  uint2 packed;
-  packed.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-  packed.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-  *reinterpret_cast<uint2*>(out + item * 128 + lane * 4) = packed;
-  if (lse != nullptr && lane == 0) lse[item] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+// Blocks of `cluster` that can be resident at once (cached per cluster size; 0 if the query fails).
+static int max_resident_blocks(int cluster, size_t smem_bytes) {
+  static int cache[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+  if (cache[cluster] != 0) return cache[cluster];
+  cudaFuncSetAttribute(sparse_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)cluster * 64, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, sparse_attn_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+  cache[cluster] = n * cluster;
+  return cache[cluster];
 }
 
 }  // namespace
 
 AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev) {
   AttnPlan plan;
+  plan.smem_bytes = (size_t)kAttnWarps * kWarpRingBytes + kAttnWarps * kAttnStages * sizeof(uint32_t);
   const int hkv = p.num_kv_heads;
-  int gcd = hkv, x = kAttnWarps;
-  while (x) { const int tmp = gcd % x; gcd = x; x = tmp; }
-  const int step = hkv / gcd;  // blocks must come in multiples of this so that 8 * blocks % Hkv == 0
-  int blocks = dev.sm_count / step * step;
-  if (blocks < step) blocks = step;
-  plan.num_blocks = blocks;
-  plan.num_spans = (int)((int64_t)blocks * kAttnWarps / hkv);
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
-  const int64_t total = rows * p.top_k;
-  int64_t sp = (total + plan.num_spans - 1) / plan.num_spans;
-  sp = (sp + kAttnStageTokens - 1) / kAttnStageTokens * kAttnStageTokens;
-  if (sp >= p.top_k) {
-    sp = (sp + p.top_k - 1) / p.top_k * p.top_k;  // whole rows per span: outputs are written directly
-    plan.max_parts = 1;
-    plan.partial_bytes = 0;
-  } else {
-    plan.max_parts = (int)((p.top_k + sp - 1) / sp) + 1;
-    plan.partial_bytes = (size_t)rows * plan.max_parts * p.num_q_heads * kPartialFloats * sizeof(float);
-  }
-  plan.span_slots = sp;
+  // Heads per block: as few as it takes for all blocks to be resident at once (more blocks, and the
+  // split over tokens then stays inside a block); all 8 warps on different heads once there are
+  // more rows than SMs.
+  int hc_max = 1;
+  while (hc_max * 2 <= kAttnWarps && hc_max * 2 <= hkv) hc_max *= 2;
+  int hc = 1;
+  while (hc < hc_max && rows * ((hkv + hc - 1) / hc) > dev.sm_count) hc *= 2;
+  // every token range should hold at least one 16-token stage
+  while (hc < hc_max && (int64_t)(kAttnWarps / hc) * kAttnStageTokens > p.top_k) hc *= 2;
+  plan.heads_per_block = hc;
+  plan.subs = kAttnWarps / hc;
+  plan.head_groups = (hkv + hc - 1) / hc;
+  // Cluster: the largest power of two that still keeps every block resident at once.
+  int c = 1;
+  const int64_t blocks = rows * plan.head_groups;
+  while (c < 8 && blocks * (c * 2) <= max_resident_blocks(c * 2, plan.smem_bytes) &&
+         (int64_t)(c * 2) * plan.subs * kAttnStageTokens <= p.top_k)
+    c *= 2;
+  plan.cluster = c;
+  (void)dev;
   return plan;
 }
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
-                               float* lse, float* partials, uint32_t* status, int reverse, const DeviceInfo& dev,
-                               cudaStream_t stream) {
+                               float* lse, uint32_t* status, int reverse, const DeviceInfo& dev, cudaStream_t stream) {
   const AttnPlan plan = make_attn_plan(p, dev);
   AttnArgs a;
   a.q = static_cast<const uint16_t*>(q);
@@ -382,33 +427,32 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.count = count;
   a.out = static_cast<uint16_t*>(out);
   a.lse = lse;
-  a.partials = partials;
   a.status = status;
-  a.num_rows = (int64_t)p.num_seqs * p.q_per_seq;
-  a.span_slots = plan.span_slots;
   a.q_per_seq = p.q_per_seq;
   a.num_q_heads = p.num_q_heads;
   a.num_kv_heads = p.num_kv_heads;
   a.group = p.num_q_heads / p.num_kv_heads;
   a.top_k = p.top_k;
-  a.num_spans = plan.num_spans;
-  a.max_parts = plan.max_parts;
+  a.heads_per_block = plan.heads_per_block;
+  a.subs = plan.subs;
   a.reverse = reverse;
   a.scale_log2 = p.sm_scale * kLog2e;
-  const size_t smem = (size_t)kAttnWarps * kWarpRingBytes + kAttnWarps * kAttnStages * sizeof(uint32_t);
-  cudaError_t err = cudaFuncSetAttribute(sparse_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t err = cudaFuncSetAttribute(sparse_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
-  sparse_attn_kernel<<<plan.num_blocks, kThreads, smem, stream>>>(a);
-  err = cudaGetLastError();
-  if (err != cudaSuccess) return err;
-  if (plan.max_parts > 1) {
-    const int64_t items = a.num_rows * p.num_q_heads;
-    const int64_t blocks = (items + 7) / 8;
-    attn_merge_kernel<<<(unsigned)blocks, 256, 0, stream>>>(partials, count, a.out, lse, a.num_rows, p.num_q_heads,
-                                                            p.top_k, plan.span_slots, plan.max_parts);
-    err = cudaGetLastError();
-  }
-  return err;
+  const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(rows * plan.cluster), (unsigned)plan.head_groups, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = plan.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)plan.cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, sparse_attn_kernel, a);
 }
 
 }  // namespace clsa
