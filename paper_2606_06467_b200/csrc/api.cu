@@ -152,7 +152,7 @@ clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t*
   CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
-  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, dev,
+  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, 1, dev,
                                       static_cast<cudaStream_t>(stream)));
 }
 
@@ -186,7 +186,11 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
   for (int l = 0; l < p->num_layers; ++l) {
     // alternate the sweep direction so that a layer starts on the rows its predecessor touched last
     // alternate the sweep direction so that a layer starts on the rows its predecessor touched last
-    err = launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p->sweep + l) & 1, dev, s);
+    // Layer 0 follows the top-k kernel and must wait for its index; every later layer reads only what
+    // was complete before its predecessor started (the index, the caches, the caller's queries), so it
+    // may overlap its predecessor's tail.
+    err = launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p->sweep + l) & 1,
+                             l == 0 ? 1 : 0, dev, s);
     if (err != cudaSuccess) return CLSA_ERR_CUDA;
   }
   return CLSA_OK;

@@ -54,6 +54,7 @@ struct AttnArgs {
   uint32_t* status;
   int q_per_seq, num_q_heads, num_kv_heads, group, top_k;
   int heads_per_block, subs, reverse;
+  int wait_prior;  // 1: inputs may come from the kernel launched just before this one (wait for it first)
   float scale_log2;
 };
 
@@ -107,18 +108,34 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   const int qcol = (lane & 3) * 2;
   const int h0 = g * G;                // first query head of this KV head
 
-  // independent loads first: the row's count and the sequence's placement
+  // Programmatic dependent launch: let the next kernel of the stream start its own prologue as soon
+  // as SMs free up, and (unless the caller vouches that every input predates the previous kernel)
+  // wait for the previous kernel's results before the first global read.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (a.wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // The row's k slots are cut into nsplit ranges of `per` slots (a multiple of the stage size); the
+  // split does not depend on the row's count, so the first positions can be fetched together with it.
+  const int per = (((a.top_k + nsplit - 1) / nsplit) + kAttnStageTokens - 1) / kAttnStageTokens * kAttnStageTokens;
+  const int range = crank * S + sub;
+  const int slot_lo = min(a.top_k, range * per), slot_hi = min(a.top_k, slot_lo + per);
+  const int32_t* row_idx = a.idx + r * a.top_k;
   int cnt = a.count[r];
   const int b = (int)(r / a.q_per_seq);
   const int64_t s0 = a.seq_start[b];
   const int n = a.seq_len[b];
+  // speculative fetch of the first/last 16 positions of the range (entries past the count are unused)
+  int first_idx = -1;
+  if (active && lane < kAttnStageTokens) {
+    const int nst = (slot_hi - slot_lo + kAttnStageTokens - 1) / kAttnStageTokens;
+    const int tt = slot_lo + (a.reverse ? (nst - 1) * kAttnStageTokens : 0) + lane;
+    if (tt < slot_hi) first_idx = row_idx[tt];
+  }
   if (cnt < 0 || cnt > a.top_k) {
     if (threadIdx.x == 0 && crank == 0 && blockIdx.y == 0) flag_status(a.status, CLSA_DEV_BAD_COUNT);
     cnt = cnt < 0 ? 0 : a.top_k;
   }
-  const int per = (((cnt + nsplit - 1) / nsplit) + kAttnStageTokens - 1) / kAttnStageTokens * kAttnStageTokens;
-  const int range = crank * S + sub;
-  const int t_lo = min(cnt, range * per), t_hi = active ? min(cnt, t_lo + per) : t_lo;
+  const int t_lo = min(cnt, slot_lo), t_hi = active ? min(cnt, slot_hi) : t_lo;
 
   float o[16][4];
 #pragma unroll
@@ -142,7 +159,6 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
     }
 
     const int nstages = (t_hi - t_lo + kAttnStageTokens - 1) / kAttnStageTokens;
-    const int32_t* row_idx = a.idx + r * a.top_k;
     const uint16_t* kbase = a.kc + g * a.head_stride + (lane & 15) * 8;
     const uint16_t* vbase = a.vc + g * a.head_stride + (lane & 15) * 8;
 
@@ -178,7 +194,12 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
     };
 
     // prologue: stages 0 .. kAttnStages-2 in flight, positions of the next one in a register
-    int next_idx = load_idx(0);
+    int next_idx;
+    if (t_hi == slot_hi) {  // the range is entirely below the count: the speculative fetch was step 0
+      next_idx = first_idx;
+    } else {
+      next_idx = load_idx(0);
+    }
 #pragma unroll
     for (int i = 0; i < kAttnStages - 1; ++i) {
       const int cur = next_idx;
@@ -413,7 +434,8 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev) {
 }
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
-                               float* lse, uint32_t* status, int reverse, const DeviceInfo& dev, cudaStream_t stream) {
+                               float* lse, uint32_t* status, int reverse, int wait_prior, const DeviceInfo& dev,
+                               cudaStream_t stream) {
   const AttnPlan plan = make_attn_plan(p, dev);
   AttnArgs a;
   a.q = static_cast<const uint16_t*>(q);
@@ -436,6 +458,7 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.heads_per_block = plan.heads_per_block;
   a.subs = plan.subs;
   a.reverse = reverse;
+  a.wait_prior = wait_prior;
   a.scale_log2 = p.sm_scale * kLog2e;
   cudaError_t err = cudaFuncSetAttribute(sparse_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
@@ -445,13 +468,15 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)plan.cluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, sparse_attn_kernel, a);
 }
 
