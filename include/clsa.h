@@ -133,6 +133,31 @@ CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, c
                              void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
                              size_t workspace_bytes, clsa_stream stream);
 
+/* The same step as clsa_decode_step for callers that cannot allocate device memory. (The paper has
+ * no counterpart: this is a convenience of the library.) Some callers have no way to obtain a
+ * workspace: code that runs inside a region where cudaMalloc is forbidden or would synchronise the
+ * device (a latency-critical serving loop, a plug-in that is handed tensors but no allocator, a
+ * process whose memory pool is already fully reserved). For them the scratch that clsa_decode_step
+ * keeps in the caller's workspace -- the status word and the fp32 score matrix -- lives in a
+ * device array built into the library: 8 MiB + 256 bytes per GPU that loads the library, held until
+ * the process exits. This entry point calls no cudaMalloc, cudaFree or any other allocating routine.
+ *   Limit: num_seqs * round_up(max_seq_len, 64) <= 2 097 152 scores (for example 16 sequences of
+ *     131 072 tokens); larger shapes return CLSA_ERR_WORKSPACE and launch nothing. T must be 1.
+ *   dev_status: DEVICE pointer to one uint32 owned by the caller that receives the CLSA_DEV_* bits
+ *     (the caller zeroes it), or NULL to drop them into the built-in array's own word, which the
+ *     call then clears first.
+ *   First call on a device: looks up the array's device address (once per device, with that device
+ *     current). Make this first call outside any stream capture.
+ *   Sharing: every call on a GPU uses the same array, which still holds the previous call's
+ *     scores. Nothing needs to be cleared between calls except the status word, which the call does
+ *     itself; but two calls whose GPU work overlaps (different streams, or different threads) race
+ *     on the scores and give wrong indices. Serialise them, or use clsa_decode_step with one
+ *     workspace per stream.
+ * All other arguments, results and error behaviour are those of clsa_decode_step. */
+CLSA_API clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, const void* const* q_layers,
+                                             void* const* out_layers, int32_t* idx, int32_t* count,
+                                             uint32_t* dev_status, clsa_stream stream);
+
 /* Zero the status word (asynchronous, on `stream`). */
 CLSA_API clsa_status clsa_clear_status(void* workspace, size_t workspace_bytes, clsa_stream stream);
 

@@ -47,17 +47,18 @@ _lib.clsa_index_scores.argtypes = [_P, _vp, _vp, _i64, _vp, _sz, _vp]
 _lib.clsa_topk.argtypes = [_P, _vp, _i64, _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_sparse_attn.argtypes = [_P, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_decode_step.argtypes = [_P, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _vp, _vp, _sz, _vp]
+_lib.clsa_decode_step_static.argtypes = [_P, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _vp, _vp, _vp]
 _lib.clsa_clear_status.argtypes = [_vp, _sz, _vp]
 _lib.clsa_device_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32), _vp]
 _lib.clsa_status_string.argtypes = [ctypes.c_int]
 _lib.clsa_status_string.restype = ctypes.c_char_p
 _lib.clsa_version.restype = ctypes.c_int
 for _name in ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_decode_step",
-              "clsa_clear_status", "clsa_device_status"):
+              "clsa_decode_step_static", "clsa_clear_status", "clsa_device_status"):
     getattr(_lib, _name).restype = ctypes.c_int
 
 EXPORTS = ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_decode_step",
-           "clsa_clear_status", "clsa_device_status", "clsa_status_string", "clsa_version")
+           "clsa_decode_step_static", "clsa_clear_status", "clsa_device_status", "clsa_status_string", "clsa_version")
 
 
 class ClsaError(RuntimeError):
@@ -148,6 +149,20 @@ def clsa_decode_step(p, q_idx, q_layers, out_layers, idx, count, workspace, work
     outs = (_vp * L)(*[_ptr(t) for t in out_layers])
     _check(_lib.clsa_decode_step(ctypes.byref(p), _ptr(q_idx), qs, outs, _ptr(idx), _ptr(count), _ptr(workspace),
                                  _nbytes(workspace, workspace_bytes), _stream(stream)), "clsa_decode_step")
+
+
+def clsa_decode_step_static(p, q_idx, q_layers, out_layers, idx, count, dev_status=None, stream=None) -> None:
+    """clsa_decode_step for callers that cannot allocate: its scratch (status word and fp32 scores) is a fixed
+    8 MiB array inside the library, shared by every call on the GPU, so no workspace is passed. Shapes with more
+    than 2 Mi score slots raise ClsaError(CLSA_ERR_WORKSPACE). Calls must not overlap on the GPU; make the first
+    call on a device outside stream capture. `dev_status`: optional caller-owned uint32 device tensor."""
+    L = p.num_layers
+    if len(q_layers) != L or len(out_layers) != L:
+        raise ValueError("q_layers and out_layers must have num_layers entries")
+    qs = (_vp * L)(*[_ptr(t) for t in q_layers])
+    outs = (_vp * L)(*[_ptr(t) for t in out_layers])
+    _check(_lib.clsa_decode_step_static(ctypes.byref(p), _ptr(q_idx), qs, outs, _ptr(idx), _ptr(count),
+                                        _ptr(dev_status), _stream(stream)), "clsa_decode_step_static")
 
 
 def clsa_clear_status(workspace, workspace_bytes=None, stream=None) -> None:

@@ -196,6 +196,70 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
   return CLSA_OK;
 }
 
+// ---- entry point that allocates nothing -----------------------------------------------------------
+// Scratch of clsa_decode_step_static: the status word followed by the fp32 score matrix, in a
+// file-scope device array that every GPU loading this library keeps until the process exits.
+namespace {
+constexpr size_t kStaticScoreSlots = (size_t)2 << 20;  // 2 Mi fp32 scores = 8 MiB
+constexpr size_t kStaticScratchBytes = kStatusBytes + kStaticScoreSlots * sizeof(float);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address: the real
+// address is asked for once per device, with that device current, and cached.
+cudaError_t static_scratch_address(unsigned char** out) {
+  static std::mutex mu;
+  static unsigned char* addr[64] = {};
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  if (addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    err = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (err != cudaSuccess) return err;
+    addr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  *out = addr[dev];
+  return cudaSuccess;
+}
+}  // namespace
+
+clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, const void* const* q_layers,
+                                    void* const* out_layers, int32_t* idx, int32_t* count, uint32_t* dev_status,
+                                    clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  CLSA_TRY(check_idx_cache(p));
+  CLSA_TRY(check_kv_cache(p));
+  if (q_idx == nullptr || q_layers == nullptr || out_layers == nullptr || idx == nullptr || count == nullptr)
+    return CLSA_ERR_INVALID_ARG;
+  if (!aligned(q_idx, 16) || !aligned(idx, 4) || !aligned(count, 4) || !aligned(dev_status, 4)) return CLSA_ERR_INVALID_ARG;
+  for (int l = 0; l < p->num_layers; ++l)
+    if (q_layers[l] == nullptr || out_layers[l] == nullptr || !aligned(q_layers[l], 16) || !aligned(out_layers[l], 16))
+      return CLSA_ERR_INVALID_ARG;
+  if (p->q_per_seq != 1) return CLSA_ERR_UNSUPPORTED;
+  const int64_t stride = ((int64_t)p->max_seq_len + 63) / 64 * 64;
+  if ((uint64_t)p->num_seqs * (uint64_t)stride > kStaticScoreSlots) return CLSA_ERR_WORKSPACE;  // beyond the fixed scratch
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  unsigned char* base = nullptr;
+  if (static_scratch_address(&base) != cudaSuccess) return CLSA_ERR_CUDA;
+  auto s = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left: the status word must start at zero. The score
+  // matrix needs no clearing (every entry that is read is written first).
+  uint32_t* status = dev_status != nullptr ? dev_status : reinterpret_cast<uint32_t*>(base);
+  if (dev_status == nullptr && cudaMemsetAsync(base, 0, kStatusBytes, s) != cudaSuccess) return CLSA_ERR_CUDA;
+  auto scores = reinterpret_cast<float*>(base + kStatusBytes);
+  if (launch_index_scores_decode(*p, q_idx, scores, stride, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
+  if (launch_topk(*p, scores, stride, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
+  for (int l = 0; l < p->num_layers; ++l)
+    if (launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p->sweep + l) & 1,
+                           l == 0 ? 1 : 0, dev, s) != cudaSuccess)
+      return CLSA_ERR_CUDA;
+  return CLSA_OK;
+}
+
 clsa_status clsa_clear_status(void* workspace, size_t workspace_bytes, clsa_stream stream) {
   CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
   return from_cuda(cudaMemsetAsync(workspace, 0, kStatusBytes, static_cast<cudaStream_t>(stream)));
