@@ -2,12 +2,16 @@
 //
 // One thread-block cluster per (sequence, query) row. The row's visible scores are cut into
 // contiguous slices, one per block; each block converts its slice once to order-preserving 32-bit
-// keys held in shared memory, so the four 8-bit radix passes never go back to global memory.
-// Per pass every warp histograms into its own 256-bin shared-memory histogram, the block folds the
-// warp histograms, and the blocks of the cluster read each other's folded histogram through
-// distributed shared memory; every block then finds, redundantly and identically, the digit bin
-// that contains the k-th largest key. After four passes the exact threshold key and the number of
-// threshold-equal elements still needed are known. The compaction is index-ordered: a block's
+// keys held in shared memory, so the radix passes never go back to global memory. Three passes
+// resolve 12 + 12 + 8 key bits. fp32 scores crowd into a few sign/exponent patterns, so a wide
+// first digit (sign, exponent and three mantissa bits) is what keeps the shared-memory histogram
+// atomics from serialising on a handful of bins; a warp whose lanes all hit one bin adds once.
+// Per pass: each block histograms its slice into shared memory, then adds its non-empty bins into
+// every block's copy of the cluster-wide histogram with distributed-shared-memory atomics; after
+// one cluster barrier every block scans its own copy from the top bin down and finds, redundantly
+// and identically, the digit that contains the k-th largest key (the copies are double-buffered,
+// so one barrier per pass is enough). After three passes the exact threshold key and the number
+// of threshold-equal elements still needed are known. The compaction is index-ordered: a block's
 // output offset is the number of selected elements in lower-ranked blocks, a warp's offset the
 // number selected in lower warps, so positions come out ascending and, among keys equal to the
 // threshold, the lowest positions win. No atomics touch global memory and nothing spins.
@@ -20,18 +24,17 @@ namespace cg = cooperative_groups;
 namespace clsa {
 namespace {
 
-constexpr int kThreads = 1024;
+constexpr int kThreads = 512;  // 512 threads and < 113 KiB of shared memory: two blocks per SM, so that 16+ clusters of 8 are resident at once
 constexpr int kWarps = kThreads / 32;
-constexpr int kBins = 256;
-constexpr int kHistStride = kBins + 1;  // odd stride: equal bins of different warps fall in different banks
+constexpr int kMaxBins = 4096;
 constexpr int kMaxCluster = 8;
 
 struct Shared {
-  uint32_t warp_hist[kWarps * kHistStride];
-  uint32_t block_hist[2][kBins];   // double-buffered: read remotely by the other blocks of the cluster
-  uint32_t global_hist[kBins];
+  uint32_t local_hist[kMaxBins];       // this block's slice
+  uint32_t cluster_hist[2][kMaxBins];  // whole row, one copy per block, filled by every block of the cluster
+  uint32_t warp_tot[kWarps];
   uint32_t warp_gt[kWarps], warp_eq[kWarps];
-  uint32_t block_gt_eq[2];         // read remotely
+  uint32_t block_gt_eq[2];             // read remotely
   uint32_t digit, k_rem;
   uint32_t out_base, eq_base;
 };
@@ -42,10 +45,94 @@ __device__ __forceinline__ uint32_t score_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// One radix pass over `BITS` key bits starting at `shift`. On return prefix/prefix_mask/k_rem are
+// updated. `buf` selects the cluster_hist copy (alternates between passes).
+template <int BITS, typename KeyAt>
+__device__ __forceinline__ void radix_pass(Shared& sh, cg::cluster_group& cluster, int nblk, int cnt, int shift, int buf,
+                                           uint32_t& prefix, uint32_t& prefix_mask, uint32_t& k_rem, KeyAt key_at) {
+  constexpr int NB = 1 << BITS;
+  constexpr int PT = (NB + kThreads - 1) / kThreads;  // bins per thread
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int i = tid; i < NB; i += kThreads) sh.local_hist[i] = 0;
+  __syncthreads();
+  for (int i0 = 0; i0 < cnt; i0 += kThreads) {
+    const int i = i0 + tid;
+    const uint32_t key = i < cnt ? key_at(i) : 0u;
+    const bool in = i < cnt && (key & prefix_mask) == prefix;
+    const uint32_t bin = (key >> shift) & (uint32_t)(NB - 1);
+    const uint32_t voters = __ballot_sync(0xffffffffu, in);
+    if (voters == 0u) continue;
+    // all participating lanes on one bin (long runs of equal scores): one add for the warp
+    const uint32_t lead_bin = __shfl_sync(0xffffffffu, bin, __ffs(voters) - 1);
+    const bool same = __all_sync(0xffffffffu, !in || bin == lead_bin);
+    if (same) {
+      if (lane == __ffs(voters) - 1) atomicAdd(&sh.local_hist[bin], (uint32_t)__popc(voters));
+    } else if (in) {
+      atomicAdd(&sh.local_hist[bin], 1u);
+    }
+  }
+  __syncthreads();
+  // add this block's non-empty bins into every block's copy of the row histogram
+  uint32_t* mine = sh.cluster_hist[buf];
+#pragma unroll
+  for (int j = 0; j < PT; ++j) {
+    const int bin = tid + j * kThreads;
+    if (bin < NB) {
+      const uint32_t v = sh.local_hist[bin];
+      if (v != 0u)
+        for (int r = 0; r < nblk; ++r) atomicAdd(cluster.map_shared_rank(mine, r) + bin, v);
+    }
+  }
+  cluster.sync();
+  // scan this block's copy from the top bin down: thread t owns bins NB-1-(t*PT+j)
+  uint32_t own[PT];
+  uint32_t tot = 0;
+#pragma unroll
+  for (int j = 0; j < PT; ++j) {
+    const int pos = tid * PT + j;
+    own[j] = pos < NB ? mine[NB - 1 - pos] : 0u;
+    tot += own[j];
+  }
+  uint32_t incl = tot;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += up;
+  }
+  if (lane == 31) sh.warp_tot[warp] = incl;
+  __syncthreads();
+  uint32_t before = 0;
+  for (int w = 0; w < warp; ++w) before += sh.warp_tot[w];
+  incl += before;
+  const uint32_t excl = incl - tot;
+  if (excl < k_rem && k_rem <= incl) {
+    uint32_t acc = excl;
+#pragma unroll
+    for (int j = 0; j < PT; ++j) {
+      if (acc < k_rem && k_rem <= acc + own[j]) {
+        sh.digit = (uint32_t)(NB - 1 - (tid * PT + j));
+        sh.k_rem = k_rem - acc;
+      }
+      acc += own[j];
+    }
+  }
+  // clear the copy for its next use (two passes on); nobody else touches it before the next barrier
+#pragma unroll
+  for (int j = 0; j < PT; ++j) {
+    const int pos = tid * PT + j;
+    if (pos < NB) mine[NB - 1 - pos] = 0u;
+  }
+  __syncthreads();
+  prefix |= sh.digit << shift;
+  prefix_mask |= (uint32_t)(NB - 1) << shift;
+  k_rem = sh.k_rem;
+}
+
 template <bool CACHED>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const int32_t* __restrict__ seq_len,
-                  int q_per_seq, int causal, int top_k, int max_seq_len, int slice_cap, int32_t* __restrict__ idx_out,
+                  int q_per_seq, int causal, int top_k, int max_seq_len, int32_t* __restrict__ idx_out,
                   int32_t* __restrict__ count_out, uint32_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
@@ -83,64 +170,16 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
     for (int i = tid; i < cnt; i += kThreads) keys[i] = score_key(src[i]);
   }
   auto key_at = [&](int i) -> uint32_t { return CACHED ? keys[i] : score_key(src[i]); };
-  __syncthreads();
+  for (int i = tid; i < 2 * kMaxBins; i += kThreads) (&sh.cluster_hist[0][0])[i] = 0;
+  // the remote adds of pass 0 may arrive as soon as a neighbour gets there: every block must have
+  // cleared its copies first
+  cluster.sync();
 
-  // ---- four radix passes -------------------------------------------------------------------
+  // ---- three radix passes: bits 31..20, 19..8, 7..0 --------------------------------------------
   uint32_t prefix = 0, prefix_mask = 0, k_rem = (uint32_t)kk;
-#pragma unroll 1
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    for (int i = tid; i < kWarps * kHistStride; i += kThreads) sh.warp_hist[i] = 0;
-    __syncthreads();
-    uint32_t* my_hist = sh.warp_hist + warp * kHistStride;
-    for (int i = tid; i < cnt; i += kThreads) {
-      const uint32_t key = key_at(i);
-      if ((key & prefix_mask) == prefix) atomicAdd(&my_hist[(key >> shift) & 0xffu], 1u);
-    }
-    __syncthreads();
-    uint32_t* bh = sh.block_hist[pass & 1];
-    if (tid < kBins) {
-      uint32_t s = 0;
-#pragma unroll 8
-      for (int w = 0; w < kWarps; ++w) s += sh.warp_hist[w * kHistStride + tid];
-      bh[tid] = s;
-    }
-    cluster.sync();
-    if (tid < kBins) {
-      uint32_t s = 0;
-      for (int r = 0; r < nblk; ++r) s += cluster.map_shared_rank(bh, r)[tid];
-      sh.global_hist[tid] = s;
-    }
-    __syncthreads();
-    if (warp == 0) {
-      // lane l owns bins 255-8l .. 248-8l, scanned from the top bin down
-      uint32_t own = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) own += sh.global_hist[255 - 8 * lane - j];
-      uint32_t incl = own;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += up;
-      }
-      const uint32_t excl = incl - own;
-      if (excl < k_rem && k_rem <= incl) {
-        uint32_t acc = excl;
-        for (int j = 0; j < 8; ++j) {
-          const int bin = 255 - 8 * lane - j;
-          const uint32_t c = sh.global_hist[bin];
-          if (acc + c >= k_rem) { sh.digit = (uint32_t)bin; sh.k_rem = k_rem - acc; break; }
-          acc += c;
-        }
-      }
-    }
-    __syncthreads();
-    prefix |= sh.digit << shift;
-    prefix_mask |= 0xffu << shift;
-    k_rem = sh.k_rem;
-    // block_hist is double-buffered, so the next pass may start without a second cluster barrier:
-    // buffer (pass & 1) is rewritten only in pass + 2, after the cluster.sync() of pass + 1.
-  }
+  radix_pass<12>(sh, cluster, nblk, cnt, 20, 0, prefix, prefix_mask, k_rem, key_at);
+  radix_pass<12>(sh, cluster, nblk, cnt, 8, 1, prefix, prefix_mask, k_rem, key_at);
+  radix_pass<8>(sh, cluster, nblk, cnt, 0, 0, prefix, prefix_mask, k_rem, key_at);
   const uint32_t thr = prefix;        // key of the kk-th largest element
   const uint32_t need_eq = k_rem;     // how many threshold-equal elements are selected (>= 1)
 
@@ -161,7 +200,7 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
   if (lane == 0) { sh.warp_gt[warp] = gt; sh.warp_eq[warp] = eq; }
   __syncthreads();
   if (warp == 0) {
-    uint32_t g = sh.warp_gt[lane], e = sh.warp_eq[lane];
+    uint32_t g = lane < kWarps ? sh.warp_gt[lane] : 0u, e = lane < kWarps ? sh.warp_eq[lane] : 0u;
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {
       g += __shfl_xor_sync(0xffffffffu, g, d);
@@ -255,7 +294,7 @@ cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, scores, score_stride, p.seq_len, (int)p.q_per_seq, (int)p.causal,
-                            (int)p.top_k, (int)p.max_seq_len, plan.slice_cap, idx, count, status);
+                            (int)p.top_k, (int)p.max_seq_len, idx, count, status);
 }
 
 }  // namespace clsa
