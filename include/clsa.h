@@ -61,6 +61,7 @@ typedef enum {
 #define CLSA_DEV_BAD_INDEX 1u   /* an idx entry < 0 or >= seq_len inside the first `count` entries: skipped */
 #define CLSA_DEV_BAD_SEQLEN 2u  /* seq_len[b] < q_per_seq or > max_seq_len: that sequence was skipped */
 #define CLSA_DEV_BAD_COUNT 4u   /* count[b,t] < 0 or > top_k: clamped */
+#define CLSA_DEV_TIMEOUT 8u     /* a bounded wait inside a kernel ran out; the kernel returned early, results are invalid */
 
 typedef void* clsa_stream; /* a cudaStream_t */
 
@@ -86,6 +87,8 @@ typedef struct {
   int64_t kv_head_stride;   /* multiple of 8 */
   const void* idx_k_cache;  /* bf16 [rows][d_idx]; element (r,j) at r*idx_token_stride + j */
   int64_t idx_token_stride; /* multiple of 8 */
+  int64_t num_cache_rows;   /* rows of the cache row space (the extent of idx_k_cache); required when q_per_seq > 1,
+                               where tiled bulk copies need the bound; ignored (may be 0) when q_per_seq == 1 */
 } clsa_params;
 
 /* Bytes of workspace that any of the calls below may need for these params (the maximum over the
@@ -100,7 +103,9 @@ CLSA_API clsa_status clsa_workspace_bytes(const clsa_params* p, size_t* bytes);
  * exact in fp32; accumulation is fp32. Entries at s >= visible(b,t) are not written.
  *   q_idx  bf16 [B][T][d_idx], 16-byte aligned
  *   scores fp32 [B][T][score_stride], score_stride >= max_seq_len
- * T == 1 streams the indexer-key cache once (HBM-bound); T > 1 is a tensor-core GEMM. */
+ * T == 1 streams the indexer-key cache once (HBM-bound); T > 1 is a tensor-core GEMM (tcgen05, operands staged by
+ * TMA), which needs p->num_cache_rows and, for 32-byte vector stores, a 32-byte aligned `scores` with
+ * score_stride % 8 == 0 (otherwise it falls back to scalar stores of the same values). */
 CLSA_API clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* scores, int64_t score_stride,
                               void* workspace, size_t workspace_bytes, clsa_stream stream);
 

@@ -15,7 +15,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libclsa.so")
 
 CLSA_OK, CLSA_ERR_INVALID_ARG, CLSA_ERR_UNSUPPORTED, CLSA_ERR_WORKSPACE, CLSA_ERR_CUDA = range(5)
-CLSA_DEV_BAD_INDEX, CLSA_DEV_BAD_SEQLEN, CLSA_DEV_BAD_COUNT = 1, 2, 4
+CLSA_DEV_BAD_INDEX, CLSA_DEV_BAD_SEQLEN, CLSA_DEV_BAD_COUNT, CLSA_DEV_TIMEOUT = 1, 2, 4, 8
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -36,7 +36,7 @@ class clsa_params(ctypes.Structure):
         ("seq_start", ctypes.c_void_p), ("seq_len", ctypes.c_void_p),
         ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
         ("kv_token_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64),
-        ("idx_k_cache", ctypes.c_void_p), ("idx_token_stride", ctypes.c_int64),
+        ("idx_k_cache", ctypes.c_void_p), ("idx_token_stride", ctypes.c_int64), ("num_cache_rows", ctypes.c_int64),
     ]
 
 
@@ -99,7 +99,8 @@ def _nbytes(ws, ws_bytes):
 
 def make_params(*, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim=128, idx_dim, top_k, num_layers=1,
                 causal=0, max_seq_len, sm_scale, sweep=0, seq_start=None, seq_len=None, k_cache=None, v_cache=None,
-                kv_token_stride=None, kv_head_stride=None, idx_k_cache=None, idx_token_stride=None) -> clsa_params:
+                kv_token_stride=None, kv_head_stride=None, idx_k_cache=None, idx_token_stride=None,
+                num_cache_rows=None) -> clsa_params:
     """Fill a clsa_params. Tensor arguments contribute their device address (and, for the caches, their strides
     unless given); the caller keeps them alive while the struct is in use."""
     p = clsa_params()
@@ -115,6 +116,9 @@ def make_params(*, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim=12
     p.kv_token_stride = kv_token_stride if kv_token_stride is not None else num_kv_heads * head_dim
     p.kv_head_stride = kv_head_stride if kv_head_stride is not None else head_dim
     p.idx_token_stride = idx_token_stride if idx_token_stride is not None else idx_dim
+    if num_cache_rows is None and idx_k_cache is not None and not isinstance(idx_k_cache, int):
+        num_cache_rows = idx_k_cache.shape[0]
+    p.num_cache_rows = num_cache_rows or 0
     return p
 
 

@@ -119,10 +119,17 @@ clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* sc
   CLSA_TRY(check_idx_cache(p));
   if (q_idx == nullptr || scores == nullptr || !aligned(q_idx, 16) || !aligned(scores, 4)) return CLSA_ERR_INVALID_ARG;
   if (score_stride < p->max_seq_len) return CLSA_ERR_INVALID_ARG;
-  if (p->q_per_seq != 1) return CLSA_ERR_UNSUPPORTED;
+  if (p->q_per_seq > 1) {
+    // the GEMM path addresses rows through 32-bit TMA coordinates and needs the extent of the cache
+    if (p->num_cache_rows < 1 || p->num_cache_rows > 0x7fffffffLL) return CLSA_ERR_INVALID_ARG;
+    if ((int64_t)p->num_seqs * p->q_per_seq > 0x7fffffffLL) return CLSA_ERR_INVALID_ARG;
+  }
   CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  if (p->q_per_seq > 1)
+    return from_cuda(launch_index_scores_gemm(*p, q_idx, scores, score_stride, static_cast<uint32_t*>(workspace), dev,
+                                              static_cast<cudaStream_t>(stream)));
   return from_cuda(launch_index_scores_decode(*p, q_idx, scores, score_stride, static_cast<uint32_t*>(workspace), dev,
                                               static_cast<cudaStream_t>(stream)));
 }

@@ -52,6 +52,8 @@ WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& de
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_index_scores_decode(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
                                        uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
+                                     uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,
                         uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,

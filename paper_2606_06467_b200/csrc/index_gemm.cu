@@ -1,0 +1,348 @@
+// Index scores for a prefill chunk (Eq. 3, first half, T > 1 queries per sequence): a dense
+// bf16 x bf16 -> fp32 contraction  scores[t][s] = sum_j Q_idx[t][j] * K_idx[s][j]  on the
+// 5th-generation tensor cores.
+//
+// Shape of the problem: M = T queries (4096), N = cached tokens (135168), K = d_idx (64 or 128).
+// K is tiny, so the kernel is bound by writing the fp32 scores, not by the MMAs; the design keeps
+// the tensor pipe and the store path busy at the same time rather than chasing MMA peak.
+//
+// One persistent block per SM walks output tiles of 128 queries x 256 keys (query block fastest,
+// so neighbouring SMs share a key tile in L2). Warp roles:
+//   warp 0, one lane : TMA producer. Per tile, 2 + 2 tiled bulk copies (128-byte swizzle) bring the
+//                      128 x d_idx query tile and the 256 x d_idx key tile into a 2-stage ring.
+//   warp 1, one lane : MMA issuer. d_idx/16 tcgen05.mma (M128 N256 K16, kind::f16, bf16 inputs, fp32
+//                      accumulate) per tile into one of two 256-column TMEM accumulators;
+//                      tcgen05.commit frees the smem stage and publishes the accumulator.
+//   warp 2           : allocates / frees the 512 TMEM columns.
+//   warps 4..7       : epilogue. Each warp owns 32 TMEM lanes (= 32 query rows): tcgen05.ld 32
+//                      columns at a time, then 32-byte vector stores of the visible part of the row
+//                      (causal limit per query), so the epilogue of tile i overlaps the MMAs of tile i+1.
+// Tiles that lie entirely above the causal diagonal are skipped by every role alike.
+// Every mbarrier wait is bounded: on expiry the block raises CLSA_DEV_TIMEOUT in the status word,
+// all roles leave their loops, in-flight copies are given time to land, TMEM is freed, and the
+// kernel returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace clsa {
+namespace {
+
+constexpr int kBM = 128, kBN = 256, kBK = 64;  // tile; kBK bf16 = one 128-byte swizzle row
+constexpr int kStages = 2, kAccBufs = 2;
+constexpr int kThreads = 256;
+constexpr int kABytes = kBM * kBK * 2;          // one k-block of the query tile (16 KiB)
+constexpr int kBBytes = kBN * kBK * 2;          // one k-block of the key tile (32 KiB)
+constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;  // up to two k-blocks each (96 KiB)
+constexpr int kBarrierBytes = 128;
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+constexpr uint32_t kSpinLimit = 1u << 22;       // polls with back-off: a few seconds at most
+
+struct GemmArgs {
+  const int64_t* seq_start;
+  const int32_t* seq_len;
+  float* scores;
+  int64_t score_stride;
+  uint32_t* status;
+  int num_seqs, q_per_seq, causal, max_seq_len, idx_dim;
+  int m_blocks, n_tiles;
+  int vec_ok;  // rows of `scores` are 32-byte aligned: 256-bit stores allowed
+};
+
+// ---- PTX wrappers ----------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait. Returns false if the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*abort_flag != 0u) return false;
+      __nanosleep(64);
+    }
+  }
+  *abort_flag = 1u;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: 8-row groups are 1024 bytes
+// apart (stride byte offset), the leading byte offset is unused inside one swizzle row.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffffu) >> 4);        // start address, 16-byte units
+  d |= (uint64_t)(1024u >> 4) << 32;               // stride byte offset
+  d |= (uint64_t)1 << 46;                          // descriptor version (sm_100)
+  d |= (uint64_t)2 << 61;                          // layout: 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N and M encoded as N/8 and M/16.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+struct TileCoord {
+  int b, mb, nt, n, valid;
+};
+// The same enumeration for every role: tile id -> (sequence, query block, key tile); valid == 0 for
+// tiles of a sequence with a bad length and for tiles wholly above the causal diagonal.
+__device__ __forceinline__ TileCoord tile_coord(const GemmArgs& a, int64_t id) {
+  TileCoord c;
+  const int per_seq = a.m_blocks * a.n_tiles;
+  c.b = (int)(id / per_seq);
+  const int rem = (int)(id - (int64_t)c.b * per_seq);
+  c.nt = rem / a.m_blocks;
+  c.mb = rem - c.nt * a.m_blocks;
+  c.n = a.seq_len[c.b];
+  const int t_last = min(a.q_per_seq, (c.mb + 1) * kBM) - 1;
+  const int v_max = a.causal ? c.n - a.q_per_seq + t_last + 1 : c.n;
+  c.valid = (c.n >= a.q_per_seq && c.n <= a.max_seq_len && c.nt * kBN < v_max) ? 1 : 0;
+  return c;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const GemmArgs a) {
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t raw = smem_u32(smem_dyn);
+  const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle wants 1024-byte aligned tiles
+  unsigned char* base_ptr = smem_dyn + (base - raw);
+  const uint32_t bars = base + kStages * kStageBytes;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 16u + 8u * s; };
+  auto tfull_bar = [&](int i) { return bars + 32u + 8u * i; };
+  auto tempty_bar = [&](int i) { return bars + 48u + 8u * i; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + 64);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + 68);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kblocks = a.idx_dim / kBK;  // 1 or 2
+  const int64_t total_tiles = (int64_t)a.num_seqs * a.m_blocks * a.n_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int i = 0; i < kAccBufs; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 4); }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(bars + 64u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
+        const TileCoord c = tile_coord(a, id);
+        if (!c.valid) continue;
+        const int s = it % kStages;
+        const uint32_t ph = (it / kStages) & 1u;
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) break;
+        const uint32_t st = base + s * kStageBytes;
+        mbar_expect_tx(full_bar(s), (uint32_t)kblocks * (kABytes + kBBytes));
+        const int qrow = c.b * a.q_per_seq + c.mb * kBM;
+        const int krow = (int)(a.seq_start[c.b] + (int64_t)c.nt * kBN);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          tma_load_2d(st + kb * kABytes, &map_q, kb * kBK, qrow, full_bar(s));
+          tma_load_2d(st + 2 * kABytes + kb * kBBytes, &map_k, kb * kBK, krow, full_bar(s));
+        }
+        ++it;
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16(kBM, kBN);
+      uint32_t it = 0;
+      for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
+        const TileCoord c = tile_coord(a, id);
+        if (!c.valid) continue;
+        const int s = it % kStages, acc = it % kAccBufs;
+        const uint32_t ph = (it / kStages) & 1u, aph = (it / kAccBufs) & 1u;
+        if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag)) break;
+        if (!mbar_wait(full_bar(s), ph, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t st = base + s * kStageBytes;
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kBN);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          const uint64_t adesc = smem_desc_sw128(st + kb * kABytes);
+          const uint64_t bdesc = smem_desc_sw128(st + 2 * kABytes + kb * kBBytes);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+            // 16 bf16 = 32 bytes further along K inside the swizzle row: +2 in 16-byte address units
+            tc_mma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+        }
+        tc_commit(empty_bar(s));     // the stage may be refilled once these MMAs have read it
+        tc_commit(tfull_bar(acc));   // the accumulator is complete
+        ++it;
+      }
+    }
+  } else if (warp >= 4) {
+    // ---------------- epilogue: TMEM -> registers -> global ----------------
+    const int quad = warp & 3;  // TMEM lanes 32*quad .. 32*quad+31
+    uint32_t it = 0;
+    for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
+      const TileCoord c = tile_coord(a, id);
+      if (!c.valid) continue;
+      const int acc = it % kAccBufs;
+      const uint32_t aph = (it / kAccBufs) & 1u;
+      if (!mbar_wait(tfull_bar(acc), aph, abort_flag)) break;
+      tc_fence_after();
+      const int t = c.mb * kBM + quad * 32 + lane;       // query of this thread's row
+      const bool row_ok = t < a.q_per_seq;
+      const int v = row_ok ? (a.causal ? c.n - a.q_per_seq + t + 1 : c.n) : 0;  // visible keys of this query
+      float* orow = a.scores + ((int64_t)c.b * a.q_per_seq + t) * a.score_stride;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kBN);
+#pragma unroll 1
+      for (int c0 = 0; c0 < kBN; c0 += 32) {
+        const int s0 = c.nt * kBN + c0;
+        if (__all_sync(0xffffffffu, s0 >= v)) break;     // the rest of the tile is above the diagonal for this warp
+        uint32_t r[32];
+        tc_ld32(taddr + (uint32_t)c0, r);
+        tc_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          const int s = s0 + j;
+          if (a.vec_ok && s + 8 <= v) {
+            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(orow + s), "r"(r[j]), "r"(r[j + 1]),
+                         "r"(r[j + 2]), "r"(r[j + 3]), "r"(r[j + 4]), "r"(r[j + 5]), "r"(r[j + 6]), "r"(r[j + 7])
+                         : "memory");
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              if (s + e < v) orow[s + e] = __uint_as_float(r[j + e]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));        // 4 arrivals (one per epilogue warp) free the accumulator
+      ++it;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag != 0u) {
+    // A wait ran out: report it, and give copies that may still be in flight time to land before
+    // the block (and its shared memory) goes away.
+    if (threadIdx.x == 0) flag_status(a.status, CLSA_DEV_TIMEOUT);
+    const long long t0 = clock64();
+    while (clock64() - t0 < 4000000LL) {}
+    __syncthreads();
+  }
+  if (warp == 2) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 [rows][cols] with `row_stride` elements between rows; box = 64 columns x box_rows rows.
+bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t row_stride, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {row_stride * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
+                                     uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
+  CUtensorMap map_q, map_k;
+  const uint64_t q_rows = (uint64_t)p.num_seqs * p.q_per_seq;
+  if (!make_map(&map_q, q_idx, q_rows, (uint64_t)p.idx_dim, (uint64_t)p.idx_dim, kBM)) return cudaErrorInvalidValue;
+  if (!make_map(&map_k, p.idx_k_cache, (uint64_t)p.num_cache_rows, (uint64_t)p.idx_dim, (uint64_t)p.idx_token_stride, kBN))
+    return cudaErrorInvalidValue;
+  GemmArgs a;
+  a.seq_start = p.seq_start;
+  a.seq_len = p.seq_len;
+  a.scores = scores;
+  a.score_stride = score_stride;
+  a.status = status;
+  a.num_seqs = p.num_seqs;
+  a.q_per_seq = p.q_per_seq;
+  a.causal = p.causal;
+  a.max_seq_len = p.max_seq_len;
+  a.idx_dim = p.idx_dim;
+  a.m_blocks = (p.q_per_seq + kBM - 1) / kBM;
+  a.n_tiles = (p.max_seq_len + kBN - 1) / kBN;
+  a.vec_ok = (score_stride % 8 == 0 && reinterpret_cast<uintptr_t>(scores) % 32 == 0) ? 1 : 0;
+  cudaError_t err = cudaFuncSetAttribute(index_scores_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (err != cudaSuccess) return err;
+  const int64_t tiles = (int64_t)p.num_seqs * a.m_blocks * a.n_tiles;
+  const int grid = (int)(tiles < dev.sm_count ? tiles : dev.sm_count);
+  index_scores_gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, a);
+  return cudaGetLastError();
+}
+
+}  // namespace clsa

@@ -1,0 +1,81 @@
+"""Prefill chunk (T > 1 queries per sequence, causal): the tcgen05 score GEMM, per-row causal top-k and sparse
+attention with one index row per query, against the oracle."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+import __graft_entry__ as entry
+
+entry._load_build_module().build()
+
+import oracle
+import paper_2606_06467_b200 as clsa
+from _harness import GpuProblem, check_attention, check_scores, check_topk_band, check_topk_exact_on_gpu_scores
+from workloads import MID, PREFILL, TINY, Workload
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_oracle(w):
+    kc, vc = w.host_kv_full()
+    return oracle.problem_from_workload(w, k_cache=kc, v_cache=vc, idx_k_cache=w.host_kidx_cache())
+
+
+@pytest.mark.parametrize("B,T,n,d_idx,causal,ragged", [
+    (1, 128, 1024, 128, 1, 0), (2, 200, 3000, 128, 1, 0), (1, 300, 2500, 64, 1, 0), (2, 77, 1111, 128, 0, 0),
+    (3, 150, 2000, 128, 1, 500), (1, 513, 700, 64, 1, 0)])
+def test_chunk_scores_topk_attention(B, T, n, d_idx, causal, ragged):
+    base = MID if d_idx == 128 else TINY
+    cfg = base.replace(num_seqs=B, ctx=n, q_per_seq=T, causal=causal, top_k=96, num_layers=2, seed=900 + T + n,
+                       ragged_min=ragged, num_short=0)
+    w = Workload(cfg)
+    g = GpuProblem(w)
+    prob = _full_oracle(w)
+    ref_scores = prob.index_scores(w.q_idx_bits())
+    gs = g.index_scores()
+    torch.cuda.synchronize()
+    assert g.status() == 0
+    check_scores(gs, ref_scores, w)
+    gi, gc = g.topk(gs)
+    check_topk_exact_on_gpu_scores(prob, gs, gi, gc, w)
+    ref_idx, ref_cnt = prob.topk(ref_scores)
+    check_topk_band(ref_scores, ref_idx, ref_cnt, gi, gc, w)
+    idx_np, cnt_np = gi.cpu().numpy().copy(), gc.cpu().numpy().copy()
+    for l in range(2):
+        out, lse = g.sparse_attn(l, sweep=l)
+        check_attention(prob, w, l, out, lse, idx_np, cnt_np)
+    assert g.status() == 0
+
+
+def test_gemm_row_equals_decode_gemv():
+    """Row t of the chunk GEMM is the decode kernel's result for the same query against the same keys."""
+    w = Workload(MID.replace(num_seqs=1, ctx=4096, q_per_seq=256, causal=0, top_k=64, num_layers=1, seed=31))
+    g = GpuProblem(w)
+    gs = g.index_scores()
+    for t in (0, 100, 255):
+        wd = Workload(MID.replace(num_seqs=1, ctx=4096, top_k=64, num_layers=1, seed=31))
+        gd = GpuProblem(wd, layers=1)
+        gd.params.idx_k_cache = g.t["idx_k_cache"].data_ptr()
+        q = g.t["q_idx"][:, t:t + 1].contiguous()
+        s = gd.new_scores()
+        clsa.clsa_index_scores(gd.params, q, s, gd.score_stride, gd.ws)
+        a, b = s[0, 0, :4096].cpu().numpy(), gs[0, t, :4096].cpu().numpy()
+        assert np.abs(a - b).max() <= 1e-4 * max(1.0, np.abs(a).max())
+
+
+def test_misaligned_score_rows_use_the_scalar_store_path():
+    w = Workload(MID.replace(num_seqs=1, ctx=1500, q_per_seq=130, causal=1, top_k=32, num_layers=1, seed=5))
+    g = GpuProblem(w)
+    prob = oracle.problem_from_workload(w, idx_k_cache=w.host_kidx_cache())
+    ref = prob.index_scores(w.q_idx_bits())
+    stride = 1501                                    # odd stride: rows are not 32-byte aligned
+    s = torch.full((1, 130, stride), float("nan"), dtype=torch.float32, device=g.dev)
+    clsa.clsa_index_scores(g.params, g.t["q_idx"], s, stride, g.ws)
+    got = s.cpu().numpy().astype(np.float64)
+    for t in range(130):
+        v = w.visible(0, t)
+        assert np.abs(got[0, t, :v] - ref[0, t, :v]).max() <= 1e-4 * max(1.0, np.abs(ref[0, t, :v]).max())
+        assert np.isnan(got[0, t, v:]).all()
