@@ -51,6 +51,20 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def profiled_traffic(workload: str, kernel: str):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) recorded from an ncu capture, from
+    profiles/traffic.txt ("workload kernel bytes ..." lines); None if that capture has not been recorded."""
+    path = os.path.join(ROOT, "profiles", "traffic.txt")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        for line in f:
+            parts = line.split()
+            if len(parts) >= 3 and not line.startswith("#") and parts[0] == workload and parts[1] == kernel:
+                return float(parts[2])
+    return None
+
+
 class ClockSampler(threading.Thread):
     """Polls NVML (read-only) for SM clock and clock-event reasons while the timed region runs."""
 
@@ -231,25 +245,37 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     w = Workload(CONFIGS[args.config])
     c = w.cfg
-    if c.q_per_seq != 1:
-        raise SystemExit("bench.py times decode workloads (q_per_seq == 1)")
+    T = c.q_per_seq
     t = w.to_device(dev)
     L = c.num_layers
     p = clsa.make_params(num_seqs=c.num_seqs, num_q_heads=c.num_q_heads, num_kv_heads=c.num_kv_heads,
                          head_dim=c.head_dim, idx_dim=c.idx_dim, top_k=c.top_k, num_layers=L, max_seq_len=w.max_seq_len,
                          sm_scale=c.sm_scale, seq_start=t["seq_start"], seq_len=t["seq_len"], k_cache=t["k_cache"],
-                         v_cache=t["v_cache"], idx_k_cache=t["idx_k_cache"])
+                         v_cache=t["v_cache"], idx_k_cache=t["idx_k_cache"], q_per_seq=T, causal=c.causal)
     ws = torch.zeros(clsa.clsa_workspace_bytes(p), dtype=torch.uint8, device=dev)
-    idx = torch.empty((c.num_seqs, 1, c.top_k), dtype=torch.int32, device=dev)
-    cnt = torch.empty((c.num_seqs, 1), dtype=torch.int32, device=dev)
+    idx = torch.empty((c.num_seqs, T, c.top_k), dtype=torch.int32, device=dev)
+    cnt = torch.empty((c.num_seqs, T), dtype=torch.int32, device=dev)
     q_layers = [t["q_layers"][l] for l in range(L)]
-    outs = [torch.empty((c.num_seqs, 1, c.num_q_heads, c.head_dim), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+    outs = [torch.empty((c.num_seqs, T, c.num_q_heads, c.head_dim), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+    stride = (w.max_seq_len + 63) // 64 * 64
+    chunk_scores = torch.empty((c.num_seqs, T, stride), dtype=torch.float32, device=dev) if T > 1 else None
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     alg_bytes = w.algorithmic_bytes()
     stream = torch.cuda.current_stream()
 
+    def run_step(q_idx_t, q_list):
+        if T == 1:
+            clsa.clsa_decode_step(p, q_idx_t, q_list, outs, idx, cnt, ws, stream=stream)
+        else:  # a prefill chunk is not chained by the library: the three calls, in order
+            clsa.clsa_index_scores(p, q_idx_t, chunk_scores, stride, ws, stream=stream)
+            clsa.clsa_topk(p, chunk_scores, stride, idx, cnt, ws, stream=stream)
+            for l in range(L):
+                p.sweep = l & 1
+                clsa.clsa_sparse_attn(p, q_list[l], idx, cnt, outs[l], None, ws, stream=stream)
+            p.sweep = 0
+
     def step():
-        clsa.clsa_decode_step(p, t["q_idx"], q_layers, outs, idx, cnt, ws, stream=stream)
+        run_step(t["q_idx"], q_layers)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -289,7 +315,7 @@ def run_ours(args):
         d_qidx.copy_(h_qidx, non_blocking=True)
         for l in range(L):
             d_q[l].copy_(h_q[l], non_blocking=True)
-        clsa.clsa_decode_step(p, d_qidx, d_q, outs, idx, cnt, ws, stream=stream)
+        run_step(d_qidx, d_q)
         for l in range(L):
             h_out[l].copy_(outs[l], non_blocking=True)
 
@@ -314,8 +340,7 @@ def run_ours(args):
     breakdown = None
     attn_us = None
     if not args.no_breakdown:
-        stride = (w.max_seq_len + 63) // 64 * 64
-        scores = torch.empty((c.num_seqs, 1, stride), dtype=torch.float32, device=dev)
+        scores = chunk_scores if T > 1 else torch.empty((c.num_seqs, 1, stride), dtype=torch.float32, device=dev)
         nb = min(K, 20)
         acc = {"index_scores": 0.0, "topk": 0.0, "sparse_attn": 0.0}
         for i in range(nb + 2):
@@ -346,7 +371,7 @@ def run_ours(args):
     peak, peak_kind = measured_peaks()
     gathered_per_layer = int(w.selected_counts().sum()) * c.num_kv_heads * c.head_dim * 4
     roofline = {
-        "bound": "hbm", "kernel": "sparse_attn_kernel (+ merge), one layer",
+        "bound": "hbm", "kernel": "sparse_attn_kernel, one layer (one launch)",
         "achieved": (gathered_per_layer / (attn_us * 1e-6) / 1e9) if attn_us else None,
         "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
         "frac": (gathered_per_layer / (attn_us * 1e-6) / 1e9 / peak) if attn_us else None,
@@ -354,13 +379,7 @@ def run_ours(args):
         "algorithmic_bytes_per_launch": gathered_per_layer,
         "step_frac": value / world / peak,
     }
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(prof):
-        try:
-            with open(prof) as f:
-                roofline["traffic"] = json.load(f).get(c.name, {}).get("sparse_attn_kernel")
-        except Exception:
-            pass
+    roofline["traffic"] = profiled_traffic(c.name, "sparse_attn_kernel")
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -393,7 +412,7 @@ def run_ours(args):
                     "ms_per_step": e2e_ms / K,
                     "note": "per-step inputs (q_idx, L query tensors) from pinned host memory and all L outputs back; "
                             "the KV and indexer-key caches are decoder state and stay resident"},
-            "gpu_launches": K * (2 + 2 * L),
+            "gpu_launches": K * (2 + L),
         }
         print(json.dumps(line))
     if dist is not None:

@@ -65,3 +65,76 @@ def test_full_size_decode_step(cfg):
     g2_idx, g2_cnt = g.topk(gs)
     np.testing.assert_array_equal(g2_idx.cpu().numpy(), idx_np)
     np.testing.assert_array_equal(g2_cnt.cpu().numpy(), cnt_np)
+
+
+def test_full_size_prefill_chunk():
+    """Config 5: 131072 cached tokens + a 4096-query causal chunk. The GPU runs the whole chunk; the oracle checks
+    64 sampled query rows completely (a query row of a causal chunk is exactly a decode problem whose sequence
+    ends at that query) and cheap invariants cover every row."""
+    from workloads import PREFILL
+
+    cfg = PREFILL
+    w = Workload(cfg)
+    g = GpuProblem(w, layers=2)            # queries of layers 0 and 1 stand for "first" and "any other" layer
+    T, n, k = cfg.q_per_seq, cfg.ctx, cfg.top_k
+    gs = g.index_scores()
+    gi, gc = g.topk(gs)
+    outs = [g.sparse_attn(l, sweep=l, lse=False)[0] for l in range(2)]
+    torch.cuda.synchronize()
+    assert g.status() == 0
+    # every row: count, range, order, finiteness
+    vis = torch.arange(T, device=g.dev) + (n - T + 1)
+    assert torch.equal(gc[0].long(), torch.clamp(vis, max=k))
+    assert (gi[0, :, 1:] > gi[0, :, :-1]).all() and (gi[0, :, 0] >= 0).all()
+    assert (gi[0, :, -1].long() < vis).all()
+    for o in outs:
+        assert torch.isfinite(o.float()).all()
+    # sampled rows against the oracle
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, 1, T - 1, T - 2, 127, 128], rng.integers(0, T, 58)]))
+    kidx = w.host_kidx_cache()
+    qi = w.q_idx_bits()[0, rows]                                            # [R, d_idx]
+    R = rows.size
+    seq_len = np.array([w.visible(0, int(t)) for t in rows], dtype=np.int32)
+    sub_prob = oracle.Problem(num_seqs=R, num_q_heads=cfg.num_q_heads, num_kv_heads=cfg.num_kv_heads,
+                              head_dim=cfg.head_dim, idx_dim=cfg.idx_dim, top_k=k, sm_scale=cfg.sm_scale,
+                              seq_start=np.zeros(R, dtype=np.int64), seq_len=seq_len, idx_k_cache=kidx)
+    ref_scores = sub_prob.index_scores(qi.reshape(R, 1, -1))
+    got_scores = gs[0, torch.from_numpy(rows).to(g.dev)].cpu().numpy().astype(np.float64)
+    for i in range(R):
+        v = seq_len[i]
+        r = ref_scores[i, 0, :v]
+        assert (np.abs(got_scores[i, :v] - r) <= 1e-4 * np.maximum(1.0, np.abs(r))).all()
+        assert np.isnan(got_scores[i, v:n]).all()
+    ref_idx, ref_cnt = sub_prob.topk(ref_scores)
+    gpu_idx = gi[0, torch.from_numpy(rows).to(g.dev)].cpu().numpy()
+    exact_idx, _ = sub_prob.topk(np.where(np.isnan(got_scores), -np.inf, got_scores)[:, None, : ref_scores.shape[2]])
+    band = 0
+    for i in range(R):
+        np.testing.assert_array_equal(gpu_idx[i], np.sort(exact_idx[i, 0]))      # exact on the GPU's own scores
+        a, b = set(gpu_idx[i].tolist()), set(ref_idx[i, 0].tolist())
+        if a != b:
+            s = ref_scores[i, 0, : seq_len[i]]
+            tau = np.sort(s)[-k]
+            diff = np.array(sorted(a ^ b))
+            assert (np.abs(s[diff] - tau) <= 1e-3 * abs(tau)).all()
+            band += 1
+    print(f"prefill: sampled rows differing from the fp64 oracle inside the band only: {band} of {R}")
+    # attention of the sampled rows, oracle fed the GPU's index
+    idx_s = gpu_idx.reshape(R, 1, k)
+    cnt_s = np.minimum(seq_len, k).reshape(R, 1).astype(np.int32)
+    kc = np.zeros((w.total_rows, cfg.num_kv_heads, cfg.head_dim), dtype=np.uint16)
+    vc = np.zeros_like(kc)
+    touched = np.unique(idx_s)
+    kc[touched] = w.kv_rows_bits("k", touched).reshape(-1, cfg.num_kv_heads, cfg.head_dim)
+    vc[touched] = w.kv_rows_bits("v", touched).reshape(-1, cfg.num_kv_heads, cfg.head_dim)
+    att_prob = oracle.Problem(num_seqs=R, num_q_heads=cfg.num_q_heads, num_kv_heads=cfg.num_kv_heads,
+                              head_dim=cfg.head_dim, idx_dim=cfg.idx_dim, top_k=k, sm_scale=cfg.sm_scale,
+                              seq_start=np.zeros(R, dtype=np.int64), seq_len=seq_len, k_cache=kc, v_cache=vc)
+    for l in range(2):
+        q = w.q_layer_bits(l)[0, rows].reshape(R, 1, cfg.num_q_heads, cfg.head_dim)
+        o_ref, _ = att_prob.sparse_attn(q, idx_s, cnt_s)
+        got = outs[l][0, torch.from_numpy(rows).to(g.dev)].float().cpu().numpy().astype(np.float64)
+        err = np.abs(got - o_ref[:, 0])
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3
+        print(f"prefill layer {l}: max abs err {err.max():.2e}, mean abs err {err.mean():.2e}")

@@ -57,7 +57,10 @@ RAGGED = Config("ragged", _SEED0 + 4, 64, 131072, 32, 8, 128, 128, 2048, 16,
 PREFILL = Config("prefill_chunk", _SEED0 + 5, 1, 131072 + 4096, 32, 8, 128, 128, 2048, 16,
                  q_per_seq=4096, causal=1)
 
-CONFIGS = {c.name: c for c in (TINY, MID, HEADLINE, RAGGED, PREFILL)}
+# a scaled-down prefill chunk (scores 285 MB, caches 142 MB: beyond L2, small enough to profile)
+PREFILL_SMALL = PREFILL.replace(name="prefill_small", ctx=32768 + 2048, q_per_seq=2048, num_layers=2)
+
+CONFIGS = {c.name: c for c in (TINY, MID, HEADLINE, RAGGED, PREFILL, PREFILL_SMALL)}
 
 
 class Workload:
