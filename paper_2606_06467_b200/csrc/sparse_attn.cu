@@ -2,8 +2,8 @@
 //
 // The kernel is bound by the gather of K/V rows from HBM (4 flops per byte per KV head), so its
 // shape is chosen for memory behaviour; the small matrix products ride on warp-level bf16 MMAs
-// (m16n8k16, fp32 accumulate) with the query heads of one KV head packed into the 16 rows of one
-// tile, far below tensor-pipe capacity.
+// (m16n8k16, fp32 accumulate) formed transposed -- tokens along M, the query heads of one KV head
+// packed into the 8 columns of one tile -- far below tensor-pipe capacity.
 //
 // Decomposition. One thread-block cluster of C blocks serves one query row (sequence, query
 // token); its selected tokens are cut into C * S contiguous ranges. A block has 8 autonomous
@@ -87,6 +87,14 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+
+// NT = number of 8-head tiles that hold the query heads of one KV head (1 for groups up to 8, 2 up to 16).
+template <int NT>
 __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   cg::cluster_group cluster = cg::this_cluster();
@@ -104,8 +112,12 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   const uint32_t ring_u32 = smem_u32(ring);
   uint32_t* stage_mask = reinterpret_cast<uint32_t*>(smem + kAttnWarps * kWarpRingBytes) + warp * kAttnStages;
 
-  const int qrow_a = lane >> 2;        // MMA row (query head within the group) of c0/c1; c2/c3 are row + 8
-  const int qcol = (lane & 3) * 2;
+  // Fragment coordinates. The products are formed transposed, tokens along M:
+  //   S^T[16 tokens x 8 heads] = K[16 x 128] Q^T,   O^T[128 x 8 heads] += V^T[128 x 16 tokens] P^T
+  // so a lane's accumulator columns are always the same two query heads (hcol, hcol+1 of each 8-head
+  // tile), and its rows are tokens (for S^T: rowq and rowq+8) or output dimensions (for O^T).
+  const int rowq = lane >> 2;
+  const int hcol = (lane & 3) * 2;
   const int h0 = g * G;                // first query head of this KV head
 
   // Programmatic dependent launch: let the next kernel of the stream start its own prologue as soon
@@ -137,24 +149,30 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   }
   const int t_lo = min(cnt, slot_lo), t_hi = active ? min(cnt, slot_hi) : t_lo;
 
-  float o[16][4];
+  float o[NT][8][4];                   // O^T: [head tile][16-wide slice of D][c0..c3]
+  float mA[NT], mB[NT], lA[NT], lB[NT];  // running max / sum of heads hcol and hcol+1 (log2 domain)
 #pragma unroll
-  for (int j = 0; j < 16; ++j) { o[j][0] = 0.f; o[j][1] = 0.f; o[j][2] = 0.f; o[j][3] = 0.f; }
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  for (int nt = 0; nt < NT; ++nt) {
+    mA[nt] = -INFINITY; mB[nt] = -INFINITY; lA[nt] = 0.f; lB[nt] = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { o[nt][j][0] = 0.f; o[nt][j][1] = 0.f; o[nt][j][2] = 0.f; o[nt][j][3] = 0.f; }
+  }
 
   if (t_lo < t_hi) {
-    // Query fragments (A operand, 16 x 128): rows >= G are zero padding.
-    uint32_t qa[8][4];
+    // Q^T fragments (B operand, 128 x 8 per head tile): head = rowq, two consecutive d per register.
+    uint32_t qb[NT][8][2];
     {
       const uint16_t* qbase = a.q + (r * a.num_q_heads + h0) * 128;
-      const bool v0 = qrow_a < G, v1 = qrow_a + 8 < G;
 #pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        const int c = kk * 16 + qcol;
-        qa[kk][0] = v0 ? *reinterpret_cast<const uint32_t*>(qbase + qrow_a * 128 + c) : 0u;
-        qa[kk][1] = v1 ? *reinterpret_cast<const uint32_t*>(qbase + (qrow_a + 8) * 128 + c) : 0u;
-        qa[kk][2] = v0 ? *reinterpret_cast<const uint32_t*>(qbase + qrow_a * 128 + c + 8) : 0u;
-        qa[kk][3] = v1 ? *reinterpret_cast<const uint32_t*>(qbase + (qrow_a + 8) * 128 + c + 8) : 0u;
+      for (int nt = 0; nt < NT; ++nt) {
+        const int head = nt * 8 + rowq;
+        const bool hv = head < G;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const int d = ks * 16 + hcol;
+          qb[nt][ks][0] = hv ? *reinterpret_cast<const uint32_t*>(qbase + head * 128 + d) : 0u;
+          qb[nt][ks][1] = hv ? *reinterpret_cast<const uint32_t*>(qbase + head * 128 + d + 8) : 0u;
+        }
       }
     }
 
@@ -219,113 +237,102 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
       const uint32_t kbuf = ring_u32 + buf * kStageBytes, vbuf = kbuf + kStageBytes / 2;
       const uint32_t okmask = stage_mask[buf];
 
-      // S = Q K^T for 16 tokens (two 8-token tiles)
-      float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      // S^T = K Q^T for 16 tokens: A = K rows (tokens) from shared memory, B = Q^T from registers
+      float s[NT][4];
 #pragma unroll
-      for (int kq = 0; kq < 4; ++kq) {
+      for (int nt = 0; nt < NT; ++nt) { s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f; }
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const int tok = 8 * j + (lane & 7), chunk = 4 * kq + (lane >> 3);
-          uint32_t bfrag[4];
-          ldmatrix_x4(bfrag, kbuf + tok * 256 + ((chunk ^ (tok & 7)) << 4));
-          mma_bf16(s[j], qa[2 * kq], bfrag[0], bfrag[1]);
-          mma_bf16(s[j], qa[2 * kq + 1], bfrag[2], bfrag[3]);
-        }
+      for (int ks = 0; ks < 8; ++ks) {
+        const int tok = (lane & 7) + 8 * ((lane >> 3) & 1), chunk = 2 * ks + (lane >> 4);
+        uint32_t kf[4];
+        ldmatrix_x4(kf, kbuf + tok * 256 + ((chunk ^ (tok & 7)) << 4));
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(s[nt], kf, qb[nt][ks][0], qb[nt][ks][1]);
       }
-      // online softmax, exp2 domain; masked tokens get -inf
-      float mx0 = -INFINITY, mx1 = -INFINITY;
+      // online softmax over tokens (rows), per head (columns), exp2 domain; masked tokens get -inf
+      const bool ok_lo = (okmask >> rowq) & 1u, ok_hi = (okmask >> (rowq + 8)) & 1u;
+      uint32_t pb0[NT], pb1[NT];
+      bool rescale = false;
+      float alphaA[NT], alphaB[NT];
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
+      for (int nt = 0; nt < NT; ++nt) {
+        const float s0v = ok_lo ? s[nt][0] * a.scale_log2 : -INFINITY;   // token rowq,   head hcol
+        const float s1v = ok_lo ? s[nt][1] * a.scale_log2 : -INFINITY;   // token rowq,   head hcol+1
+        const float s2v = ok_hi ? s[nt][2] * a.scale_log2 : -INFINITY;   // token rowq+8, head hcol
+        const float s3v = ok_hi ? s[nt][3] * a.scale_log2 : -INFINITY;   // token rowq+8, head hcol+1
+        float mxA = fmaxf(s0v, s2v), mxB = fmaxf(s1v, s3v);
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const bool ok = (okmask >> (8 * j + qcol + e)) & 1u;
-          s[j][e] = ok ? s[j][e] * a.scale_log2 : -INFINITY;
-          s[j][2 + e] = ok ? s[j][2 + e] * a.scale_log2 : -INFINITY;
-          mx0 = fmaxf(mx0, s[j][e]);
-          mx1 = fmaxf(mx1, s[j][2 + e]);
+        for (int d = 4; d <= 16; d <<= 1) {
+          mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, d));
+          mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, d));
         }
-      }
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-      const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-      const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
-      const float alpha0 = fast_exp2(m0 - mu0), alpha1 = fast_exp2(m1 - mu1);
-      const bool rescale = (mn0 != m0) || (mn1 != m1);
-      m0 = mn0;
-      m1 = mn1;
-      uint32_t pa[4];
-      {
-        const uint32_t p00 = pack_bf16x2(fast_exp2(s[0][0] - mu0), fast_exp2(s[0][1] - mu0));
-        const uint32_t p01 = pack_bf16x2(fast_exp2(s[0][2] - mu1), fast_exp2(s[0][3] - mu1));
-        const uint32_t p10 = pack_bf16x2(fast_exp2(s[1][0] - mu0), fast_exp2(s[1][1] - mu0));
-        const uint32_t p11 = pack_bf16x2(fast_exp2(s[1][2] - mu1), fast_exp2(s[1][3] - mu1));
-        pa[0] = p00; pa[1] = p01; pa[2] = p10; pa[3] = p11;
+        const float mnA = fmaxf(mA[nt], mxA), mnB = fmaxf(mB[nt], mxB);
+        const float muA = mnA == -INFINITY ? 0.f : mnA, muB = mnB == -INFINITY ? 0.f : mnB;
+        alphaA[nt] = fast_exp2(mA[nt] - muA);
+        alphaB[nt] = fast_exp2(mB[nt] - muB);
+        rescale = rescale || mnA != mA[nt] || mnB != mB[nt];
+        mA[nt] = mnA;
+        mB[nt] = mnB;
+        const uint32_t p_lo = pack_bf16x2(fast_exp2(s0v - muA), fast_exp2(s1v - muB));  // token rowq
+        const uint32_t p_hi = pack_bf16x2(fast_exp2(s2v - muA), fast_exp2(s3v - muB));  // token rowq + 8
         // the denominators use the same bf16-rounded weights as the numerators
-        l0 = l0 * alpha0 + (bf16_lo(p00) + bf16_hi(p00)) + (bf16_lo(p10) + bf16_hi(p10));
-        l1 = l1 * alpha1 + (bf16_lo(p01) + bf16_hi(p01)) + (bf16_lo(p11) + bf16_hi(p11));
+        lA[nt] = lA[nt] * alphaA[nt] + (bf16_lo(p_lo) + bf16_lo(p_hi));
+        lB[nt] = lB[nt] * alphaB[nt] + (bf16_hi(p_lo) + bf16_hi(p_hi));
+        // P is held [token][head]; the PV product wants P^T as its B operand: transpose the two 8x8 halves
+        pb0[nt] = movmatrix_trans(p_lo);
+        pb1[nt] = movmatrix_trans(p_hi);
       }
       if (__any_sync(0xffffffffu, rescale)) {  // the running max moved for some head: rescale the accumulators
 #pragma unroll
-        for (int j = 0; j < 16; ++j) { o[j][0] *= alpha0; o[j][1] *= alpha0; o[j][2] *= alpha1; o[j][3] *= alpha1; }
-      }
-      // O += P V
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-      for (int jp = 0; jp < 8; ++jp) {
-        const int tok = (lane & 7) + 8 * ((lane >> 3) & 1), chunk = 2 * jp + (lane >> 4);
-        uint32_t vfrag[4];
-        ldmatrix_x4_trans(vfrag, vbuf + tok * 256 + ((chunk ^ (tok & 7)) << 4));
-        mma_bf16(o[2 * jp], pa, vfrag[0], vfrag[1]);
-        mma_bf16(o[2 * jp + 1], pa, vfrag[2], vfrag[3]);
+          for (int j = 0; j < 8; ++j) {
+            o[nt][j][0] *= alphaA[nt]; o[nt][j][1] *= alphaB[nt]; o[nt][j][2] *= alphaA[nt]; o[nt][j][3] *= alphaB[nt];
+          }
+      }
+      // O^T += V^T P^T: A = V^T (transposing ldmatrix of the [token][d] tile), 8 slices of 16 output dimensions
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int tok = (lane & 7) + 8 * (lane >> 4), chunk = 2 * j + ((lane >> 3) & 1);
+        uint32_t vf[4];
+        ldmatrix_x4_trans(vf, vbuf + tok * 256 + ((chunk ^ (tok & 7)) << 4));
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(o[nt][j], vf, pb0[nt], pb1[nt]);
       }
       __syncwarp();  // everyone is done with this buffer before the next step refills it
     }
     cp_async_wait<0>();
 
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-  }
-
-  if (nsplit == 1) {
-    // the warp saw the whole row: normalise and write straight from the accumulators
-    if (active) {
-      const float inv0 = l0 > 0.f ? 1.f / l0 : 0.f, inv1 = l1 > 0.f ? 1.f / l1 : 0.f;
-      uint16_t* obase = a.out + (r * a.num_q_heads + h0) * 128;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        if (qrow_a < G)
-          *reinterpret_cast<uint32_t*>(obase + qrow_a * 128 + j * 8 + qcol) = pack_bf16x2(o[j][0] * inv0, o[j][1] * inv0);
-        if (qrow_a + 8 < G)
-          *reinterpret_cast<uint32_t*>(obase + (qrow_a + 8) * 128 + j * 8 + qcol) = pack_bf16x2(o[j][2] * inv1, o[j][3] * inv1);
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int d = 4; d <= 16; d <<= 1) {
+        lA[nt] += __shfl_xor_sync(0xffffffffu, lA[nt], d);
+        lB[nt] += __shfl_xor_sync(0xffffffffu, lB[nt], d);
       }
-      if (a.lse != nullptr && (lane & 3) == 0) {
-        if (qrow_a < G) a.lse[r * a.num_q_heads + h0 + qrow_a] = l0 > 0.f ? (m0 + log2f(l0)) * kLn2 : -INFINITY;
-        if (qrow_a + 8 < G) a.lse[r * a.num_q_heads + h0 + qrow_a + 8] = l1 > 0.f ? (m1 + log2f(l1)) * kLn2 : -INFINITY;
-      }
-    }
-    return;  // uniform over the cluster (a cluster of one block)
   }
 
-  // ---- split-K merge through distributed shared memory ---------------------------------------------
-  // Each warp parks its partial in its own (now idle) staging ring: [G][kPartialStride] floats.
+  // ---- split-K merge through (distributed) shared memory --------------------------------------------
+  // Each warp parks its partial in its own (now idle) staging ring: [G][kPartialStride] floats, row = head.
   float* mypart = reinterpret_cast<float*>(ring);
   if (active) {
+    __syncwarp();
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      if (qrow_a < G)
-        *reinterpret_cast<float2*>(mypart + qrow_a * kPartialStride + j * 8 + qcol) = make_float2(o[j][0], o[j][1]);
-      if (qrow_a + 8 < G)
-        *reinterpret_cast<float2*>(mypart + (qrow_a + 8) * kPartialStride + j * 8 + qcol) = make_float2(o[j][2], o[j][3]);
-    }
-    if ((lane & 3) == 0) {
-      if (qrow_a < G) *reinterpret_cast<float2*>(mypart + qrow_a * kPartialStride + 128) = make_float2(m0, l0);
-      if (qrow_a + 8 < G) *reinterpret_cast<float2*>(mypart + (qrow_a + 8) * kPartialStride + 128) = make_float2(m1, l1);
+    for (int nt = 0; nt < NT; ++nt) {
+      const int headA = nt * 8 + hcol, headB = headA + 1;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int d = 16 * j + rowq;
+        if (headA < G) { mypart[headA * kPartialStride + d] = o[nt][j][0]; mypart[headA * kPartialStride + d + 8] = o[nt][j][2]; }
+        if (headB < G) { mypart[headB * kPartialStride + d] = o[nt][j][1]; mypart[headB * kPartialStride + d + 8] = o[nt][j][3]; }
+      }
+      if (rowq == 0) {
+        if (headA < G) *reinterpret_cast<float2*>(mypart + headA * kPartialStride + 128) = make_float2(mA[nt], lA[nt]);
+        if (headB < G) *reinterpret_cast<float2*>(mypart + headB * kPartialStride + 128) = make_float2(mB[nt], lB[nt]);
+      }
     }
   }
-  cluster.sync();
+  if (C == 1) __syncthreads(); else cluster.sync();
 
   // Output jobs (KV head of this block's group, query head of the group) dealt over the cluster's warps.
   const int heads_here = min(HC, a.num_kv_heads - (int)blockIdx.y * HC);
@@ -335,8 +342,8 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
     // partial p = (block p / S, range p % S) was left by warp (p % S) * HC + jg of block p / S
     auto part_ptr = [&](int p) -> const float* {
       const int c2 = p / S, sub2 = p - c2 * S;
-      return cluster.map_shared_rank(reinterpret_cast<float*>(smem + (sub2 * HC + jg) * kWarpRingBytes), c2) +
-             hh * kPartialStride;
+      float* local = reinterpret_cast<float*>(smem + (sub2 * HC + jg) * kWarpRingBytes);
+      return (C == 1 ? local : cluster.map_shared_rank(local, c2)) + hh * kPartialStride;
     };
     float M = -INFINITY;
     for (int p = lane; p < nsplit; p += 32) M = fmaxf(M, part_ptr(p)[128]);
@@ -378,14 +385,14 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
     *reinterpret_cast<uint2*>(a.out + item * 128 + lane * 4) = packed;
     if (a.lse != nullptr && lane == 0) a.lse[item] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
   }
-  cluster.sync();  // no block may exit while a neighbour can still read its shared memory
+  if (C > 1) cluster.sync();  // no block may exit while a neighbour can still read its shared memory
 }
 
 // Blocks of `cluster` that can be resident at once (cached per cluster size; 0 if the query fails).
 static int max_resident_blocks(int cluster, size_t smem_bytes) {
   static int cache[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
   if (cache[cluster] != 0) return cache[cluster];
-  cudaFuncSetAttribute(sparse_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  cudaFuncSetAttribute(sparse_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)cluster * 64, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -398,7 +405,7 @@ static int max_resident_blocks(int cluster, size_t smem_bytes) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, sparse_attn_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+  if (cudaOccupancyMaxActiveClusters(&n, sparse_attn_kernel<1>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
   cache[cluster] = n * cluster;
   return cache[cluster];
 }
@@ -460,7 +467,8 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.reverse = reverse;
   a.wait_prior = wait_prior;
   a.scale_log2 = p.sm_scale * kLog2e;
-  cudaError_t err = cudaFuncSetAttribute(sparse_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
+  auto kernel = a.group <= 8 ? sparse_attn_kernel<1> : sparse_attn_kernel<2>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   cudaLaunchConfig_t cfg = {};
@@ -477,7 +485,7 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, sparse_attn_kernel, a);
+  return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
 }  // namespace clsa
