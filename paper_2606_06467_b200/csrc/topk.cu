@@ -2,19 +2,28 @@
 //
 // One thread-block cluster per (sequence, query) row. The row's visible scores are cut into
 // contiguous slices, one per block; each block converts its slice once to order-preserving 32-bit
-// keys held in shared memory, so the radix passes never go back to global memory. Three passes
-// resolve 12 + 12 + 8 key bits. fp32 scores crowd into a few sign/exponent patterns, so a wide
-// first digit (sign, exponent and three mantissa bits) is what keeps the shared-memory histogram
-// atomics from serialising on a handful of bins; a warp whose lanes all hit one bin adds once.
-// Per pass: each block histograms its slice into shared memory, then adds its non-empty bins into
-// every block's copy of the cluster-wide histogram with distributed-shared-memory atomics; after
-// one cluster barrier every block scans its own copy from the top bin down and finds, redundantly
-// and identically, the digit that contains the k-th largest key (the copies are double-buffered,
-// so one barrier per pass is enough). After three passes the exact threshold key and the number
-// of threshold-equal elements still needed are known. The compaction is index-ordered: a block's
-// output offset is the number of selected elements in lower-ranked blocks, a warp's offset the
-// number selected in lower warps, so positions come out ascending and, among keys equal to the
-// threshold, the lowest positions win. No atomics touch global memory and nothing spins.
+// keys held in shared memory, so nothing goes back to global memory afterwards.
+//
+// First digit: 12 key bits (sign, exponent, three mantissa bits). fp32 scores crowd into a few
+// sign/exponent patterns, so a wide first digit is what keeps the shared-memory histogram atomics
+// from serialising on a handful of bins; a warp whose lanes all hit one bin adds once. The
+// histogram is built in the same sweep that loads the scores. Each block adds its non-empty bins
+// into every block's copy of the row histogram with distributed-shared-memory atomics; after one
+// cluster barrier every block scans its own copy from the top bin down and finds, redundantly and
+// identically, the bin that contains the k-th largest key.
+//
+// Remaining 20 bits, common case: that bin holds few keys (a fraction of a percent of the row). A
+// second sweep counts, per warp, the keys above the bin and collects the keys inside it
+// ("candidates") with their positions; the blocks read each other's short candidate lists through
+// distributed shared memory and each finishes the select locally with two 10-bit passes over the
+// candidates only. Rare case (more than kCandCap keys share the first 12 bits, e.g. long runs of
+// equal scores): two more full radix passes (12 + 8 bits) with the same cluster-wide histograms.
+//
+// Either way the exact threshold key and the number of threshold-equal keys still needed are
+// known, and the last sweep is an index-ordered compaction: a block's output offset is the number
+// of selected keys in lower-ranked blocks, a warp's offset the number selected in lower warps, so
+// positions come out ascending and, among keys equal to the threshold, the lowest positions win.
+// No atomics touch global memory and nothing spins.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -24,18 +33,22 @@ namespace cg = cooperative_groups;
 namespace clsa {
 namespace {
 
-constexpr int kThreads = 512;  // 512 threads and < 113 KiB of shared memory: two blocks per SM, so that 16+ clusters of 8 are resident at once
+// 512 threads and < 113 KiB of shared memory: two blocks fit on an SM, so 16 and more clusters of 8
+// are resident at once (with one block per SM only 15 clusters of 8 fit the GPCs of a B200).
+constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxBins = 4096;
 constexpr int kMaxCluster = 8;
+constexpr int kCandCap = 2048;  // candidates (row-wide) the short path handles
 
 struct Shared {
-  uint32_t local_hist[kMaxBins];       // this block's slice
-  uint32_t cluster_hist[2][kMaxBins];  // whole row, one copy per block, filled by every block of the cluster
+  uint32_t local_hist[kMaxBins];       // this block's slice; later: gathered candidates + 1024-bin histogram
+  uint32_t cluster_hist[2][kMaxBins];  // whole row, one copy per block; [1] later: this block's candidate list
   uint32_t warp_tot[kWarps];
   uint32_t warp_gt[kWarps], warp_eq[kWarps];
   uint32_t block_gt_eq[2];             // read remotely
-  uint32_t digit, k_rem;
+  uint32_t cand_count;                 // read remotely
+  uint32_t digit, k_rem, bin_count;
   uint32_t out_base, eq_base;
 };
 
@@ -45,53 +58,32 @@ __device__ __forceinline__ uint32_t score_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// One radix pass over `BITS` key bits starting at `shift`. On return prefix/prefix_mask/k_rem are
-// updated. `buf` selects the cluster_hist copy (alternates between passes).
-template <int BITS, typename KeyAt>
-__device__ __forceinline__ void radix_pass(Shared& sh, cg::cluster_group& cluster, int nblk, int cnt, int shift, int buf,
-                                           uint32_t& prefix, uint32_t& prefix_mask, uint32_t& k_rem, KeyAt key_at) {
-  constexpr int NB = 1 << BITS;
+// Adds one to hist[bin] for every lane with `in`; a warp whose voters all share one bin adds once.
+__device__ __forceinline__ void hist_add(uint32_t* hist, bool in, uint32_t bin, int lane) {
+  const uint32_t voters = __ballot_sync(0xffffffffu, in);
+  if (voters == 0u) return;
+  const int leader = __ffs(voters) - 1;
+  const uint32_t lead_bin = __shfl_sync(0xffffffffu, bin, leader);
+  if (__all_sync(0xffffffffu, !in || bin == lead_bin)) {
+    if (lane == leader) atomicAdd(&hist[bin], (uint32_t)__popc(voters));
+  } else if (in) {
+    atomicAdd(&hist[bin], 1u);
+  }
+}
+
+// Block-wide scan of hist[0..NB) from the top bin down: finds the bin in which the running count
+// reaches k_rem. On return (after a __syncthreads) sh.digit is that bin, sh.k_rem what is still
+// needed inside it, sh.bin_count its population. If `clear`, the histogram is zeroed on the way.
+template <int NB>
+__device__ __forceinline__ void scan_from_top(Shared& sh, uint32_t* hist, uint32_t k_rem, bool clear) {
   constexpr int PT = (NB + kThreads - 1) / kThreads;  // bins per thread
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-  for (int i = tid; i < NB; i += kThreads) sh.local_hist[i] = 0;
-  __syncthreads();
-  for (int i0 = 0; i0 < cnt; i0 += kThreads) {
-    const int i = i0 + tid;
-    const uint32_t key = i < cnt ? key_at(i) : 0u;
-    const bool in = i < cnt && (key & prefix_mask) == prefix;
-    const uint32_t bin = (key >> shift) & (uint32_t)(NB - 1);
-    const uint32_t voters = __ballot_sync(0xffffffffu, in);
-    if (voters == 0u) continue;
-    // all participating lanes on one bin (long runs of equal scores): one add for the warp
-    const uint32_t lead_bin = __shfl_sync(0xffffffffu, bin, __ffs(voters) - 1);
-    const bool same = __all_sync(0xffffffffu, !in || bin == lead_bin);
-    if (same) {
-      if (lane == __ffs(voters) - 1) atomicAdd(&sh.local_hist[bin], (uint32_t)__popc(voters));
-    } else if (in) {
-      atomicAdd(&sh.local_hist[bin], 1u);
-    }
-  }
-  __syncthreads();
-  // add this block's non-empty bins into every block's copy of the row histogram
-  uint32_t* mine = sh.cluster_hist[buf];
-#pragma unroll
-  for (int j = 0; j < PT; ++j) {
-    const int bin = tid + j * kThreads;
-    if (bin < NB) {
-      const uint32_t v = sh.local_hist[bin];
-      if (v != 0u)
-        for (int r = 0; r < nblk; ++r) atomicAdd(cluster.map_shared_rank(mine, r) + bin, v);
-    }
-  }
-  cluster.sync();
-  // scan this block's copy from the top bin down: thread t owns bins NB-1-(t*PT+j)
   uint32_t own[PT];
   uint32_t tot = 0;
 #pragma unroll
   for (int j = 0; j < PT; ++j) {
-    const int pos = tid * PT + j;
-    own[j] = pos < NB ? mine[NB - 1 - pos] : 0u;
+    const int pos = tid * PT + j;  // thread t owns bins NB-1-(t*PT+j)
+    own[j] = pos < NB ? hist[NB - 1 - pos] : 0u;
     tot += own[j];
   }
   uint32_t incl = tot;
@@ -113,17 +105,49 @@ __device__ __forceinline__ void radix_pass(Shared& sh, cg::cluster_group& cluste
       if (acc < k_rem && k_rem <= acc + own[j]) {
         sh.digit = (uint32_t)(NB - 1 - (tid * PT + j));
         sh.k_rem = k_rem - acc;
+        sh.bin_count = own[j];
       }
       acc += own[j];
     }
   }
-  // clear the copy for its next use (two passes on); nobody else touches it before the next barrier
+  if (clear) {
 #pragma unroll
-  for (int j = 0; j < PT; ++j) {
-    const int pos = tid * PT + j;
-    if (pos < NB) mine[NB - 1 - pos] = 0u;
+    for (int j = 0; j < PT; ++j) {
+      const int pos = tid * PT + j;
+      if (pos < NB) hist[NB - 1 - pos] = 0u;
+    }
   }
   __syncthreads();
+}
+
+// Adds this block's non-empty local bins into every block's copy `buf` of the row histogram.
+template <int NB>
+__device__ __forceinline__ void push_hist(Shared& sh, cg::cluster_group& cluster, int nblk, int buf) {
+  uint32_t* mine = sh.cluster_hist[buf];
+  for (int bin = threadIdx.x; bin < NB; bin += kThreads) {
+    const uint32_t v = sh.local_hist[bin];
+    if (v != 0u)
+      for (int r = 0; r < nblk; ++r) atomicAdd(cluster.map_shared_rank(mine, r) + bin, v);
+  }
+}
+
+// One full radix pass over `BITS` key bits at `shift` (used by the rare long path).
+template <int BITS, typename KeyAt>
+__device__ __forceinline__ void radix_pass(Shared& sh, cg::cluster_group& cluster, int nblk, int cnt, int shift, int buf,
+                                           uint32_t& prefix, uint32_t& prefix_mask, uint32_t& k_rem, KeyAt key_at) {
+  constexpr int NB = 1 << BITS;
+  const int tid = threadIdx.x, lane = tid & 31;
+  for (int i = tid; i < NB; i += kThreads) sh.local_hist[i] = 0;
+  __syncthreads();
+  for (int i0 = 0; i0 < cnt; i0 += kThreads) {
+    const int i = i0 + tid;
+    const uint32_t key = i < cnt ? key_at(i) : 0u;
+    hist_add(sh.local_hist, i < cnt && (key & prefix_mask) == prefix, (key >> shift) & (uint32_t)(NB - 1), lane);
+  }
+  __syncthreads();
+  push_hist<NB>(sh, cluster, nblk, buf);
+  cluster.sync();
+  scan_from_top<NB>(sh, sh.cluster_hist[buf], k_rem, true);
   prefix |= sh.digit << shift;
   prefix_mask |= (uint32_t)(NB - 1) << shift;
   k_rem = sh.k_rem;
@@ -158,7 +182,7 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
     if (tid == 0) count_out[row] = kk;
     for (int i = kk + tid; i < top_k; i += kThreads) out[i] = -1;
   }
-  const int per = (v + nblk - 1) / nblk;
+  const int per = ((v + nblk - 1) / nblk + 3) & ~3;  // slice length, a multiple of 4 so slices keep their 16-byte phase
   const int lo = min(v, rank * per), hi = min(v, lo + per);
   const int cnt = hi - lo;
   if (kk == v) {  // nothing to select: every visible position is taken, in order
@@ -166,39 +190,186 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
     return;
   }
   const float* src = scores + (int64_t)row * score_stride + lo;
-  if (CACHED) {
-    for (int i = tid; i < cnt; i += kThreads) keys[i] = score_key(src[i]);
-  }
   auto key_at = [&](int i) -> uint32_t { return CACHED ? keys[i] : score_key(src[i]); };
-  for (int i = tid; i < 2 * kMaxBins; i += kThreads) (&sh.cluster_hist[0][0])[i] = 0;
-  // the remote adds of pass 0 may arrive as soon as a neighbour gets there: every block must have
-  // cleared its copies first
-  cluster.sync();
 
-  // ---- three radix passes: bits 31..20, 19..8, 7..0 --------------------------------------------
-  uint32_t prefix = 0, prefix_mask = 0, k_rem = (uint32_t)kk;
-  radix_pass<12>(sh, cluster, nblk, cnt, 20, 0, prefix, prefix_mask, k_rem, key_at);
-  radix_pass<12>(sh, cluster, nblk, cnt, 8, 1, prefix, prefix_mask, k_rem, key_at);
-  radix_pass<8>(sh, cluster, nblk, cnt, 0, 0, prefix, prefix_mask, k_rem, key_at);
-  const uint32_t thr = prefix;        // key of the kk-th largest element
-  const uint32_t need_eq = k_rem;     // how many threshold-equal elements are selected (>= 1)
-
-  // ---- index-ordered compaction ----------------------------------------------------------------
-  const int chunk = ((cnt + kWarps - 1) / kWarps + 31) & ~31;  // contiguous positions per warp
-  const int c_lo = min(cnt, warp * chunk), c_hi = min(cnt, c_lo + chunk);
-  uint32_t gt = 0, eq = 0;
-  for (int i = c_lo + lane; i < c_hi; i += 32) {
-    const uint32_t key = key_at(i);
-    gt += key > thr;
-    eq += key == thr;
-  }
-#pragma unroll
-  for (int d = 16; d >= 1; d >>= 1) {
-    gt += __shfl_xor_sync(0xffffffffu, gt, d);
-    eq += __shfl_xor_sync(0xffffffffu, eq, d);
-  }
-  if (lane == 0) { sh.warp_gt[warp] = gt; sh.warp_eq[warp] = eq; }
+  for (int i = tid; i < kMaxBins; i += kThreads) { sh.local_hist[i] = 0; sh.cluster_hist[0][i] = 0; sh.cluster_hist[1][i] = 0; }
+  if (tid == 0) sh.cand_count = 0;
   __syncthreads();
+
+  // ---- sweep 1: scores -> keys (kept in shared memory) and the 12-bit histogram of this slice --------
+  if (CACHED && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+    const float4* src4 = reinterpret_cast<const float4*>(src);
+    const int n4 = cnt >> 2;
+    constexpr int kBatch = 8;  // 16-byte loads a thread issues before it touches the first of them
+    for (int i0 = 0; i0 < n4; i0 += kThreads * kBatch) {
+      float4 f[kBatch];
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = i0 + u * kThreads + tid;
+        f[u] = i < n4 ? src4[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = i0 + u * kThreads + tid;
+        const bool in = i < n4;
+        const uint32_t k0 = score_key(f[u].x), k1 = score_key(f[u].y), k2 = score_key(f[u].z), k3 = score_key(f[u].w);
+        if (in) *reinterpret_cast<uint4*>(keys + 4 * i) = make_uint4(k0, k1, k2, k3);
+        if (__any_sync(0xffffffffu, in)) {
+          hist_add(sh.local_hist, in, k0 >> 20, lane);
+          hist_add(sh.local_hist, in, k1 >> 20, lane);
+          hist_add(sh.local_hist, in, k2 >> 20, lane);
+          hist_add(sh.local_hist, in, k3 >> 20, lane);
+        }
+      }
+    }
+    for (int i0 = n4 * 4; i0 < cnt; i0 += 32) {  // up to three leftover scores, handled by warp 0
+      if (warp == 0) {
+        const int i = i0 + lane;
+        const uint32_t key = i < cnt ? score_key(src[i]) : 0u;
+        if (i < cnt) keys[i] = key;
+        hist_add(sh.local_hist, i < cnt, key >> 20, lane);
+      }
+    }
+  } else {
+    constexpr int kBatch = 8;
+    for (int i0 = 0; i0 < cnt; i0 += kThreads * kBatch) {
+      float f[kBatch];
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = i0 + u * kThreads + tid;
+        f[u] = i < cnt ? src[i] : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = i0 + u * kThreads + tid;
+        const uint32_t key = score_key(f[u]);
+        if (CACHED && i < cnt) keys[i] = key;
+        hist_add(sh.local_hist, i < cnt, key >> 20, lane);
+      }
+    }
+  }
+  // the remote adds below may land in a neighbour's copy as soon as it exists: every block has
+  // cleared its copies before this barrier
+  cluster.sync();
+  push_hist<4096>(sh, cluster, nblk, 0);
+  cluster.sync();
+  scan_from_top<4096>(sh, sh.cluster_hist[0], (uint32_t)kk, true);
+  const uint32_t digit0 = sh.digit;
+  uint32_t k_rem = sh.k_rem;
+  const uint32_t in_bin = sh.bin_count;  // keys of the whole row that share the threshold's first 12 bits
+
+  const int chunk = ((cnt + kWarps - 1) / kWarps + 31) & ~31;  // contiguous positions per warp in the ordered sweeps
+  const int c_lo = min(cnt, warp * chunk), c_hi = min(cnt, c_lo + chunk);
+  uint32_t thr, need_eq;
+
+  if (in_bin <= (uint32_t)kCandCap) {
+    // ---- short path: sweep 2 counts keys above the bin per warp and collects the bin's keys ----------
+    uint2* cand = reinterpret_cast<uint2*>(sh.cluster_hist[1]);  // (key, slice position), unordered
+    uint32_t gt = 0;
+    for (int i0 = c_lo; i0 < c_hi; i0 += 128) {
+      uint32_t key[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + 32 * u + lane;
+        key[u] = i < c_hi ? key_at(i) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + 32 * u + lane;
+        const uint32_t top = key[u] >> 20;
+        gt += (i < c_hi && top > digit0) ? 1u : 0u;
+        const bool is_c = i < c_hi && top == digit0;
+        const uint32_t cb = __ballot_sync(0xffffffffu, is_c);
+        if (cb != 0u) {
+          uint32_t base = 0;
+          if (lane == 0) base = atomicAdd(&sh.cand_count, (uint32_t)__popc(cb));
+          base = __shfl_sync(0xffffffffu, base, 0);
+          if (is_c) cand[base + __popc(cb & ((1u << lane) - 1u))] = make_uint2(key[u], (uint32_t)i);
+        }
+      }
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) gt += __shfl_xor_sync(0xffffffffu, gt, d);
+    if (lane == 0) { sh.warp_gt[warp] = gt; sh.warp_eq[warp] = 0; }
+    cluster.sync();  // every block's candidate list and count are complete
+    // gather the row's candidates (keys only) into local_hist[0..in_bin)
+    uint32_t* allc = sh.local_hist;
+    uint32_t* hist10 = sh.local_hist + kCandCap;  // 1024 bins
+    {
+      // lane r of every warp reads block r's count; an exclusive scan gives the blocks' offsets
+      const uint32_t nr = lane < nblk ? *cluster.map_shared_rank(&sh.cand_count, lane) : 0u;
+      uint32_t incl = nr;
+#pragma unroll
+      for (int d = 1; d < kMaxCluster; d <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
+      }
+      const uint32_t excl = incl - nr;
+      uint32_t start[kMaxCluster];  // first flat index of each block's list (all lanes hold all eight)
+#pragma unroll
+      for (int q = 0; q < kMaxCluster; ++q) start[q] = q < nblk ? __shfl_sync(0xffffffffu, excl, q) : 0xffffffffu;
+      for (uint32_t i = tid; i < in_bin; i += kThreads) {
+        int r = 0;
+        uint32_t off = 0;
+#pragma unroll
+        for (int q = 1; q < kMaxCluster; ++q)
+          if (i >= start[q]) { r = q; off = start[q]; }
+        const uint2* rc = reinterpret_cast<const uint2*>(cluster.map_shared_rank(&sh.cluster_hist[1][0], r));
+        allc[i] = rc[i - off].x;
+      }
+    }
+    for (int i = tid; i < 1024; i += kThreads) hist10[i] = 0;
+    __syncthreads();
+    // two local 10-bit passes over the candidates: bits 19..10, then 9..0
+    uint32_t prefix = digit0 << 20, prefix_mask = 0xfff00000u;
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+      const int shift = 10 - 10 * pass;
+      for (uint32_t i0 = 0; i0 < in_bin; i0 += kThreads) {
+        const uint32_t i = i0 + tid;
+        const uint32_t key = i < in_bin ? allc[i] : 0u;
+        hist_add(hist10, i < in_bin && (key & prefix_mask) == prefix, (key >> shift) & 1023u, lane);
+      }
+      __syncthreads();
+      scan_from_top<1024>(sh, hist10, k_rem, true);
+      prefix |= sh.digit << shift;
+      prefix_mask |= 1023u << shift;
+      k_rem = sh.k_rem;
+    }
+    thr = prefix;
+    need_eq = k_rem;
+    // per-warp counts of this block: keys above the bin (already counted) plus candidates above / equal to thr
+    const uint32_t my_n = sh.cand_count;
+    for (uint32_t i = tid; i < my_n; i += kThreads) {
+      const uint2 c = cand[i];
+      const int w = (int)c.y / chunk;
+      if (c.x > thr) atomicAdd(&sh.warp_gt[w], 1u);
+      else if (c.x == thr) atomicAdd(&sh.warp_eq[w], 1u);
+    }
+    __syncthreads();
+  } else {
+    // ---- long path: two more cluster-wide radix passes, then a counting sweep ------------------------
+    uint32_t prefix = digit0 << 20, prefix_mask = 0xfff00000u;
+    radix_pass<12>(sh, cluster, nblk, cnt, 8, 1, prefix, prefix_mask, k_rem, key_at);
+    radix_pass<8>(sh, cluster, nblk, cnt, 0, 0, prefix, prefix_mask, k_rem, key_at);
+    thr = prefix;
+    need_eq = k_rem;
+    uint32_t gt = 0, eq = 0;
+    for (int i = c_lo + lane; i < c_hi; i += 32) {
+      const uint32_t key = key_at(i);
+      gt += key > thr;
+      eq += key == thr;
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+      gt += __shfl_xor_sync(0xffffffffu, gt, d);
+      eq += __shfl_xor_sync(0xffffffffu, eq, d);
+    }
+    if (lane == 0) { sh.warp_gt[warp] = gt; sh.warp_eq[warp] = eq; }
+    __syncthreads();
+  }
+
+  // ---- index-ordered compaction ----------------------------------------------------------------------
   if (warp == 0) {
     uint32_t g = lane < kWarps ? sh.warp_gt[lane] : 0u, e = lane < kWarps ? sh.warp_eq[lane] : 0u;
 #pragma unroll
@@ -222,7 +393,7 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
     sh.eq_base = eq_before;
   }
   __syncthreads();
-  // offsets of this warp: selected / threshold-equal elements in lower warps of this block
+  // offsets of this warp: selected / threshold-equal keys in lower warps of this block
   uint32_t out_pos = sh.out_base, eq_rank = sh.eq_base;
   for (int w = 0; w < warp; ++w) {
     const uint32_t e = sh.warp_eq[w];
@@ -231,20 +402,33 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
     eq_rank += e;
   }
   const uint32_t lt_mask = (1u << lane) - 1u;
-  for (int i0 = c_lo; i0 < c_hi; i0 += 32) {
-    const int i = i0 + lane;
-    const uint32_t key = i < c_hi ? key_at(i) : 0u;
-    const bool is_gt = i < c_hi && key > thr;
-    const bool is_eq = i < c_hi && key == thr;
-    const uint32_t eq_ballot = __ballot_sync(0xffffffffu, is_eq);
-    const bool take = is_gt || (is_eq && eq_rank + __popc(eq_ballot & lt_mask) < need_eq);
-    const uint32_t take_ballot = __ballot_sync(0xffffffffu, take);
-    if (take) {
-      const uint32_t pos = out_pos + __popc(take_ballot & lt_mask);
-      if (pos < (uint32_t)kk) out[pos] = lo + i;
+  for (int i0 = c_lo; i0 < c_hi; i0 += 128) {
+    uint32_t key[4], eq_ballot[4], gt_ballot[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + 32 * u + lane;
+      key[u] = i < c_hi ? key_at(i) : 0u;
     }
-    out_pos += __popc(take_ballot);
-    eq_rank += __popc(eq_ballot);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + 32 * u + lane;
+      gt_ballot[u] = __ballot_sync(0xffffffffu, i < c_hi && key[u] > thr);
+      eq_ballot[u] = __ballot_sync(0xffffffffu, i < c_hi && key[u] == thr);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + 32 * u + lane;
+      const bool is_gt = (gt_ballot[u] >> lane) & 1u, is_eq = (eq_ballot[u] >> lane) & 1u;
+      // threshold-equal keys are taken in position order until need_eq of them are in
+      const bool take = is_gt || (is_eq && eq_rank + __popc(eq_ballot[u] & lt_mask) < need_eq);
+      const uint32_t take_ballot = __ballot_sync(0xffffffffu, take);
+      if (take) {
+        const uint32_t pos = out_pos + __popc(take_ballot & lt_mask);
+        if (pos < (uint32_t)kk) out[pos] = lo + i;
+      }
+      out_pos += __popc(take_ballot);
+      eq_rank += __popc(eq_ballot[u]);
+    }
   }
   cluster.sync();  // no block may exit while a neighbour can still read its shared memory
 }
@@ -262,13 +446,15 @@ TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev) {
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   while (pow2 < kMaxCluster && rows * pow2 * 2 <= dev.sm_count && p.max_seq_len / (pow2 * 2) >= 2048) pow2 <<= 1;
   plan.cluster = pow2;
-  const int per = (p.max_seq_len + plan.cluster - 1) / plan.cluster;
+  const int per = (((p.max_seq_len + plan.cluster - 1) / plan.cluster) + 3) & ~3;
   const size_t want = sizeof(Shared) + (size_t)per * sizeof(uint32_t);
-  if (want <= (size_t)dev.max_smem_optin) {
+  // two blocks per SM: each may use half of the SM's shared memory less the per-block reservation
+  const size_t half_sm = ((size_t)dev.max_smem_optin + 1024) / 2 - 1024;
+  if (want <= half_sm || (want <= (size_t)dev.max_smem_optin && rows * plan.cluster <= dev.sm_count)) {
     plan.slice_cap = per;
     plan.smem_bytes = want;
   } else {
-    plan.slice_cap = 0;  // slice too long for shared memory: keys are recomputed from global memory each pass
+    plan.slice_cap = 0;  // slice too long for shared memory: keys are recomputed from global memory in every sweep
     plan.smem_bytes = sizeof(Shared);
   }
   return plan;
