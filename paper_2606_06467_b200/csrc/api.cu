@@ -159,7 +159,7 @@ clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t*
   CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
-  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, 1, dev,
+  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, 1, 0, dev,
                                       static_cast<cudaStream_t>(stream)));
 }
 
@@ -197,7 +197,7 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
     // was complete before its predecessor started (the index, the caches, the caller's queries), so it
     // may overlap its predecessor's tail.
     err = launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p->sweep + l) & 1,
-                             l == 0 ? 1 : 0, dev, s);
+                             l == 0 ? 1 : 0, l + 1 < p->num_layers ? 1 : 0, dev, s);
     if (err != cudaSuccess) return CLSA_ERR_CUDA;
   }
   return CLSA_OK;
@@ -262,7 +262,7 @@ clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, con
   if (launch_topk(*p, scores, stride, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
   for (int l = 0; l < p->num_layers; ++l)
     if (launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p->sweep + l) & 1,
-                           l == 0 ? 1 : 0, dev, s) != cudaSuccess)
+                           l == 0 ? 1 : 0, l + 1 < p->num_layers ? 1 : 0, dev, s) != cudaSuccess)
       return CLSA_ERR_CUDA;
   return CLSA_OK;
 }

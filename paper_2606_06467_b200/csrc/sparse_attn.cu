@@ -55,12 +55,30 @@ struct AttnArgs {
   int q_per_seq, num_q_heads, num_kv_heads, group, top_k;
   int heads_per_block, subs, reverse;
   int wait_prior;  // 1: inputs may come from the kernel launched just before this one (wait for it first)
+  int keep_permille;  // share of each warp's sweep (its end) whose rows are asked to stay in L2 for the next layer
   float scale_log2;
 };
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+// 16-byte asynchronous copy global -> shared with an L2 eviction-priority hint.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid, uint64_t policy) {
   const int bytes = valid ? 16 : 0;  // 0 source bytes: the 16 destination bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;\n"
+               ::"r"(dst), "l"(src), "r"(bytes), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
@@ -188,8 +206,17 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
       const int tt = stage_t0(i) + lane;
       return tt < t_hi ? row_idx[tt] : -1;
     };
+    // L2 residency across layers: consecutive layers walk the same rows in opposite directions, so
+    // the rows a warp reads LAST are the ones the next layer reads FIRST. Those are fetched with the
+    // evict_last priority; everything else (including their re-read by the next layer, which
+    // demotes them again) with evict_first, so that the protected share of the gathered set fits L2.
+    // (A launch that protects nothing leaves the replacement policy alone.)
+    const uint64_t pol_keep = l2_policy_evict_last();
+    const uint64_t pol_stream = a.keep_permille > 0 ? l2_policy_evict_first() : l2_policy_evict_normal();
+    const int keep_from = nstages - (nstages * a.keep_permille + 500) / 1000;  // steps >= keep_from are kept
     auto issue = [&](int i, int my_idx) {
       if (i < nstages) {
+        const uint64_t pol = i >= keep_from ? pol_keep : pol_stream;
         const int buf = i % kAttnStages;
         const uint32_t kdst = ring_u32 + buf * kStageBytes, vdst = kdst + kStageBytes / 2;
         const bool in_range = my_idx >= 0 && my_idx < n;
@@ -204,8 +231,8 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
           const bool ok = (okmask >> j) & 1u;
           const int64_t off = (s0 + (ok ? tok : 0)) * a.tok_stride;
           const uint32_t sw = (uint32_t)(j * 256 + (((lane & 15) ^ (j & 7)) << 4));
-          cp_async16(kdst + sw, kbase + off, ok);
-          cp_async16(vdst + sw, vbase + off, ok);
+          cp_async16(kdst + sw, kbase + off, ok, pol);
+          cp_async16(vdst + sw, vbase + off, ok, pol);
         }
       }
       cp_async_commit();
@@ -441,8 +468,8 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev) {
 }
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
-                               float* lse, uint32_t* status, int reverse, int wait_prior, const DeviceInfo& dev,
-                               cudaStream_t stream) {
+                               float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
+                               const DeviceInfo& dev, cudaStream_t stream) {
   const AttnPlan plan = make_attn_plan(p, dev);
   AttnArgs a;
   a.q = static_cast<const uint16_t*>(q);
@@ -466,6 +493,13 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.subs = plan.subs;
   a.reverse = reverse;
   a.wait_prior = wait_prior;
+  {
+    // protect at most about half of L2 with the tail of this layer's sweep
+    const double gathered = (double)p.num_seqs * p.q_per_seq * (double)p.top_k * p.num_kv_heads * 512.0;
+    double share = 0.5 * (double)dev.l2_bytes / gathered;
+    if (share > 1.0) share = 1.0;
+    a.keep_permille = keep_for_next ? (int)(share * 1000.0) : 0;
+  }
   a.scale_log2 = p.sm_scale * kLog2e;
   auto kernel = a.group <= 8 ? sparse_attn_kernel<1> : sparse_attn_kernel<2>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
