@@ -37,6 +37,7 @@ def parse():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="headline128k")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--block-size", type=int, default=0, help="page the caches into scattered blocks of this many rows")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-breakdown", action="store_true", help="skip the per-kernel instrumented loop")
     return ap.parse_args()
@@ -247,11 +248,14 @@ def run_ours(args):
     c = w.cfg
     T = c.q_per_seq
     t = w.to_device(dev)
+    if args.block_size:
+        t = w.paginate_device(t, args.block_size)
     L = c.num_layers
     p = clsa.make_params(num_seqs=c.num_seqs, num_q_heads=c.num_q_heads, num_kv_heads=c.num_kv_heads,
                          head_dim=c.head_dim, idx_dim=c.idx_dim, top_k=c.top_k, num_layers=L, max_seq_len=w.max_seq_len,
                          sm_scale=c.sm_scale, seq_start=t["seq_start"], seq_len=t["seq_len"], k_cache=t["k_cache"],
-                         v_cache=t["v_cache"], idx_k_cache=t["idx_k_cache"], q_per_seq=T, causal=c.causal)
+                         v_cache=t["v_cache"], idx_k_cache=t["idx_k_cache"], q_per_seq=T, causal=c.causal,
+                         block_table=t.get("block_table"), block_size=args.block_size)
     ws = torch.zeros(clsa.clsa_workspace_bytes(p), dtype=torch.uint8, device=dev)
     idx = torch.empty((c.num_seqs, T, c.top_k), dtype=torch.int32, device=dev)
     cnt = torch.empty((c.num_seqs, T), dtype=torch.int32, device=dev)
@@ -425,7 +429,8 @@ def run_ours(args):
             "config": {"workload": c.name, "num_seqs": c.num_seqs, "context": c.ctx, "top_k": c.top_k, "layers": L,
                        "q_heads": c.num_q_heads, "kv_heads": c.num_kv_heads, "idx_dim": c.idx_dim,
                        "algorithmic_bytes_per_step": alg_bytes, "l2": "flushed between steps (512 MiB rewrite, then 256 MiB read so no dirty lines remain)",
-                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "cache_layout": f"paged, {args.block_size}-row blocks" if args.block_size else "contiguous sequences"},
             "clocks": clocks, "roofline": roofline, "breakdown_us": breakdown, "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms / K,

@@ -23,7 +23,8 @@
  *   than max_seq_len) never trap: the offending element is skipped and a bit is set in the status
  *   word at the start of the workspace (see clsa_device_status).
  * Layout: bf16 = IEEE bfloat16 bit patterns. Strides are in elements. Cache rows of sequence b are
- *   rows seq_start[b] .. seq_start[b] + seq_len[b] - 1 of one row space shared by K, V and K_idx.
+ *   rows seq_start[b] .. seq_start[b] + seq_len[b] - 1 of one row space shared by K, V and K_idx (or, with a
+ *   block table, the rows of its blocks: see clsa_params).
  *   The last q_per_seq tokens of a sequence are its query tokens (their own K/V/K_idx rows have
  *   already been appended by the caller).
  * Visibility: with causal == 0 every query sees all seq_len[b] tokens (decoding); with causal == 1
@@ -89,6 +90,13 @@ typedef struct {
   int64_t idx_token_stride; /* multiple of 8 */
   int64_t num_cache_rows;   /* rows of the cache row space (the extent of idx_k_cache); required when q_per_seq > 1,
                                where tiled bulk copies need the bound; ignored (may be 0) when q_per_seq == 1 */
+  /* Paged caches (optional). With block_table == NULL sequence b occupies the contiguous rows starting at
+   * seq_start[b]. Otherwise the row space is cut into blocks of block_size rows and position s of sequence b is
+   * cache row  block_table[b * max_blocks_per_seq + s / block_size] * block_size + s % block_size  (the same
+   * mapping for K, V and K_idx); seq_start is then ignored and may be NULL. */
+  const int32_t* block_table; /* int32 [B][max_blocks_per_seq] physical block numbers, or NULL */
+  int32_t block_size;         /* a power of two, 16 .. 4096 (paged only) */
+  int32_t max_blocks_per_seq; /* >= ceil(max_seq_len / block_size) (paged only) */
 } clsa_params;
 
 /* Bytes of workspace that any of the calls below may need for these params (the maximum over the
@@ -105,7 +113,8 @@ CLSA_API clsa_status clsa_workspace_bytes(const clsa_params* p, size_t* bytes);
  *   scores fp32 [B][T][score_stride], score_stride >= max_seq_len
  * T == 1 streams the indexer-key cache once (HBM-bound); T > 1 is a tensor-core GEMM (tcgen05, operands staged by
  * TMA), which needs p->num_cache_rows and, for 32-byte vector stores, a 32-byte aligned `scores` with
- * score_stride % 8 == 0 (otherwise it falls back to scalar stores of the same values). */
+ * score_stride % 8 == 0 (otherwise it falls back to scalar stores of the same values). Paged caches are supported for
+ * T == 1 only (T > 1 with a block table returns CLSA_ERR_UNSUPPORTED). */
 CLSA_API clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* scores, int64_t score_stride,
                               void* workspace, size_t workspace_bytes, clsa_stream stream);
 

@@ -35,6 +35,7 @@ class _Problem(ctypes.Structure):
         ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
         ("kv_token_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64),
         ("idx_k_cache", ctypes.c_void_p), ("idx_token_stride", ctypes.c_int64),
+        ("block_table", ctypes.c_void_p), ("block_size", ctypes.c_int32), ("max_blocks_per_seq", ctypes.c_int32),
     ]
 
 
@@ -71,7 +72,8 @@ class Problem:
     """
 
     def __init__(self, *, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim, idx_dim, top_k,
-                 causal=0, sm_scale, seq_start, seq_len, k_cache=None, v_cache=None, idx_k_cache=None):
+                 causal=0, sm_scale, seq_start, seq_len, k_cache=None, v_cache=None, idx_k_cache=None,
+                 block_table=None, block_size=0):
         self.B, self.T, self.Hq, self.Hkv = int(num_seqs), int(q_per_seq), int(num_q_heads), int(num_kv_heads)
         self.D, self.d_idx, self.k, self.causal = int(head_dim), int(idx_dim), int(top_k), int(causal)
         self.seq_start = _c(seq_start, np.int64)
@@ -94,6 +96,12 @@ class Problem:
         if self.idx_k_cache is not None:
             assert self.idx_k_cache.ndim == 2 and self.idx_k_cache.shape[1] == self.d_idx
             s.idx_k_cache, s.idx_token_stride = _ptr(self.idx_k_cache), self.d_idx
+        self.block_table = None
+        if block_table is not None:
+            self.block_table = _c(block_table, np.int32)
+            assert self.block_table.ndim == 2 and self.block_table.shape[0] == self.B
+            s.block_table = _ptr(self.block_table)
+            s.block_size, s.max_blocks_per_seq = int(block_size), int(self.block_table.shape[1])
         self._s = s
 
     @property
@@ -160,10 +168,11 @@ class Problem:
         return {"scores": scores, "idx": idx, "count": count, "out": out, "lse": lse}
 
 
-def problem_from_workload(w, k_cache=None, v_cache=None, idx_k_cache=None) -> Problem:
+def problem_from_workload(w, k_cache=None, v_cache=None, idx_k_cache=None, block_table=None, block_size=0) -> Problem:
     """Problem for a `workloads.Workload` (duck-typed: only its cfg fields and packing are read)."""
     c = w.cfg
     return Problem(num_seqs=c.num_seqs, q_per_seq=c.q_per_seq, num_q_heads=c.num_q_heads,
                    num_kv_heads=c.num_kv_heads, head_dim=c.head_dim, idx_dim=c.idx_dim, top_k=c.top_k,
                    causal=c.causal, sm_scale=c.sm_scale, seq_start=w.seq_start, seq_len=w.seq_len,
-                   k_cache=k_cache, v_cache=v_cache, idx_k_cache=idx_k_cache)
+                   k_cache=k_cache, v_cache=v_cache, idx_k_cache=idx_k_cache, block_table=block_table,
+                   block_size=block_size)

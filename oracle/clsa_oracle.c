@@ -48,6 +48,9 @@ typedef struct {
   int64_t kv_token_stride, kv_head_stride;
   const uint16_t* idx_k_cache; /* bf16 [rows][d_idx] */
   int64_t idx_token_stride;
+  /* optional paging: position s of sequence b lives in block block_table[b][s / block_size] */
+  const int32_t* block_table; /* [B][max_blocks_per_seq] or NULL (contiguous sequences) */
+  int32_t block_size, max_blocks_per_seq;
 } oracle_problem;
 
 static double bf16_to_double(uint16_t h) {
@@ -55,6 +58,13 @@ static double bf16_to_double(uint16_t h) {
   float f;
   memcpy(&f, &u, sizeof f);
   return (double)f;
+}
+
+/* cache row that holds position s of sequence b */
+static int64_t cache_row(const oracle_problem* p, int b, int64_t s) {
+  if (p->block_table == NULL) return p->seq_start[b] + s;
+  const int64_t block = p->block_table[(int64_t)b * p->max_blocks_per_seq + s / p->block_size];
+  return block * p->block_size + s % p->block_size;
 }
 
 /* number of cached tokens query t of sequence b may attend to */
@@ -76,7 +86,7 @@ void oracle_index_scores(const oracle_problem* p, const uint16_t* q_idx, double*
       double* out = scores + ((int64_t)b * T + t) * score_stride;
       const int64_t v = visible_tokens(p, b, t);
       for (int64_t s = 0; s < v; ++s) {
-        const uint16_t* key = p->idx_k_cache + (p->seq_start[b] + s) * p->idx_token_stride;
+        const uint16_t* key = p->idx_k_cache + cache_row(p, b, s) * p->idx_token_stride;
         double acc = 0.0;
         for (int j = 0; j < d; ++j) acc += bf16_to_double(q[j]) * bf16_to_double(key[j]);
         out[s] = acc;
@@ -191,7 +201,7 @@ void oracle_sparse_attn(const oracle_problem* p, const uint16_t* q, const int32_
         double* z = (double*)malloc(sizeof(double) * (size_t)c);
         double m = -INFINITY;
         for (int32_t i = 0; i < c; ++i) {
-          const uint16_t* kr = p->k_cache + (p->seq_start[b] + sel[i]) * p->kv_token_stride + g * p->kv_head_stride;
+          const uint16_t* kr = p->k_cache + cache_row(p, b, sel[i]) * p->kv_token_stride + g * p->kv_head_stride;
           double acc = 0.0;
           for (int d = 0; d < D; ++d) acc += bf16_to_double(qv[d]) * bf16_to_double(kr[d]);
           z[i] = p->sm_scale * acc;
@@ -200,7 +210,7 @@ void oracle_sparse_attn(const oracle_problem* p, const uint16_t* q, const int32_
         double denom = 0.0;
         for (int32_t i = 0; i < c; ++i) {
           const double w = exp(z[i] - m);
-          const uint16_t* vr = p->v_cache + (p->seq_start[b] + sel[i]) * p->kv_token_stride + g * p->kv_head_stride;
+          const uint16_t* vr = p->v_cache + cache_row(p, b, sel[i]) * p->kv_token_stride + g * p->kv_head_stride;
           denom += w;
           for (int d = 0; d < D; ++d) o[d] += w * bf16_to_double(vr[d]);
         }
@@ -226,7 +236,7 @@ void oracle_dense_attn(const oracle_problem* p, const uint16_t* q, double* out, 
         double* logits = (double*)malloc(sizeof(double) * (size_t)(v > 0 ? v : 1));
         double top = -INFINITY;
         for (int64_t s = 0; s < v; ++s) {
-          const uint16_t* kr = p->k_cache + (p->seq_start[b] + s) * p->kv_token_stride + head_off;
+          const uint16_t* kr = p->k_cache + cache_row(p, b, s) * p->kv_token_stride + head_off;
           double dot = 0.0;
           for (int d = 0; d < D; ++d) dot += bf16_to_double(kr[d]) * bf16_to_double(qv[d]);
           logits[s] = dot * p->sm_scale;
@@ -238,7 +248,7 @@ void oracle_dense_attn(const oracle_problem* p, const uint16_t* q, double* out, 
           double acc = 0.0;
           for (int64_t s = 0; s < v; ++s)
             acc += (logits[s] / total) *
-                   bf16_to_double(p->v_cache[(p->seq_start[b] + s) * p->kv_token_stride + head_off + d]);
+                   bf16_to_double(p->v_cache[cache_row(p, b, s) * p->kv_token_stride + head_off + d]);
           out[r * D + d] = acc;
         }
         if (lse) lse[r] = v > 0 ? top + log(total) : -INFINITY;

@@ -37,6 +37,7 @@ class clsa_params(ctypes.Structure):
         ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
         ("kv_token_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64),
         ("idx_k_cache", ctypes.c_void_p), ("idx_token_stride", ctypes.c_int64), ("num_cache_rows", ctypes.c_int64),
+        ("block_table", ctypes.c_void_p), ("block_size", ctypes.c_int32), ("max_blocks_per_seq", ctypes.c_int32),
     ]
 
 
@@ -100,7 +101,7 @@ def _nbytes(ws, ws_bytes):
 def make_params(*, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim=128, idx_dim, top_k, num_layers=1,
                 causal=0, max_seq_len, sm_scale, sweep=0, seq_start=None, seq_len=None, k_cache=None, v_cache=None,
                 kv_token_stride=None, kv_head_stride=None, idx_k_cache=None, idx_token_stride=None,
-                num_cache_rows=None) -> clsa_params:
+                num_cache_rows=None, block_table=None, block_size=0, max_blocks_per_seq=None) -> clsa_params:
     """Fill a clsa_params. Tensor arguments contribute their device address (and, for the caches, their strides
     unless given); the caller keeps them alive while the struct is in use."""
     p = clsa_params()
@@ -119,6 +120,11 @@ def make_params(*, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim=12
     if num_cache_rows is None and idx_k_cache is not None and not isinstance(idx_k_cache, int):
         num_cache_rows = idx_k_cache.shape[0]
     p.num_cache_rows = num_cache_rows or 0
+    p.block_table = _ptr(block_table)
+    p.block_size = block_size
+    if max_blocks_per_seq is None and block_table is not None and not isinstance(block_table, int):
+        max_blocks_per_seq = block_table.shape[1]
+    p.max_blocks_per_seq = max_blocks_per_seq or 0
     return p
 
 

@@ -64,8 +64,15 @@ clsa_status check_shape(const clsa_params* p) {
 }
 
 clsa_status check_seq(const clsa_params* p) {
-  if (p->seq_start == nullptr || p->seq_len == nullptr) return CLSA_ERR_INVALID_ARG;
-  if (!aligned(p->seq_start, 8) || !aligned(p->seq_len, 4)) return CLSA_ERR_INVALID_ARG;
+  if (p->seq_len == nullptr || !aligned(p->seq_len, 4)) return CLSA_ERR_INVALID_ARG;
+  if (p->block_table == nullptr) {
+    if (p->seq_start == nullptr || !aligned(p->seq_start, 8)) return CLSA_ERR_INVALID_ARG;
+  } else {
+    if (!aligned(p->block_table, 4)) return CLSA_ERR_INVALID_ARG;
+    const int bs = p->block_size;
+    if (bs < 16 || bs > 4096 || (bs & (bs - 1)) != 0) return CLSA_ERR_INVALID_ARG;
+    if ((int64_t)p->max_blocks_per_seq * bs < p->max_seq_len) return CLSA_ERR_INVALID_ARG;
+  }
   return CLSA_OK;
 }
 
@@ -119,6 +126,7 @@ clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* sc
   CLSA_TRY(check_idx_cache(p));
   if (q_idx == nullptr || scores == nullptr || !aligned(q_idx, 16) || !aligned(scores, 4)) return CLSA_ERR_INVALID_ARG;
   if (score_stride < p->max_seq_len) return CLSA_ERR_INVALID_ARG;
+  if (p->q_per_seq > 1 && p->block_table != nullptr) return CLSA_ERR_UNSUPPORTED;  // the GEMM path reads contiguous key tiles
   if (p->q_per_seq > 1) {
     // the GEMM path addresses rows through 32-bit TMA coordinates and needs the extent of the cache
     if (p->num_cache_rows < 1 || p->num_cache_rows > 0x7fffffffLL) return CLSA_ERR_INVALID_ARG;

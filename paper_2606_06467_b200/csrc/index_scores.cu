@@ -21,7 +21,8 @@ __global__ void __launch_bounds__(kThreads, 4)
 index_scores_decode_kernel(const uint16_t* __restrict__ kidx, int64_t tok_stride, const uint16_t* __restrict__ q_idx,
                            const int64_t* __restrict__ seq_start, const int32_t* __restrict__ seq_len,
                            float* __restrict__ scores, int64_t score_stride, int num_seqs, int tiles_per_seq,
-                           int max_seq_len, uint32_t* status) {
+                           int max_seq_len, const int32_t* __restrict__ block_table, int block_shift, int max_blocks,
+                           uint32_t* status) {
   constexpr int LPR = DIDX / 8;               // lanes per key row
   constexpr int RPI = 32 / LPR;               // rows covered by one warp-wide load
   constexpr int ROWS_PER_WARP = RPI * kLoads;
@@ -49,13 +50,28 @@ index_scores_decode_kernel(const uint16_t* __restrict__ kidx, int64_t tok_stride
       q[4] = bf16_lo(qw.z); q[5] = bf16_hi(qw.z); q[6] = bf16_lo(qw.w); q[7] = bf16_hi(qw.w);
       cur_b = b;
     }
-    const uint16_t* base = kidx + (seq_start[b] + row0 + sub) * tok_stride + col;
-
     uint4 kw[kLoads];
+    if (block_table == nullptr) {
+      const uint16_t* base = kidx + (seq_start[b] + row0 + sub) * tok_stride + col;
 #pragma unroll
-    for (int u = 0; u < kLoads; ++u) {
-      const int r = row0 + u * RPI + sub;
-      kw[u] = r < n ? __ldcs(reinterpret_cast<const uint4*>(base + (int64_t)u * RPI * tok_stride)) : make_uint4(0, 0, 0, 0);
+      for (int u = 0; u < kLoads; ++u) {
+        const int r = row0 + u * RPI + sub;
+        kw[u] = r < n ? __ldcs(reinterpret_cast<const uint4*>(base + (int64_t)u * RPI * tok_stride)) : make_uint4(0, 0, 0, 0);
+      }
+    } else {
+      // paged cache: position r lives in block table[b][r >> shift] at offset r & (block_size - 1)
+      const int32_t* table = block_table + (int64_t)b * max_blocks;
+      int64_t prow[kLoads];
+#pragma unroll
+      for (int u = 0; u < kLoads; ++u) {
+        const int r = row0 + u * RPI + sub;
+        prow[u] = r < n ? ((int64_t)__ldg(table + (r >> block_shift)) << block_shift) + (r & ((1 << block_shift) - 1)) : 0;
+      }
+#pragma unroll
+      for (int u = 0; u < kLoads; ++u) {
+        const int r = row0 + u * RPI + sub;
+        kw[u] = r < n ? __ldcs(reinterpret_cast<const uint4*>(kidx + prow[u] * tok_stride + col)) : make_uint4(0, 0, 0, 0);
+      }
     }
     float v[kLoads];
 #pragma unroll
@@ -110,14 +126,16 @@ cudaError_t launch_index_scores_decode(const clsa_params& p, const void* q_idx, 
   if (grid > total) grid = total;
   auto kidx = static_cast<const uint16_t*>(p.idx_k_cache);
   auto q = static_cast<const uint16_t*>(q_idx);
+  int block_shift = 0;
+  while (p.block_table != nullptr && (1 << block_shift) < p.block_size) ++block_shift;
   if (p.idx_dim == 128) {
     index_scores_decode_kernel<128><<<(unsigned)grid, kThreads, 0, stream>>>(
         kidx, p.idx_token_stride, q, p.seq_start, p.seq_len, scores, score_stride, p.num_seqs, tiles_per_seq,
-        p.max_seq_len, status);
+        p.max_seq_len, p.block_table, block_shift, p.max_blocks_per_seq, status);
   } else {
     index_scores_decode_kernel<64><<<(unsigned)grid, kThreads, 0, stream>>>(
         kidx, p.idx_token_stride, q, p.seq_start, p.seq_len, scores, score_stride, p.num_seqs, tiles_per_seq,
-        p.max_seq_len, status);
+        p.max_seq_len, p.block_table, block_shift, p.max_blocks_per_seq, status);
   }
   return cudaGetLastError();
 }

@@ -33,6 +33,7 @@ namespace clsa {
 namespace {
 
 constexpr int kThreads = kAttnWarps * 32;
+static_assert(kAttnStages == 3, "the position pipeline in the kernel is written for a 3-deep ring");
 constexpr int kStageBytes = kAttnStageTokens * 256 * 2;  // 16 K rows + 16 V rows of 256 bytes
 constexpr int kWarpRingBytes = kAttnStages * kStageBytes;
 constexpr int kPartialStride = 132;                      // floats per head of a partial: 128 outputs, max, sum, pad
@@ -49,6 +50,8 @@ struct AttnArgs {
   const int32_t* seq_len;
   const int32_t* idx;
   const int32_t* count;
+  const int32_t* block_table;  // paged caches: [B][max_blocks] physical block numbers, or nullptr
+  int block_shift, max_blocks;
   uint16_t* out;
   float* lse;
   uint32_t* status;
@@ -112,7 +115,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
 }
 
 // NT = number of 8-head tiles that hold the query heads of one KV head (1 for groups up to 8, 2 up to 16).
-template <int NT>
+template <int NT, bool PAGED>
 __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   cg::cluster_group cluster = cg::this_cluster();
@@ -152,14 +155,22 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   const int32_t* row_idx = a.idx + r * a.top_k;
   int cnt = a.count[r];
   const int b = (int)(r / a.q_per_seq);
-  const int64_t s0 = a.seq_start[b];
+  constexpr bool paged = PAGED;
+  const int64_t s0 = paged ? 0 : a.seq_start[b];  // paged: positions are translated to cache rows when they are fetched
+  const int32_t* table = paged ? a.block_table + (int64_t)b * a.max_blocks : nullptr;
   const int n = a.seq_len[b];
-  // speculative fetch of the first/last 16 positions of the range (entries past the count are unused)
-  int first_idx = -1;
+  // Positions are fetched two pipeline steps before they are used and (paged caches) their block numbers one
+  // step before, so that no load is consumed in the step that issued it. The first four steps' positions are
+  // fetched here, speculatively for a range that lies entirely below the row's count (entries past the count
+  // are never used).
+  const int nst_full = (slot_hi - slot_lo + kAttnStageTokens - 1) / kAttnStageTokens;
+  int spec_raw[4] = {-1, -1, -1, -1};
   if (active && lane < kAttnStageTokens) {
-    const int nst = (slot_hi - slot_lo + kAttnStageTokens - 1) / kAttnStageTokens;
-    const int tt = slot_lo + (a.reverse ? (nst - 1) * kAttnStageTokens : 0) + lane;
-    if (tt < slot_hi) first_idx = row_idx[tt];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int tt = slot_lo + (a.reverse ? nst_full - 1 - i : i) * kAttnStageTokens + lane;
+      if (i < nst_full && tt < slot_hi) spec_raw[i] = row_idx[tt];
+    }
   }
   if (cnt < 0 || cnt > a.top_k) {
     if (threadIdx.x == 0 && crank == 0 && blockIdx.y == 0) flag_status(a.status, CLSA_DEV_BAD_COUNT);
@@ -200,11 +211,16 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
 
     // token offset of pipeline step i
     auto stage_t0 = [&](int i) { return t_lo + (a.reverse ? nstages - 1 - i : i) * kAttnStageTokens; };
-    // lanes 0..15 fetch the 16 positions of step i (-1 past the end)
-    auto load_idx = [&](int i) -> int {
+    // lanes 0..15 fetch the 16 positions of step i (-1 past the end); the value is not touched here
+    auto load_raw = [&](int i) -> int {
       if (i >= nstages || lane >= kAttnStageTokens) return -1;
       const int tt = stage_t0(i) + lane;
       return tt < t_hi ? row_idx[tt] : -1;
+    };
+    // paged caches: block number of a position fetched at least one step ago (not touched here either)
+    auto load_blk = [&](int raw) -> int {
+      if (!paged || raw < 0 || raw >= n) return 0;
+      return __ldg(table + (raw >> a.block_shift));
     };
     // L2 residency across layers: consecutive layers walk the same rows in opposite directions, so
     // the rows a warp reads LAST are the ones the next layer reads FIRST. Those are fetched with the
@@ -214,12 +230,14 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
     const uint64_t pol_keep = l2_policy_evict_last();
     const uint64_t pol_stream = a.keep_permille > 0 ? l2_policy_evict_first() : l2_policy_evict_normal();
     const int keep_from = nstages - (nstages * a.keep_permille + 500) / 1000;  // steps >= keep_from are kept
-    auto issue = [&](int i, int my_idx) {
+    auto issue = [&](int i, int raw, int blk) {
       if (i < nstages) {
         const uint64_t pol = i >= keep_from ? pol_keep : pol_stream;
         const int buf = i % kAttnStages;
         const uint32_t kdst = ring_u32 + buf * kStageBytes, vdst = kdst + kStageBytes / 2;
-        const bool in_range = my_idx >= 0 && my_idx < n;
+        const bool in_range = raw >= 0 && raw < n;
+        // cache row relative to s0: the position itself, or its place inside its block
+        const int my_idx = paged ? (blk << a.block_shift) + (raw & ((1 << a.block_shift) - 1)) : raw;
         const uint32_t okmask = __ballot_sync(0xffffffffu, in_range) & 0xffffu;
         const bool bad = lane < kAttnStageTokens && !in_range && (stage_t0(i) + lane) < t_hi;
         if (bad) flag_status(a.status, CLSA_DEV_BAD_INDEX);
@@ -238,25 +256,26 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
       cp_async_commit();
     };
 
-    // prologue: stages 0 .. kAttnStages-2 in flight, positions of the next one in a register
-    int next_idx;
-    if (t_hi == slot_hi) {  // the range is entirely below the count: the speculative fetch was step 0
-      next_idx = first_idx;
-    } else {
-      next_idx = load_idx(0);
+    // prologue: stages 0 and 1 in flight; positions of steps 2 and 3 (and step 2's block numbers) in registers
+    int r0 = spec_raw[0], r1 = spec_raw[1], rawA = spec_raw[2], rawB = spec_raw[3];
+    if (t_hi != slot_hi) {  // the count cuts this range short: fetch the real first positions
+      r0 = load_raw(0); r1 = load_raw(1); rawA = load_raw(2); rawB = load_raw(3);
     }
-#pragma unroll
-    for (int i = 0; i < kAttnStages - 1; ++i) {
-      const int cur = next_idx;
-      next_idx = load_idx(i + 1);
-      issue(i, cur);
+    {
+      const int b0 = load_blk(r0), b1 = load_blk(r1);
+      int blkA_init = load_blk(rawA);
+      issue(0, r0, b0);
+      issue(1, r1, b1);
+      r0 = blkA_init;  // reuse the register: block numbers of step 2
     }
+    int blkA = r0;
 #pragma unroll 1
     for (int i = 0; i < nstages; ++i) {
-      {  // refill the buffer freed by step i-1
-        const int cur = next_idx;
-        next_idx = load_idx(i + kAttnStages);
-        issue(i + kAttnStages - 1, cur);
+      {  // refill the buffer freed by step i-1, then advance the position pipeline
+        issue(i + kAttnStages - 1, rawA, blkA);
+        rawA = rawB;
+        blkA = load_blk(rawB);
+        rawB = load_raw(i + kAttnStages + 1);
       }
       cp_async_wait<kAttnStages - 1>();
       __syncwarp();
@@ -419,7 +438,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
 static int max_resident_blocks(int cluster, size_t smem_bytes) {
   static int cache[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
   if (cache[cluster] != 0) return cache[cluster];
-  cudaFuncSetAttribute(sparse_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  cudaFuncSetAttribute(sparse_attn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)cluster * 64, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -432,7 +451,7 @@ static int max_resident_blocks(int cluster, size_t smem_bytes) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, sparse_attn_kernel<1>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+  if (cudaOccupancyMaxActiveClusters(&n, sparse_attn_kernel<1, false>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
   cache[cluster] = n * cluster;
   return cache[cluster];
 }
@@ -481,6 +500,10 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.seq_len = p.seq_len;
   a.idx = idx;
   a.count = count;
+  a.block_table = p.block_table;
+  a.block_shift = 0;
+  while (p.block_table != nullptr && (1 << a.block_shift) < p.block_size) ++a.block_shift;
+  a.max_blocks = p.max_blocks_per_seq;
   a.out = static_cast<uint16_t*>(out);
   a.lse = lse;
   a.status = status;
@@ -501,7 +524,8 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
     a.keep_permille = keep_for_next ? (int)(share * 1000.0) : 0;
   }
   a.scale_log2 = p.sm_scale * kLog2e;
-  auto kernel = a.group <= 8 ? sparse_attn_kernel<1> : sparse_attn_kernel<2>;
+  auto kernel = a.group <= 8 ? (p.block_table ? sparse_attn_kernel<1, true> : sparse_attn_kernel<1, false>)
+                             : (p.block_table ? sparse_attn_kernel<2, true> : sparse_attn_kernel<2, false>);
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;

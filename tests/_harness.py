@@ -31,17 +31,20 @@ OUT_MEAN_ABS = 2e-3
 class GpuProblem:
     """Device tensors, params and workspace of one workload."""
 
-    def __init__(self, w: Workload, device="cuda:0", layers=None):
+    def __init__(self, w: Workload, device="cuda:0", layers=None, block_size=0):
         self.w, self.cfg = w, w.cfg
         c = w.cfg
         self.dev = torch.device(device)
         self.t = w.to_device(self.dev, layers=layers)
+        if block_size:  # same contents, caches rearranged into scattered blocks
+            self.t = w.paginate_device(self.t, block_size)
         self.L = c.num_layers if layers is None else layers
         self.params = clsa.make_params(
             num_seqs=c.num_seqs, q_per_seq=c.q_per_seq, num_q_heads=c.num_q_heads, num_kv_heads=c.num_kv_heads,
             head_dim=c.head_dim, idx_dim=c.idx_dim, top_k=c.top_k, num_layers=self.L, causal=c.causal,
             max_seq_len=w.max_seq_len, sm_scale=c.sm_scale, seq_start=self.t["seq_start"], seq_len=self.t["seq_len"],
-            k_cache=self.t["k_cache"], v_cache=self.t["v_cache"], idx_k_cache=self.t["idx_k_cache"])
+            k_cache=self.t["k_cache"], v_cache=self.t["v_cache"], idx_k_cache=self.t["idx_k_cache"],
+            block_table=self.t.get("block_table"), block_size=block_size)
         self.ws = torch.zeros(clsa.clsa_workspace_bytes(self.params), dtype=torch.uint8, device=self.dev)
         self.score_stride = (w.max_seq_len + 63) // 64 * 64
         B, T = c.num_seqs, c.q_per_seq

@@ -1,0 +1,76 @@
+"""Paged caches (block tables): the CUDA path on scattered blocks against the oracle on contiguous sequences.
+Paging changes addresses only, so scores, indices and outputs must agree exactly as in the contiguous case --
+and byte for byte with the CUDA path's own contiguous run."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+import __graft_entry__ as entry
+
+entry._load_build_module().build()
+
+import oracle
+import paper_2606_06467_b200 as clsa
+from _harness import GpuProblem, check_attention, check_scores, check_topk_band, check_topk_exact_on_gpu_scores
+from workloads import MID, RAGGED, TINY, Workload
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("cfg,bs", [
+    (MID.replace(num_seqs=3, ctx=5000 + 7, top_k=384, num_layers=3), 16),
+    (RAGGED.replace(num_seqs=5, ctx=9000, ragged_min=100, num_short=2, top_k=700, num_layers=2), 64),
+    (TINY.replace(num_seqs=2, ctx=3000, top_k=128, num_layers=2), 32),
+    (MID.replace(num_seqs=2, ctx=2500, top_k=256, num_layers=2, num_q_heads=20, num_kv_heads=4), 256),
+], ids=["mid-bs16", "ragged-bs64", "tiny-bs32", "paper-heads-bs256"])
+def test_paged_decode_matches_oracle_and_contiguous_run(cfg, bs):
+    w = Workload(cfg)
+    kc, vc = w.host_kv_full()
+    prob = oracle.problem_from_workload(w, k_cache=kc, v_cache=vc, idx_k_cache=w.host_kidx_cache())
+    ref_scores = prob.index_scores(w.q_idx_bits())
+    ref_idx, ref_cnt = prob.topk(ref_scores)
+    flat = GpuProblem(w)
+    flat_outs = flat.decode_step()
+    torch.cuda.synchronize()
+    g = GpuProblem(w, block_size=bs)
+    gs = g.index_scores()
+    check_scores(gs, ref_scores, w)
+    assert torch.equal(gs.nan_to_num(7.0), flat.index_scores().nan_to_num(7.0))
+    outs = g.decode_step()
+    torch.cuda.synchronize()
+    assert g.status() == 0
+    check_topk_exact_on_gpu_scores(prob, gs, g.idx, g.count, w)
+    check_topk_band(ref_scores, ref_idx, ref_cnt, g.idx, g.count, w)
+    assert torch.equal(g.idx, flat.idx) and torch.equal(g.count, flat.count)
+    idx_np, cnt_np = g.idx.cpu().numpy(), g.count.cpu().numpy()
+    for l in range(g.L):
+        check_attention(prob, w, l, outs[l], None, idx_np, cnt_np)
+        assert torch.equal(outs[l].view(torch.int16), flat_outs[l].view(torch.int16))
+    # separate calls on the paged layout too, with LSE
+    out0, lse0 = g.sparse_attn(0)
+    check_attention(prob, w, 0, out0, lse0, idx_np, cnt_np)
+
+
+def test_paged_arguments_are_validated():
+    w = Workload(MID.replace(num_seqs=2, ctx=1000, top_k=64, num_layers=1))
+    g = GpuProblem(w, block_size=16)
+    s = g.new_scores()
+    for bad_bs in (8, 24, 8192):
+        g.params.block_size = bad_bs
+        with pytest.raises(clsa.ClsaError) as e:
+            clsa.clsa_index_scores(g.params, g.t["q_idx"], s, g.score_stride, g.ws)
+        assert e.value.status == clsa.CLSA_ERR_INVALID_ARG
+    g.params.block_size = 16
+    g.params.max_blocks_per_seq = 10          # 160 < 1000 positions
+    with pytest.raises(clsa.ClsaError) as e:
+        clsa.clsa_topk(g.params, s, g.score_stride, g.idx, g.count, g.ws)
+    assert e.value.status == clsa.CLSA_ERR_INVALID_ARG
+    g.params.max_blocks_per_seq = g.t["block_table"].shape[1]
+    g.params.q_per_seq = 4                    # chunked scores on a paged cache are not built
+    g.params.num_cache_rows = g.t["idx_k_cache"].shape[0]
+    with pytest.raises(clsa.ClsaError) as e:
+        clsa.clsa_index_scores(g.params, g.t["q_idx"], s, g.score_stride, g.ws)
+    assert e.value.status == clsa.CLSA_ERR_UNSUPPORTED

@@ -401,3 +401,27 @@ def test_oracle_on_tiny_workload_shape():
     ref_o, ref_l = _np_attention(p, ql[1], [[step["idx"][0, 0].tolist()]])
     np.testing.assert_allclose(step["out"][1], ref_o, rtol=1e-12, atol=1e-13)
     np.testing.assert_allclose(step["lse"][1], ref_l, rtol=1e-12)
+
+
+def test_paged_layout_gives_the_same_results_as_contiguous_sequences():
+    """Paging is addressing only: the oracle on a block-table layout (blocks scattered by a permutation) must
+    return exactly what it returns on contiguous sequences."""
+    from workloads import RAGGED, Workload
+
+    w = Workload(RAGGED.replace(num_seqs=4, ctx=700, ragged_min=40, num_short=1, top_k=64, num_layers=2,
+                                num_q_heads=8, num_kv_heads=2))
+    kc, vc = w.host_kv_full()
+    kidx = w.host_kidx_cache()
+    ql = np.stack([w.q_layer_bits(l) for l in range(2)])
+    flat = oracle.problem_from_workload(w, k_cache=kc, v_cache=vc, idx_k_cache=kidx).decode_step(w.q_idx_bits(), ql)
+    for bs in (16, 64):
+        table, nblocks = w.block_table(bs)
+        assert sorted(table[table >= 0].tolist()).count(0) >= 1 and nblocks == sum((int(n) + bs - 1) // bs for n in w.seq_len)
+        paged = oracle.problem_from_workload(w, k_cache=w.paginate_host(kc, bs), v_cache=w.paginate_host(vc, bs),
+                                             idx_k_cache=w.paginate_host(kidx, bs), block_table=table, block_size=bs)
+        got = paged.decode_step(w.q_idx_bits(), ql)
+        for key in ("idx", "count", "out", "lse"):
+            np.testing.assert_array_equal(got[key], flat[key])
+        for b in range(4):
+            n = int(w.seq_len[b])
+            np.testing.assert_array_equal(got["scores"][b, 0, :n], flat["scores"][b, 0, :n])

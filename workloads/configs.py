@@ -16,6 +16,7 @@ from . import generator as g
 
 TID_Q_IDX, TID_K_IDX, TID_K, TID_V = 0, 1, 2, 3
 TID_LEN, TID_DUP_FLAG, TID_DUP_SRC, TID_PLANT = 4, 5, 6, 7
+TID_BLOCK_PERM = 8
 TID_Q_LAYER0 = 16
 
 
@@ -229,6 +230,57 @@ class Workload:
         k = self.kv_rows_bits("k", rows).reshape(-1, c.num_kv_heads, c.head_dim)
         v = self.kv_rows_bits("v", rows).reshape(-1, c.num_kv_heads, c.head_dim)
         return k, v
+
+    # ------------------------------------------------------------------ paged layout
+    def block_table(self, block_size: int):
+        """(table int32 [B, max_blocks], num_blocks): a hashed permutation scatters the blocks of all sequences over
+        the cache, as a block allocator under churn would."""
+        B = self.cfg.num_seqs
+        per_seq = [(int(n) + block_size - 1) // block_size for n in self.seq_len]
+        total = sum(per_seq)
+        order = np.argsort(g.hash_u64(self.cfg.seed, TID_BLOCK_PERM, np.arange(total, dtype=np.uint64)), kind="stable")
+        table = np.zeros((B, max(per_seq)), dtype=np.int32)
+        pos = 0
+        for b in range(B):
+            table[b, : per_seq[b]] = order[pos: pos + per_seq[b]]
+            pos += per_seq[b]
+        return table, total
+
+    def paged_rows(self, block_size: int):
+        """(src, num_rows): src[r] = contiguous-layout row whose contents sit in paged row r (-1 for padding)."""
+        table, total = self.block_table(block_size)
+        src = np.full(total * block_size, -1, dtype=np.int64)
+        for b in range(self.cfg.num_seqs):
+            n, s0 = int(self.seq_len[b]), int(self.seq_start[b])
+            s = np.arange(n, dtype=np.int64)
+            rows = table[b, s // block_size].astype(np.int64) * block_size + s % block_size
+            src[rows] = s0 + s
+        return src, total * block_size
+
+    def paginate_host(self, arr: np.ndarray, block_size: int) -> np.ndarray:
+        """Rearrange a host cache [total_rows, ...] (contiguous sequences) into the paged layout."""
+        src, nrows = self.paged_rows(block_size)
+        out = np.zeros((nrows,) + arr.shape[1:], dtype=arr.dtype)
+        ok = src >= 0
+        out[ok] = arr[src[ok]]
+        return out
+
+    def paginate_device(self, tensors: dict, block_size: int) -> dict:
+        """Paged copies of the device caches in `tensors` plus the block table (torch)."""
+        import torch
+
+        src, nrows = self.paged_rows(block_size)
+        dev = tensors["k_cache"].device
+        src_t = torch.from_numpy(np.where(src >= 0, src, 0)).to(dev)
+        ok = torch.from_numpy(src >= 0).to(dev)
+        out = dict(tensors)
+        for name in ("k_cache", "v_cache", "idx_k_cache"):
+            t = tensors[name][src_t]
+            t[~ok] = 0
+            out[name] = t.contiguous()
+        table, _ = self.block_table(block_size)
+        out["block_table"] = torch.from_numpy(table).to(dev)
+        return out
 
     # ------------------------------------------------------------------ device tensors
     def to_device(self, device="cuda", layers=None):
