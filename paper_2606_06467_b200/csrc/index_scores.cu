@@ -33,6 +33,8 @@ index_scores_decode_kernel(const uint16_t* __restrict__ kidx, int64_t tok_stride
   const int col = (lane % LPR) * 8;           // first element of this lane's 16 bytes
   const int64_t total_tiles = (int64_t)num_seqs * tiles_per_seq;
 
+  // let a dependent launch (the top-k) be scheduled onto SMs as this grid's blocks retire
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   int cur_b = -1;
   float q[8];
   for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {

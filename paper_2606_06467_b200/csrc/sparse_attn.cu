@@ -272,10 +272,12 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
 #pragma unroll 1
     for (int i = 0; i < nstages; ++i) {
       {  // refill the buffer freed by step i-1, then advance the position pipeline
+        const int raw_new = load_raw(i + kAttnStages + 1);
+        const int blk_new = load_blk(rawB);
         issue(i + kAttnStages - 1, rawA, blkA);
         rawA = rawB;
-        blkA = load_blk(rawB);
-        rawB = load_raw(i + kAttnStages + 1);
+        blkA = blk_new;
+        rawB = raw_new;
       }
       cp_async_wait<kAttnStages - 1>();
       __syncwarp();

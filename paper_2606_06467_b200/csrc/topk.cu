@@ -169,6 +169,11 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
   const int b = row / q_per_seq, t = row % q_per_seq;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+  // Programmatic dependent launch: this grid may have been scheduled before the kernel that writes
+  // the scores has finished; wait for it here, before the first global read, and let the kernel
+  // after this one be scheduled early in turn.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // Everything up to the first cluster.sync() is uniform over the cluster (same row, same lengths).
   const int n = seq_len[b];
   int v = causal ? n - q_per_seq + t + 1 : n;
@@ -472,13 +477,15 @@ cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)plan.cluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, scores, score_stride, p.seq_len, (int)p.q_per_seq, (int)p.causal,
                             (int)p.top_k, (int)p.max_seq_len, idx, count, status);
 }
