@@ -141,11 +141,13 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   const int hcol = (lane & 3) * 2;
   const int h0 = g * G;                // first query head of this KV head
 
-  // Programmatic dependent launch: let the next kernel of the stream start its own prologue as soon
-  // as SMs free up, and (unless the caller vouches that every input predates the previous kernel)
-  // wait for the previous kernel's results before the first global read.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Programmatic dependent launch. Unless the caller vouches that every input predates the previous
+  // kernel, wait for that kernel's results before the first global read; only then let the next
+  // kernel of the stream be scheduled (as SMs free up). The order matters: a kernel launched behind
+  // this one may skip its own wait on the grounds that everything it reads was complete before this
+  // grid started reading -- which holds only if this grid has waited before it releases anybody.
   if (a.wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // The row's k slots are cut into nsplit ranges of `per` slots (a multiple of the stage size); the
   // split does not depend on the row's count, so the first positions can be fetched together with it.
