@@ -37,6 +37,12 @@ def parse():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="headline128k")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--num-seqs", type=int, default=0, help="override the workload's batch size")
+    ap.add_argument("--ctx", type=int, default=0, help="override the workload's context length")
+    ap.add_argument("--top-k", type=int, default=0, help="override the workload's k")
+    ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads")
+    ap.add_argument("--kv-heads", type=int, default=0, help="override the number of KV heads")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of cross-decoder layers")
     ap.add_argument("--block-size", type=int, default=0, help="page the caches into scattered blocks of this many rows")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-breakdown", action="store_true", help="skip the per-kernel instrumented loop")
@@ -128,6 +134,21 @@ def aggregate_value(world: int, bytes_per_rank_step: int, ms_per_step: float) ->
     return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
 
 
+def pick_config(args):
+    """The named workload, with any command-line overrides applied (the name then says so)."""
+    from workloads import CONFIGS
+
+    c = CONFIGS[args.config]
+    over = {}
+    for field, val in (("num_seqs", args.num_seqs), ("ctx", args.ctx), ("top_k", args.top_k),
+                       ("num_q_heads", args.q_heads), ("num_kv_heads", args.kv_heads), ("num_layers", args.layers)):
+        if val:
+            over[field] = val
+    if over:
+        c = c.replace(name=c.name + "+" + ",".join(f"{k}={v}" for k, v in sorted(over.items())), **over)
+    return c
+
+
 def physical_gpu_index(local: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -194,7 +215,7 @@ def run_reference(args):
     from workloads import CONFIGS, Workload
 
     oracle.build()
-    w = Workload(CONFIGS[args.config])
+    w = Workload(pick_config(args))
     c = w.cfg
     seqs = [0]
     sample = f"sequence 0 of {c.num_seqs}, all {c.num_layers} layers, whole context, per step"
@@ -244,7 +265,7 @@ def run_ours(args):
     from workloads import CONFIGS, Workload
 
     dev = torch.device("cuda", local)
-    w = Workload(CONFIGS[args.config])
+    w = Workload(pick_config(args))
     c = w.cfg
     T = c.q_per_seq
     t = w.to_device(dev)
