@@ -60,12 +60,12 @@ __device__ __forceinline__ uint32_t score_key(float x) {
 
 // Adds one to hist[bin] for every lane with `in`; a warp whose voters all share one bin adds once.
 __device__ __forceinline__ void hist_add(uint32_t* hist, bool in, uint32_t bin, int lane) {
-  const uint32_t voters = __ballot_sync(0xffffffffu, in);
-  if (voters == 0u) return;
-  const int leader = __ffs(voters) - 1;
-  const uint32_t lead_bin = __shfl_sync(0xffffffffu, bin, leader);
-  if (__all_sync(0xffffffffu, !in || bin == lead_bin)) {
-    if (lane == leader) atomicAdd(&hist[bin], (uint32_t)__popc(voters));
+  // one vote decides whether the whole warp agrees on one bin
+  int same = 0;
+  const uint32_t voters = __match_all_sync(0xffffffffu, in ? bin : 0xffffffffu, &same);
+  (void)voters;
+  if (same) {
+    if (in && lane == 0) atomicAdd(&hist[bin], 32u);
   } else if (in) {
     atomicAdd(&hist[bin], 1u);
   }
@@ -450,6 +450,10 @@ TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev) {
   while (pow2 < c) pow2 <<= 1;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   while (pow2 < kMaxCluster && rows * pow2 * 2 <= dev.sm_count && p.max_seq_len / (pow2 * 2) >= 2048) pow2 <<= 1;
+  // Many more rows than SMs (a prefill chunk): throughput matters, not the latency of one row. One block per
+  // row needs no cluster barriers and keeps more rows in flight; its keys are re-read from global memory in
+  // each of the three sweeps when they do not fit in shared memory.
+  if (rows >= 4 * (int64_t)dev.sm_count) pow2 = 1;
   plan.cluster = pow2;
   const int per = (((p.max_seq_len + plan.cluster - 1) / plan.cluster) + 3) & ~3;
   const size_t want = sizeof(Shared) + (size_t)per * sizeof(uint32_t);
