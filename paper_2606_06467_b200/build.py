@@ -52,7 +52,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
             raise RuntimeError(f"nvcc failed on {src}")
     if force or procs or _stale(LIB, objs):
         tmp = LIB + f".{os.getpid()}.tmp"
-        subprocess.check_call([_nvcc(), "-shared", "-o", tmp] + objs + ["-Xcompiler", "-fPIC"])
+        subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs
+                              + ["-Xcompiler", "-fPIC"])
         os.replace(tmp, LIB)
     return LIB
 

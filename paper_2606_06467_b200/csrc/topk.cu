@@ -33,12 +33,13 @@ namespace cg = cooperative_groups;
 namespace clsa {
 namespace {
 
-// 512 threads and < 113 KiB of shared memory: two blocks fit on an SM, so 16 and more clusters of 8
-// are resident at once (with one block per SM only 15 clusters of 8 fit the GPCs of a B200).
-constexpr int kThreads = 512;
+// 1024 threads per block for latency hiding (the sweeps are chains of votes and shared-memory atomics), clusters
+// of at most 4: a block then fills an SM, and 33 clusters of 4 are resident at once on a B200, whereas only 15
+// clusters of 8 one-per-SM blocks fit its GPCs (16 rows would run in two waves).
+constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxBins = 4096;
-constexpr int kMaxCluster = 8;
+constexpr int kMaxCluster = 4;
 constexpr int kCandCap = 2048;  // candidates (row-wide) the short path handles
 
 struct Shared {
@@ -154,7 +155,7 @@ __device__ __forceinline__ void radix_pass(Shared& sh, cg::cluster_group& cluste
 }
 
 template <bool CACHED>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const int32_t* __restrict__ seq_len,
                   int q_per_seq, int causal, int top_k, int max_seq_len, int32_t* __restrict__ idx_out,
                   int32_t* __restrict__ count_out, uint32_t* status) {
@@ -442,9 +443,9 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
 
 TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev) {
   TopkPlan plan;
-  // One block per 16K visible scores, capped at the portable cluster size and rounded to a power of
-  // two; when there are few rows, spread each over more blocks (down to 2K scores per block).
-  int c = (p.max_seq_len + 16383) / 16384;
+  // One block per 32K visible scores, capped at kMaxCluster and rounded to a power of two; when there are few
+  // rows, spread each over more blocks (down to 2K scores per block).
+  int c = (p.max_seq_len + 32767) / 32768;
   if (c > kMaxCluster) c = kMaxCluster;
   int pow2 = 1;
   while (pow2 < c) pow2 <<= 1;
