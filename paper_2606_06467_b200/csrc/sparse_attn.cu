@@ -387,35 +387,49 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   // Output jobs (KV head of this block's group, query head of the group) dealt over the cluster's warps.
   const int heads_here = min(HC, a.num_kv_heads - (int)blockIdx.y * HC);
   const int njobs = heads_here * G;
+  const uint32_t smem_base = smem_u32(smem);
   for (int job = crank + C * warp; job < njobs; job += C * kAttnWarps) {
     const int jg = job / G, hh = job - jg * G;   // local KV head, query head within the group
-    // partial p = (block p / S, range p % S) was left by warp (p % S) * HC + jg of block p / S
-    auto part_ptr = [&](int p) -> const float* {
-      const int c2 = p / S, sub2 = p - c2 * S;
-      float* local = reinterpret_cast<float*>(smem + (sub2 * HC + jg) * kWarpRingBytes);
-      return (C == 1 ? local : cluster.map_shared_rank(local, c2)) + hh * kPartialStride;
-    };
-    float M = -INFINITY;
-    for (int p = lane; p < nsplit; p += 32) M = fmaxf(M, part_ptr(p)[128]);
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, d));
-    const float mu = M == -INFINITY ? 0.f : M;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float L = 0.f;
+    float L = 0.f, M = -INFINITY;
+    // Partial p = (block p / S, range p % S) was left by warp (p % S) * HC + jg of block p / S. Lane p of each
+    // 32-partial chunk resolves that partial's shared::cluster address once; everyone then reads through it.
     for (int p0 = 0; p0 < nsplit; p0 += 32) {
-      float wl = 0.f;
-      if (p0 + lane < nsplit) {
-        const float2 ml = *reinterpret_cast<const float2*>(part_ptr(p0 + lane) + 128);
-        wl = fast_exp2(ml.x - mu);
-        L += wl * ml.y;
+      const int p = p0 + lane;
+      uint32_t src = 0;
+      float2 ml = make_float2(-INFINITY, 0.f);
+      if (p < nsplit) {
+        const int c2 = p / S, sub2 = p - c2 * S;
+        const uint32_t local = smem_base + (uint32_t)((sub2 * HC + jg) * kWarpRingBytes + hh * kPartialStride * 4);
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(src) : "r"(local), "r"(c2));
+        asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(ml.x), "=f"(ml.y) : "r"(src + 512u) : "memory");
       }
+      // running max over this chunk and what came before; rescale what came before
+      float mc = ml.x;
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xffffffffu, mc, d));
+      const float Mn = fmaxf(M, mc);
+      const float mu = Mn == -INFINITY ? 0.f : Mn;
+      const float rescale = fast_exp2(M - mu);
+      acc.x *= rescale; acc.y *= rescale; acc.z *= rescale; acc.w *= rescale;
+      L *= rescale;
+      M = Mn;
+      const float wl = fast_exp2(ml.x - mu);   // 0 for lanes past the end
+      float lsum = wl * ml.y;
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, d);
+      L += lsum;
       const int chunk_n = min(32, nsplit - p0);
       for (int q0 = 0; q0 < chunk_n; q0 += kMergeBatch) {
         float4 v[kMergeBatch];
 #pragma unroll
-        for (int qq = 0; qq < kMergeBatch; ++qq)
-          v[qq] = q0 + qq < chunk_n ? *reinterpret_cast<const float4*>(part_ptr(p0 + q0 + qq) + lane * 4)
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int qq = 0; qq < kMergeBatch; ++qq) {
+          const uint32_t sq = __shfl_sync(0xffffffffu, src, (q0 + qq) & 31);
+          v[qq] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (q0 + qq < chunk_n)
+            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                         : "=f"(v[qq].x), "=f"(v[qq].y), "=f"(v[qq].z), "=f"(v[qq].w) : "r"(sq + (uint32_t)lane * 16u) : "memory");
+        }
 #pragma unroll
         for (int qq = 0; qq < kMergeBatch; ++qq) {
           const float w = __shfl_sync(0xffffffffu, wl, (q0 + qq) & 31);
@@ -425,8 +439,6 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
         }
       }
     }
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) L += __shfl_xor_sync(0xffffffffu, L, d);
     const float inv = L > 0.f ? 1.f / L : 0.f;
     const int64_t item = r * a.num_q_heads + (int64_t)(blockIdx.y * HC + jg) * G + hh;
     uint2 packed;
