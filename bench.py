@@ -43,6 +43,9 @@ def parse():
     ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads")
     ap.add_argument("--kv-heads", type=int, default=0, help="override the number of KV heads")
     ap.add_argument("--layers", type=int, default=0, help="override the number of cross-decoder layers")
+    ap.add_argument("--compare", action="store_true",
+                    help="also time, on the same inputs, dense attention over the whole cache (Eq. 1) and routing "
+                         "repeated in every layer, and print them as a second JSON line")
     ap.add_argument("--block-size", type=int, default=0, help="page the caches into scattered blocks of this many rows")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-breakdown", action="store_true", help="skip the per-kernel instrumented loop")
@@ -239,6 +242,67 @@ def run_reference(args):
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+def compare_baselines(clsa, torch, w, t, p, ws, idx, cnt, q_layers, outs, flush, stream, sparse_ms):
+    """Two comparison points on the same inputs and kernels (context for the shared-routing design, Sec. 2.3):
+    (a) routing recomputed in every layer (index scores + top-k + attention, L times), as a per-layer token-sparse
+        design would do; (b) dense cross attention over the whole cache (Eq. 1), run as the k = n case of the same
+        attention kernel with an index row that lists every position."""
+    c = w.cfg
+    L, B, n = c.num_layers, c.num_seqs, w.max_seq_len
+    stride = (n + 63) // 64 * 64
+    scores = torch.empty((B, 1, stride), dtype=torch.float32, device=idx.device)
+
+    def timed(fn, reps=5):
+        fn()
+        torch.cuda.synchronize()
+        tot = 0.0
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            tot += e0.elapsed_time(e1)
+        return tot / reps
+
+    def per_layer_routing():
+        for l in range(L):
+            clsa.clsa_index_scores(p, t["q_idx"], scores, stride, ws, stream=stream)
+            clsa.clsa_topk(p, scores, stride, idx, cnt, ws, stream=stream)
+            p.sweep = l & 1
+            clsa.clsa_sparse_attn(p, q_layers[l], idx, cnt, outs[l], None, ws, stream=stream)
+        p.sweep = 0
+
+    unamortised_ms = timed(per_layer_routing)
+    # dense: every position selected
+    pd = clsa.make_params(num_seqs=B, num_q_heads=c.num_q_heads, num_kv_heads=c.num_kv_heads, head_dim=c.head_dim,
+                          idx_dim=c.idx_dim, top_k=n, num_layers=L, max_seq_len=n, sm_scale=c.sm_scale,
+                          seq_start=t["seq_start"], seq_len=t["seq_len"], k_cache=t["k_cache"], v_cache=t["v_cache"],
+                          idx_k_cache=t["idx_k_cache"], block_table=t.get("block_table"), block_size=p.block_size)
+    all_idx = torch.arange(n, dtype=torch.int32, device=idx.device).repeat(B, 1).reshape(B, 1, n)
+    all_idx = torch.where(all_idx < t["seq_len"].reshape(B, 1, 1), all_idx, torch.full_like(all_idx, -1))
+    all_cnt = t["seq_len"].reshape(B, 1).to(torch.int32).contiguous()
+
+    def dense_layers():
+        for l in range(L):
+            pd.sweep = l & 1
+            clsa.clsa_sparse_attn(pd, q_layers[l], all_idx, all_cnt, outs[l], None, ws, stream=stream)
+
+    dense_ms = timed(dense_layers, reps=2)
+    return {
+        "comparison": "same inputs, same kernels, one GPU; context only",
+        "workload": c.name,
+        "clsa_step_us": sparse_ms * 1e3,
+        "routing_in_every_layer_step_us": unamortised_ms * 1e3,
+        "dense_cross_attention_L_layers_us": dense_ms * 1e3,
+        "dense_per_layer_us": dense_ms * 1e3 / L,
+        "dense_GBps": L * int(t["seq_len"].sum().item()) * c.num_kv_heads * c.head_dim * 4 / (dense_ms * 1e-3) / 1e9,
+        "speedup_vs_dense_attention": dense_ms / sparse_ms,
+        "speedup_vs_routing_in_every_layer": unamortised_ms / sparse_ms,
+    }
 
 
 # --------------------------------------------------------------------------------------- CUDA arm
@@ -442,6 +506,10 @@ def run_ours(args):
                         "sample": f"{len(seqs)} of {c.num_seqs} sequences, all {L} layers, {passes} passes "
                                   f"({secs:.1f} s of oracle time; input synthesis not timed)"}
 
+    comparison = None
+    if args.compare and rank == 0 and world == 1 and T == 1:
+        comparison = compare_baselines(clsa, torch, w, t, p, ws, idx, cnt, q_layers, outs, flush, stream, ms_per_step)
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
@@ -461,6 +529,8 @@ def run_ours(args):
             "gpu_launches": K * (2 + L),
         }
         print(json.dumps(line))
+        if comparison is not None:
+            print(json.dumps(comparison))
     if dist is not None:
         dist.destroy_process_group()
 

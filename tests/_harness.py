@@ -1,7 +1,7 @@
 """Shared plumbing of the GPU parity tests: run the CUDA path through the C ABI, run the oracle on the
 same seeded inputs, and compare under the stated tolerances.
 
-Tolerances (from the benchmark spec, with their derivation):
+Tolerances (the acceptance tolerances of this library, with their derivation):
   scores   |gpu - oracle| <= 1e-4 * max(1, |oracle|): bf16 x bf16 products are exact in fp32, so the only
            error is the fp32 accumulation of d_idx <= 128 terms (<= 128 * 2^-24 relative to the sum of
            magnitudes, about 8e-6 * sum|terms|).
