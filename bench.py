@@ -314,17 +314,16 @@ def run_ours(args):
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if rank == 0:
-        entry._load_build_module().build()
     dist = None
+    torch.cuda.set_device(local)
     if world > 1:
         import torch.distributed as dist
 
-        torch.cuda.set_device(local)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist.barrier()
-    else:
-        torch.cuda.set_device(local)
+    if rank == 0:
+        entry._load_build_module().build()
+    if dist is not None:
+        dist.barrier()   # nobody loads the library before rank 0 has (re)built it
     import paper_2606_06467_b200 as clsa
     from workloads import CONFIGS, Workload
 

@@ -25,6 +25,8 @@
 // layers makes layer l+1 start on the rows layer l touched last, which are the ones still in L2.
 #include <cooperative_groups.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace cg = cooperative_groups;
@@ -450,10 +452,15 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   if (C > 1) cluster.sync();  // no block may exit while a neighbour can still read its shared memory
 }
 
-// Blocks of `cluster` that can be resident at once (cached per cluster size; 0 if the query fails).
+// Blocks of `cluster` that can be resident at once on the current device (cached per device and cluster size;
+// 0 if the query fails).
 static int max_resident_blocks(int cluster, size_t smem_bytes) {
-  static int cache[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
-  if (cache[cluster] != 0) return cache[cluster];
+  static std::mutex mu;
+  static int cache[64][9] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 0; }
+  std::lock_guard<std::mutex> lock(mu);
+  if (cache[dev][cluster] != 0) return cache[dev][cluster];
   cudaFuncSetAttribute(sparse_attn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)cluster * 64, 1, 1);
@@ -468,8 +475,8 @@ static int max_resident_blocks(int cluster, size_t smem_bytes) {
   cfg.numAttrs = 1;
   int n = 0;
   if (cudaOccupancyMaxActiveClusters(&n, sparse_attn_kernel<1, false>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-  cache[cluster] = n * cluster;
-  return cache[cluster];
+  cache[dev][cluster] = n * cluster;
+  return cache[dev][cluster];
 }
 
 }  // namespace

@@ -222,3 +222,29 @@ def test_sequence_longer_than_max_seq_len_is_skipped_and_flagged():
     clsa.clsa_topk(g.params, s, g.score_stride, g.idx, g.count, g.ws)
     assert g.status() & clsa.CLSA_DEV_BAD_SEQLEN
     assert (g.count.cpu().numpy() == 0).all() and torch.isnan(s).all()
+
+
+def test_non_finite_scores_never_fault_and_keep_the_index_contract():
+    """Scores must be finite by contract; NaN and infinities are ordered by their bit patterns, and whatever the
+    order, the result keeps the index contract (count, distinct ascending in-range positions) without faulting."""
+    n, k = 50000, 777
+    w = Workload(MID.replace(num_seqs=3, ctx=n, top_k=k, num_layers=1))
+    g = GpuProblem(w, layers=1)
+    rng = np.random.default_rng(12)
+    sc = torch.from_numpy(rng.standard_normal((3, 1, g.score_stride)).astype(np.float32)).to(g.dev)
+    sc[0, 0, ::7] = float("nan")
+    sc[1, 0, ::5] = float("inf")
+    sc[1, 0, 1::5] = float("-inf")
+    sc[2, 0, :n] = float("nan")
+    gi, gc = g.topk(sc)
+    torch.cuda.synchronize()
+    assert g.status() == 0
+    gi, gc = gi.cpu().numpy(), gc.cpu().numpy()
+    for b in range(3):
+        assert gc[b, 0] == k
+        row = gi[b, 0]
+        assert (np.diff(row) > 0).all() and row[0] >= 0 and row[-1] < n
+    assert np.isin(gi[1, 0], np.arange(0, n, 5)).all()       # +inf outranks every finite score
+    # attention on those indices still runs and stays finite (the caches are finite)
+    out, _ = g.sparse_attn(0)
+    assert torch.isfinite(out.float()).all()
