@@ -43,6 +43,9 @@ def parse():
     ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads")
     ap.add_argument("--kv-heads", type=int, default=0, help="override the number of KV heads")
     ap.add_argument("--layers", type=int, default=0, help="override the number of cross-decoder layers")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture the step once into a CUDA graph and time replays (removes host launch gaps; matters "
+                         "for small, launch-bound workloads)")
     ap.add_argument("--compare", action="store_true",
                     help="also time, on the same inputs, dense attention over the whole cache (Eq. 1) and routing "
                          "repeated in every layer, and print them as a second JSON line")
@@ -367,13 +370,13 @@ def run_ours(args):
     def run_step(q_idx_t, q_list, out_list=None):
         out_list = outs if out_list is None else out_list
         if T == 1:
-            clsa.clsa_decode_step(p, q_idx_t, q_list, out_list, idx, cnt, ws, stream=stream)
+            clsa.clsa_decode_step(p, q_idx_t, q_list, out_list, idx, cnt, ws, stream=None)
         else:  # a prefill chunk is not chained by the library: the three calls, in order
-            clsa.clsa_index_scores(p, q_idx_t, chunk_scores, stride, ws, stream=stream)
-            clsa.clsa_topk(p, chunk_scores, stride, idx, cnt, ws, stream=stream)
+            clsa.clsa_index_scores(p, q_idx_t, chunk_scores, stride, ws, stream=None)
+            clsa.clsa_topk(p, chunk_scores, stride, idx, cnt, ws, stream=None)
             for l in range(L):
                 p.sweep = l & 1
-                clsa.clsa_sparse_attn(p, q_list[l], idx, cnt, out_list[l], None, ws, stream=stream)
+                clsa.clsa_sparse_attn(p, q_list[l], idx, cnt, out_list[l], None, ws, stream=None)
             p.sweep = 0
 
     def step():
@@ -389,6 +392,19 @@ def run_ours(args):
         flush.zero_()
         step()
     sync_all()
+    if args.graph:
+        eager_step = step
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):   # the binding launches on torch's current stream: the capture stream here
+            eager_step()
+
+        def step():  # noqa: F811
+            graph.replay()
+
+        for _ in range(3):
+            flush.zero_()
+            step()
+        sync_all()
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
     K = args.steps
@@ -518,7 +534,8 @@ def run_ours(args):
                        "q_heads": c.num_q_heads, "kv_heads": c.num_kv_heads, "idx_dim": c.idx_dim,
                        "algorithmic_bytes_per_step": alg_bytes, "l2": "flushed between steps (512 MiB rewrite, then 256 MiB read so no dirty lines remain)",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "cache_layout": f"paged, {args.block_size}-row blocks" if args.block_size else "contiguous sequences"},
+                       "cache_layout": f"paged, {args.block_size}-row blocks" if args.block_size else "contiguous sequences",
+                       "launch": "CUDA graph replay" if args.graph else "stream launches"},
             "clocks": clocks, "roofline": roofline, "breakdown_us": breakdown, "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms / K,
