@@ -42,16 +42,24 @@ constexpr int kMaxBins = 4096;
 constexpr int kMaxCluster = 4;
 constexpr int kCandCap = 2048;  // candidates (row-wide) the short path handles
 
-struct Shared {
+struct alignas(16) Shared {  // the keys follow it in shared memory and are written 16 bytes at a time
   uint32_t local_hist[kMaxBins];       // this block's slice; later: gathered candidates + 1024-bin histogram
   uint32_t cluster_hist[2][kMaxBins];  // whole row, one copy per block; [1] later: this block's candidate list
   uint32_t warp_tot[kWarps];
   uint32_t warp_gt[kWarps], warp_eq[kWarps];
-  uint32_t block_gt_eq[2];             // read remotely
+  uint32_t block_gt_eq[2];             // read remotely (long path)
   uint32_t cand_count;                 // read remotely
+  uint32_t block_gt0;                  // keys of this block above the threshold's 12-bit bin; read remotely
+  uint32_t rank_gt[kMaxCluster], rank_eq[kMaxCluster];  // per block of the cluster: candidates above / equal to the threshold
   uint32_t digit, k_rem, bin_count;
   uint32_t out_base, eq_base;
 };
+
+// Split cluster barrier: arrive early, wait late, so the barrier's latency hides behind independent work.
+static_assert(sizeof(Shared) % 16 == 0, "the key array behind Shared must stay 16-byte aligned");
+
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t score_key(float x) {
   uint32_t u = __float_as_uint(x);
@@ -198,9 +206,13 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
   const float* src = scores + (int64_t)row * score_stride + lo;
   auto key_at = [&](int i) -> uint32_t { return CACHED ? keys[i] : score_key(src[i]); };
 
-  for (int i = tid; i < kMaxBins; i += kThreads) { sh.local_hist[i] = 0; sh.cluster_hist[0][i] = 0; sh.cluster_hist[1][i] = 0; }
-  if (tid == 0) sh.cand_count = 0;
+  for (int i = tid; i < kMaxBins; i += kThreads) { sh.local_hist[i] = 0; sh.cluster_hist[0][i] = 0; }
+  if (tid < kMaxCluster) { sh.rank_gt[tid] = 0; sh.rank_eq[tid] = 0; }
+  if (tid == 0) { sh.cand_count = 0; sh.block_gt0 = 0; }
   __syncthreads();
+  // Remote adds may land in this block's histogram copy only after it has been cleared: every block arrives
+  // here and waits just before it starts adding, with the whole first sweep in between.
+  cluster_arrive();
 
   // ---- sweep 1: scores -> keys (kept in shared memory) and the 12-bit histogram of this slice --------
   if (CACHED && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
@@ -254,9 +266,8 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
       }
     }
   }
-  // the remote adds below may land in a neighbour's copy as soon as it exists: every block has
-  // cleared its copies before this barrier
-  cluster.sync();
+  __syncthreads();   // this block's histogram is complete
+  cluster_wait();    // every block has cleared its copy of the row histogram
   push_hist<4096>(sh, cluster, nblk, 0);
   cluster.sync();
   scan_from_top<4096>(sh, sh.cluster_hist[0], (uint32_t)kk, true);
@@ -296,14 +307,17 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
     }
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) gt += __shfl_xor_sync(0xffffffffu, gt, d);
-    if (lane == 0) { sh.warp_gt[warp] = gt; sh.warp_eq[warp] = 0; }
-    cluster.sync();  // every block's candidate list and count are complete
+    if (lane == 0) { sh.warp_gt[warp] = gt; sh.warp_eq[warp] = 0; atomicAdd(&sh.block_gt0, gt); }
+    cluster.sync();  // every block's candidate list, candidate count and above-the-bin count are complete
     // gather the row's candidates (keys only) into local_hist[0..in_bin)
     uint32_t* allc = sh.local_hist;
     uint32_t* hist10 = sh.local_hist + kCandCap;  // 1024 bins
+    uint32_t start[kMaxCluster];  // first flat index of each block's candidates (all lanes hold all of them)
+    uint32_t gt0_of_lane = 0;     // lane r: keys of block r above the bin
     {
-      // lane r of every warp reads block r's count; an exclusive scan gives the blocks' offsets
+      // lane r of every warp reads block r's counts; an exclusive scan gives the blocks' offsets
       const uint32_t nr = lane < nblk ? *cluster.map_shared_rank(&sh.cand_count, lane) : 0u;
+      gt0_of_lane = lane < nblk ? *cluster.map_shared_rank(&sh.block_gt0, lane) : 0u;
       uint32_t incl = nr;
 #pragma unroll
       for (int d = 1; d < kMaxCluster; d <<= 1) {
@@ -311,7 +325,6 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
         if (lane >= d) incl += up;
       }
       const uint32_t excl = incl - nr;
-      uint32_t start[kMaxCluster];  // first flat index of each block's list (all lanes hold all eight)
 #pragma unroll
       for (int q = 0; q < kMaxCluster; ++q) start[q] = q < nblk ? __shfl_sync(0xffffffffu, excl, q) : 0xffffffffu;
       for (uint32_t i = tid; i < in_bin; i += kThreads) {
@@ -326,6 +339,9 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
     }
     for (int i = tid; i < 1024; i += kThreads) hist10[i] = 0;
     __syncthreads();
+    // This block reads nobody's shared memory from here on: arrive now on the barrier that keeps every block
+    // alive until its neighbours are done with it, and wait on it only at the very end.
+    cluster_arrive();
     // two local 10-bit passes over the candidates: bits 19..10, then 9..0
     uint32_t prefix = digit0 << 20, prefix_mask = 0xfff00000u;
 #pragma unroll 1
@@ -352,10 +368,37 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
       if (c.x > thr) atomicAdd(&sh.warp_gt[w], 1u);
       else if (c.x == thr) atomicAdd(&sh.warp_eq[w], 1u);
     }
+    // the same two counts for every block of the cluster, from the gathered candidates (grouped by block):
+    // with them each block derives its output offset alone, without another exchange
+    for (uint32_t i = tid; i < in_bin; i += kThreads) {
+      int r = 0;
+#pragma unroll
+      for (int q = 1; q < kMaxCluster; ++q)
+        if (i >= start[q]) r = q;
+      const uint32_t key = allc[i];
+      if (key > thr) atomicAdd(&sh.rank_gt[r], 1u);
+      else if (key == thr) atomicAdd(&sh.rank_eq[r], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane r holds the totals of block r; the offset of this block is a prefix over the lower-ranked ones
+      const uint32_t g = lane < nblk ? gt0_of_lane + sh.rank_gt[lane] : 0u;
+      const uint32_t e = lane < nblk ? sh.rank_eq[lane] : 0u;
+      uint32_t eq_before = 0, sel_before = 0;
+      for (int r = 0; r < rank; ++r) {
+        const uint32_t gr = __shfl_sync(0xffffffffu, g, r), er = __shfl_sync(0xffffffffu, e, r);
+        const uint32_t take = eq_before >= need_eq ? 0u : min(er, need_eq - eq_before);
+        sel_before += gr + take;
+        eq_before += er;
+      }
+      if (lane == 0) { sh.out_base = sel_before; sh.eq_base = eq_before; }
+    }
     __syncthreads();
   } else {
     // ---- long path: two more cluster-wide radix passes, then a counting sweep ------------------------
     uint32_t prefix = digit0 << 20, prefix_mask = 0xfff00000u;
+    for (int i = tid; i < kMaxBins; i += kThreads) sh.cluster_hist[1][i] = 0;
+    cluster.sync();  // every block's second histogram copy is clear before anybody adds into it
     radix_pass<12>(sh, cluster, nblk, cnt, 8, 1, prefix, prefix_mask, k_rem, key_at);
     radix_pass<8>(sh, cluster, nblk, cnt, 0, 0, prefix, prefix_mask, k_rem, key_at);
     thr = prefix;
@@ -373,32 +416,33 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
     }
     if (lane == 0) { sh.warp_gt[warp] = gt; sh.warp_eq[warp] = eq; }
     __syncthreads();
+    if (warp == 0) {
+      uint32_t g = lane < kWarps ? sh.warp_gt[lane] : 0u, e = lane < kWarps ? sh.warp_eq[lane] : 0u;
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) {
+        g += __shfl_xor_sync(0xffffffffu, g, d);
+        e += __shfl_xor_sync(0xffffffffu, e, d);
+      }
+      if (lane == 0) { sh.block_gt_eq[0] = g; sh.block_gt_eq[1] = e; }
+    }
+    cluster.sync();
+    if (tid == 0) {
+      uint32_t eq_before = 0, sel_before = 0;
+      for (int r = 0; r < rank; ++r) {
+        const uint32_t* ge = cluster.map_shared_rank(sh.block_gt_eq, r);
+        const uint32_t g = ge[0], e = ge[1];
+        const uint32_t take = eq_before >= need_eq ? 0u : min(e, need_eq - eq_before);
+        sel_before += g + take;
+        eq_before += e;
+      }
+      sh.out_base = sel_before;
+      sh.eq_base = eq_before;
+    }
+    __syncthreads();
+    cluster_arrive();  // pairs with the wait at the very end
   }
 
   // ---- index-ordered compaction ----------------------------------------------------------------------
-  if (warp == 0) {
-    uint32_t g = lane < kWarps ? sh.warp_gt[lane] : 0u, e = lane < kWarps ? sh.warp_eq[lane] : 0u;
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) {
-      g += __shfl_xor_sync(0xffffffffu, g, d);
-      e += __shfl_xor_sync(0xffffffffu, e, d);
-    }
-    if (lane == 0) { sh.block_gt_eq[0] = g; sh.block_gt_eq[1] = e; }
-  }
-  cluster.sync();
-  if (tid == 0) {
-    uint32_t eq_before = 0, sel_before = 0;
-    for (int r = 0; r < rank; ++r) {
-      const uint32_t* ge = cluster.map_shared_rank(sh.block_gt_eq, r);
-      const uint32_t g = ge[0], e = ge[1];
-      const uint32_t take = eq_before >= need_eq ? 0u : min(e, need_eq - eq_before);
-      sel_before += g + take;
-      eq_before += e;
-    }
-    sh.out_base = sel_before;
-    sh.eq_base = eq_before;
-  }
-  __syncthreads();
   // offsets of this warp: selected / threshold-equal keys in lower warps of this block
   uint32_t out_pos = sh.out_base, eq_rank = sh.eq_base;
   for (int w = 0; w < warp; ++w) {
@@ -436,7 +480,7 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
       eq_rank += __popc(eq_ballot[u]);
     }
   }
-  cluster.sync();  // no block may exit while a neighbour can still read its shared memory
+  cluster_wait();  // no block may exit while a neighbour can still read its shared memory (arrived earlier)
 }
 
 }  // namespace
