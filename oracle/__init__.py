@@ -48,6 +48,8 @@ def lib():
         _lib = ctypes.CDLL(build())
         _lib.oracle_visible.restype = ctypes.c_int64
         _lib.oracle_num_threads.restype = ctypes.c_int32
+        _lib.oracle_bf16_from_double.restype = ctypes.c_uint16
+        _lib.oracle_bf16_from_double.argtypes = [ctypes.c_double]
     return _lib
 
 
@@ -62,6 +64,24 @@ def _ptr(a):
 def _c(a, dtype):
     a = np.ascontiguousarray(a, dtype=dtype)
     return a
+
+
+def linear(h, w) -> np.ndarray:
+    """Eq. 2 as a plain product: float64 [rows, n_out] = h [rows, d_model] . w[n_out, d_model]^T from bf16 bits."""
+    h, w = _c(h, np.uint16), _c(w, np.uint16)
+    assert h.ndim == 2 and w.ndim == 2 and h.shape[1] == w.shape[1]
+    y = np.empty((h.shape[0], w.shape[0]), dtype=np.float64)
+    lib().oracle_linear(_ptr(h), _ptr(w), ctypes.c_int64(h.shape[0]), ctypes.c_int64(w.shape[0]),
+                        ctypes.c_int64(h.shape[1]), _ptr(y))
+    return y
+
+
+def round_bf16(x) -> np.ndarray:
+    """Nearest-even bf16 bit patterns (uint16) of float64 values, rounded once."""
+    x = _c(x, np.float64)
+    out = np.empty(x.shape, dtype=np.uint16)
+    lib().oracle_round_bf16(_ptr(x), ctypes.c_int64(x.size), _ptr(out))
+    return out
 
 
 class Problem:
@@ -149,6 +169,26 @@ class Problem:
         lse = np.empty((self.B, self.T, self.Hq), dtype=np.float64)
         lib().oracle_dense_attn(ctypes.byref(self._s), _ptr(q), _ptr(out), _ptr(lse))
         return out, lse
+
+    # Eq. 2 + cache append ----------------------------------------------------------------
+    def project_append(self, h, w_q_idx, w_k_idx, w_k=None, w_v=None) -> np.ndarray:
+        """Projects the T newest tokens of every sequence (h: uint16 [B,T,d_model]; weights uint16 [n_out, d_model])
+        and writes their K_idx (and, with w_k/w_v, K and V) rows into this problem's caches IN PLACE.
+        Returns q_idx as uint16 [B,T,d_idx]."""
+        h = _c(h, np.uint16)
+        d_model = h.shape[-1]
+        h = h.reshape(self.B, self.T, d_model)
+        w_q_idx, w_k_idx = _c(w_q_idx, np.uint16), _c(w_k_idx, np.uint16)
+        assert w_q_idx.shape == (self.d_idx, d_model) and w_k_idx.shape == (self.d_idx, d_model)
+        assert self.idx_k_cache is not None and self.idx_k_cache.flags.writeable
+        if w_k is not None:
+            w_k, w_v = _c(w_k, np.uint16), _c(w_v, np.uint16)
+            assert w_k.shape == (self.Hkv * self.D, d_model) and w_v.shape == w_k.shape
+            assert self.k_cache is not None and self.k_cache.flags.writeable and self.v_cache.flags.writeable
+        q_idx = np.empty((self.B, self.T, self.d_idx), dtype=np.uint16)
+        lib().oracle_project_append(ctypes.byref(self._s), ctypes.c_int32(d_model), _ptr(h), _ptr(w_q_idx),
+                                    _ptr(w_k_idx), _ptr(w_k), _ptr(w_v), _ptr(q_idx))
+        return q_idx
 
     # whole step --------------------------------------------------------------------------
     def decode_step(self, q_idx, q_layers):

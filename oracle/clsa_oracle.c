@@ -10,6 +10,8 @@
  *   dense attn     O^(l) = Attn(Q^(l), K, V)    (Eq. 1) -- an independent routine used only to
  *                                               check the k >= n limit of Eq. 4
  *   decode step    one S_t, reused by every cross-decoder layer   (Sec. 2.1, closing paragraph)
+ *   projections    Q_idx = H W^Q_idx, K_idx = H W^K_idx  (Eq. 2) for the newest tokens, and the
+ *                  append of their K_idx / K / V rows to the shared caches (the step before Eq. 3)
  *
  * These results are plain definitions (a matrix product, an exact selection, a softmax-weighted
  * mean over a subset), so each function is that definition written out with no blocking, fusion
@@ -22,7 +24,10 @@
  *   - fewer than k visible tokens: all of them are selected (k is stated as a maximum);
  *   - decode: every cached token is visible; causal chunk: query t of T sees s <= n - T + t;
  *   - Attn is scaled dot-product attention with an explicit sm_scale, no positional rotation
- *     (NoPE in global attention), GQA with contiguous groups: KV head = query head / group size.
+ *     (NoPE in global attention), GQA with contiguous groups: KV head = query head / group size;
+ *   - the shared K and V rows are linear maps of the same hidden state, K = H W^K, V = H W^V
+ *     (the paper only says the cache corresponds to H); no normalisation is applied here;
+ *   - projected values are stored as bf16, rounded to nearest-even once from the exact sum.
  *
  * Only tests, the smoke check and the bench's CPU-baseline leg may call this file.
  */
@@ -269,6 +274,71 @@ void oracle_decode_step(const oracle_problem* p, int32_t num_layers, const uint1
   for (int32_t l = 0; l < num_layers; ++l)
     oracle_sparse_attn(p, q_layers + l * per_layer * p->head_dim, idx, count, out + l * per_layer * p->head_dim,
                        lse ? lse + l * per_layer : NULL);
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Eq. 2 and the cache append. Weights are stored one output feature per row: w is bf16
+ * [n_out][d_model], so y[m][o] = sum_j h[m][j] * w[o][j]  (y = h W with W = w^T). */
+void oracle_linear(const uint16_t* h, const uint16_t* w, int64_t rows, int64_t n_out, int64_t d_model, double* y) {
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < rows; ++m)
+    for (int64_t o = 0; o < n_out; ++o) {
+      double acc = 0.0;
+      for (int64_t j = 0; j < d_model; ++j) acc += bf16_to_double(h[m * d_model + j]) * bf16_to_double(w[o * d_model + j]);
+      y[m * n_out + o] = acc;
+    }
+}
+
+/* Nearest bf16 (8 significant bits, exponent range of binary32), ties to the even significand, rounded
+ * ONCE from the double (going through binary32 first would round twice). */
+uint16_t oracle_bf16_from_double(double x) {
+  if (isnan(x)) return 0x7FC0;
+  const uint16_t sign = signbit(x) ? 0x8000 : 0;
+  double a = fabs(x), r;
+  if (a == 0.0) return sign;
+  if (isinf(a)) return sign | 0x7F80;
+  int e;
+  (void)frexp(a, &e);                         /* a = m * 2^e, m in [0.5, 1) */
+  if (e - 1 < -126) r = ldexp(nearbyint(ldexp(a, 133)), -133);   /* subnormal grid: multiples of 2^-133 */
+  else r = ldexp(nearbyint(ldexp(a, 8 - e)), e - 8);             /* 8 significant bits; nearbyint = ties-to-even */
+  if (r >= ldexp(1.0, 128)) return sign | 0x7F80;
+  const float f = (float)r;                   /* exact: r is a bf16 number */
+  uint32_t u;
+  memcpy(&u, &f, sizeof u);
+  return sign | (uint16_t)(u >> 16);
+}
+
+void oracle_round_bf16(const double* x, int64_t n, uint16_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = oracle_bf16_from_double(x[i]);
+}
+
+/* For query token t of sequence b (position s = n_b - T + t, the sequence's newest tokens), with
+ * h bf16 [B][T][d_model]:
+ *   q_idx_out[b][t][:]            = bf16(h W^Q_idx)                        (Eq. 2)
+ *   K_idx cache row of (b, s)     = bf16(h W^K_idx)                        (Eq. 2)
+ *   K / V cache rows of (b, s)    = bf16(h W^K), bf16(h W^V), laid out [Hkv][D]   (skipped when w_k is NULL)
+ * The caches of `p` are written in place; no other row is touched. */
+void oracle_project_append(const oracle_problem* p, int32_t d_model, const uint16_t* h, const uint16_t* w_q_idx,
+                           const uint16_t* w_k_idx, const uint16_t* w_k, const uint16_t* w_v, uint16_t* q_idx_out) {
+  const int B = p->num_seqs, T = p->q_per_seq, d = p->idx_dim, Hkv = p->num_kv_heads, D = p->head_dim;
+  double* y = (double*)malloc(sizeof(double) * (size_t)(Hkv * D > d ? Hkv * D : d));
+  for (int b = 0; b < B; ++b)
+    for (int t = 0; t < T; ++t) {
+      const uint16_t* hv = h + ((int64_t)b * T + t) * d_model;
+      const int64_t row = cache_row(p, b, (int64_t)p->seq_len[b] - T + t);
+      oracle_linear(hv, w_q_idx, 1, d, d_model, y);
+      oracle_round_bf16(y, d, q_idx_out + ((int64_t)b * T + t) * d);
+      oracle_linear(hv, w_k_idx, 1, d, d_model, y);
+      oracle_round_bf16(y, d, (uint16_t*)p->idx_k_cache + row * p->idx_token_stride);
+      if (w_k == NULL) continue;
+      oracle_linear(hv, w_k, 1, (int64_t)Hkv * D, d_model, y);
+      for (int g = 0; g < Hkv; ++g)
+        oracle_round_bf16(y + (int64_t)g * D, D, (uint16_t*)p->k_cache + row * p->kv_token_stride + g * p->kv_head_stride);
+      oracle_linear(hv, w_v, 1, (int64_t)Hkv * D, d_model, y);
+      for (int g = 0; g < Hkv; ++g)
+        oracle_round_bf16(y + (int64_t)g * D, D, (uint16_t*)p->v_cache + row * p->kv_token_stride + g * p->kv_head_stride);
+    }
+  free(y);
 }
 
 int32_t oracle_num_threads(void) {

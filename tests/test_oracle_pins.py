@@ -10,6 +10,11 @@ transposed operand, a wrong head mapping -- fails at least one of these):
             (Eq. 1 vs Eq. 4), closed forms (uniform logits, constant V, single token, dominant
             logit), invariances (permutation, logit shift, GQA grouping), the hand example.
   chain   : one index reused by all layers; decode_step == the separate calls.
+  projections + append (Eq. 2): the rounding against every bf16 value, constructed ties, a double-rounding
+            trap and torch's float32 -> bf16 conversion (library); the product against numpy float64 matmul
+            with asymmetric shapes; selector weights (a projected row must reproduce chosen components
+            of h exactly, which fixes operand order and the [Hkv][D] layout); untouched rows stay
+            byte-identical; contiguous and paged placement; the newest token's score in closed form.
 """
 import json
 import math
@@ -425,3 +430,121 @@ def test_paged_layout_gives_the_same_results_as_contiguous_sequences():
         for b in range(4):
             n = int(w.seq_len[b])
             np.testing.assert_array_equal(got["scores"][b, 0, :n], flat["scores"][b, 0, :n])
+
+
+# ======================================================================================= Eq. 2 + append
+def test_bf16_rounding_every_value_ties_and_library():
+    import torch
+
+    bits = np.arange(65536, dtype=np.uint16)
+    finite = (bits & 0x7F80) != 0x7F80
+    vals = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).double().numpy()  # torch decodes the bits
+    got = oracle.round_bf16(vals[finite])
+    np.testing.assert_array_equal(got, bits[finite])  # every finite bf16 number (subnormals, both zeros) is a fixed point
+    one = 1.0
+    cases = [(one + 2.0 ** -8, 0x3F80),               # tie between 1 and 1 + 2^-7: the even significand wins
+             (one + 3 * 2.0 ** -8, 0x3F82),           # tie between odd 1 + 2^-7 and even 1 + 2^-6
+             (one + 2.0 ** -8 + 2.0 ** -40, 0x3F81),  # just above a tie: float32 would lose the 2^-40 and round to even
+             (one + 2.0 ** -8 - 2.0 ** -40, 0x3F80),
+             (-(one + 2.0 ** -8 + 2.0 ** -40), 0xBF81),
+             (2.0 ** -134, 0x0000), (2.0 ** -134 * 1.0001, 0x0001), (3 * 2.0 ** -134, 0x0002),  # subnormal grid 2^-133
+             (2.0 ** 128, 0x7F80), ((2 - 2.0 ** -8) * 2.0 ** 127, 0x7F80), ((2 - 2.0 ** -7) * 2.0 ** 127, 0x7F7F)]
+    for x, want in cases:
+        assert int(oracle.round_bf16(np.array([x]))[0]) == want, (x, hex(want))
+    rng = np.random.default_rng(50)
+    f32 = (rng.standard_normal(200000) * np.exp(rng.uniform(-30, 30, 200000))).astype(np.float32)
+    lib_bits = torch.from_numpy(f32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(oracle.round_bf16(f32.astype(np.float64)), lib_bits)  # one rounding on both sides
+    x = np.sort(rng.standard_normal(5000))
+    r = f64(oracle.round_bf16(x))
+    assert (np.diff(r) >= 0).all() and (np.abs(r - x) <= np.abs(x) * 2.0 ** -8).all()  # monotone, half an ulp at most
+
+
+def test_linear_matches_numpy_matmul():
+    rng = np.random.default_rng(51)
+    h, w = rand_bits(rng, (5, 11)), rand_bits(rng, (3, 11), 0.3)
+    y = oracle.linear(h, w)
+    assert y.shape == (5, 3)
+    np.testing.assert_allclose(y, f64(h) @ f64(w).T, rtol=0, atol=1e-12)
+    e = np.zeros((1, 11)); e[0, 4] = 1.0
+    np.testing.assert_array_equal(oracle.linear(bf16(e), w)[0], f64(w)[:, 4])  # a unit state reads column 4 of every row
+    np.testing.assert_array_equal(oracle.linear(h, bf16(e))[:, 0], f64(h)[:, 4])
+
+
+def _selector(n_out, d_model, cols):
+    w = np.zeros((n_out, d_model))
+    w[np.arange(n_out), cols] = 1.0
+    return bf16(w)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_project_append_places_exact_rows_and_touches_nothing_else(paged):
+    rng = np.random.default_rng(52)
+    B, T, Hkv, D, d_idx, dm = 3, 2, 2, 8, 6, 40
+    lens = (9, 13, 4)
+    p = make_problem(rng, B=B, T=T, Hq=4, Hkv=Hkv, D=D, d_idx=d_idx, lens=lens, causal=1)
+    if paged:
+        bs = 4
+        nblk = [(n + bs - 1) // bs for n in lens]
+        perm = rng.permutation(sum(nblk) + 2)
+        table = np.zeros((B, max(nblk)), dtype=np.int32)
+        at = 0
+        for b in range(B):
+            table[b, : nblk[b]] = perm[at: at + nblk[b]]
+            at += nblk[b]
+        rows = (sum(nblk) + 2) * bs
+        p = oracle.Problem(num_seqs=B, q_per_seq=T, num_q_heads=4, num_kv_heads=Hkv, head_dim=D, idx_dim=d_idx, top_k=5,
+                           causal=1, sm_scale=1.0, seq_start=np.zeros(B, np.int64), seq_len=np.asarray(lens, np.int32),
+                           k_cache=rand_bits(rng, (rows, Hkv, D)), v_cache=rand_bits(rng, (rows, Hkv, D)),
+                           idx_k_cache=rand_bits(rng, (rows, d_idx)), block_table=table, block_size=bs)
+        row_of = lambda b, s: int(table[b, s // bs]) * bs + s % bs
+    else:
+        row_of = lambda b, s: int(p.seq_start[b]) + s
+    before = (p.idx_k_cache.copy(), p.k_cache.copy(), p.v_cache.copy())
+    h = rand_bits(rng, (B, T, dm))
+    cq, ck = rng.permutation(dm)[:d_idx], rng.permutation(dm)[:d_idx]
+    ckk, cv = rng.permutation(dm)[: Hkv * D], rng.permutation(dm)[: Hkv * D]
+    q = p.project_append(h, _selector(d_idx, dm, cq), _selector(d_idx, dm, ck), _selector(Hkv * D, dm, ckk),
+                         _selector(Hkv * D, dm, cv))
+    touched = set()
+    for b in range(B):
+        for t in range(T):
+            r = row_of(b, lens[b] - T + t)
+            touched.add(r)
+            np.testing.assert_array_equal(q[b, t], h[b, t, cq])              # bf16 in, selector weights: exact
+            np.testing.assert_array_equal(p.idx_k_cache[r], h[b, t, ck])
+            np.testing.assert_array_equal(p.k_cache[r].reshape(-1), h[b, t, ckk])  # feature g*D + d lands at [g][d]
+            np.testing.assert_array_equal(p.v_cache[r].reshape(-1), h[b, t, cv])
+    keep = np.array(sorted(set(range(p.idx_k_cache.shape[0])) - touched))
+    assert len(touched) == B * T
+    for now, was in zip((p.idx_k_cache, p.k_cache, p.v_cache), before):
+        np.testing.assert_array_equal(now[keep], was[keep])
+
+
+def test_project_append_general_weights_and_indexer_only():
+    rng = np.random.default_rng(53)
+    B, T, Hkv, D, d_idx, dm = 2, 1, 2, 8, 6, 33
+    p = make_problem(rng, B=B, T=T, Hkv=Hkv, D=D, d_idx=d_idx, lens=(9, 13))
+    h = rand_bits(rng, (B, T, dm))
+    wq, wk = rand_bits(rng, (d_idx, dm), 0.2), rand_bits(rng, (d_idx, dm), 0.2)
+    wkk, wv = rand_bits(rng, (Hkv * D, dm), 0.2), rand_bits(rng, (Hkv * D, dm), 0.2)
+    k_before = p.k_cache.copy()
+    q = p.project_append(h, wq, wk)                    # indexer branch only: K and V stay as they were
+    np.testing.assert_array_equal(p.k_cache, k_before)
+    hf = f64(h).reshape(B, dm)
+    np.testing.assert_array_equal(q.reshape(B, d_idx), oracle.round_bf16(hf @ f64(wq).T))
+    q2 = p.project_append(h, wq, wk, wkk, wv)
+    np.testing.assert_array_equal(q2, q)
+    for b in range(B):
+        r = int(p.seq_start[b]) + int(p.seq_len[b]) - 1
+        np.testing.assert_array_equal(p.idx_k_cache[r], oracle.round_bf16(hf[b] @ f64(wk).T))
+        np.testing.assert_array_equal(p.k_cache[r].reshape(-1), oracle.round_bf16(hf[b] @ f64(wkk).T))
+        np.testing.assert_array_equal(p.v_cache[r].reshape(-1), oracle.round_bf16(hf[b] @ f64(wv).T))
+    # the appended key is what Eq. 3 then scores: with both indexer weights selecting the same components of h,
+    # the newest token's score is the sum of their squares
+    cols = np.arange(d_idx) * 3
+    sel = _selector(d_idx, dm, cols)
+    q3 = p.project_append(h, sel, sel)
+    sc = p.index_scores(q3)
+    for b in range(B):
+        np.testing.assert_allclose(sc[b, 0, int(p.seq_len[b]) - 1], (hf[b, cols] ** 2).sum(), rtol=0, atol=1e-12)

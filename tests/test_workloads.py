@@ -89,3 +89,17 @@ def test_to_device_matches_host_on_cpu():
     h = Workload(HEADLINE.replace(num_seqs=2, ctx=4096))
     dh = h.to_device("cpu", layers=1)
     np.testing.assert_array_equal(bits(dh["idx_k_cache"])[4096:], h.kidx_bits(1))
+
+
+def test_projection_inputs_host_equal_device_and_are_scaled_exactly():
+    import torch
+
+    w = Workload(TINY.replace(d_model=96))
+    d = w.projection_to_device("cpu")
+    bits = lambda t: t.view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(bits(d["h"]), w.hidden_bits())
+    for which in ("q_idx", "k_idx", "k", "v"):
+        host = w.weight_bits(which)
+        assert host.shape == w.weight_shape(which)
+        np.testing.assert_array_equal(bits(d["w_" + which]), host)
+    assert abs(g.bf16_bits_to_f64(w.weight_bits("k")).std() * 64 - 1.0) < 0.05

@@ -17,6 +17,8 @@ from . import generator as g
 TID_Q_IDX, TID_K_IDX, TID_K, TID_V = 0, 1, 2, 3
 TID_LEN, TID_DUP_FLAG, TID_DUP_SRC, TID_PLANT = 4, 5, 6, 7
 TID_BLOCK_PERM = 8
+TID_H, TID_W_QIDX, TID_W_KIDX, TID_W_K, TID_W_V = 9, 10, 11, 12, 13
+WEIGHT_SHIFT = 6  # projection weights are table values times 2^-6 (about 1/sqrt(d_model)): exact in bf16
 TID_Q_LAYER0 = 16
 
 
@@ -39,6 +41,7 @@ class Config:
     planted: int = 0         # planted high-score tokens per sequence (decode only)
     plant_boost: float = 4.0
     dup_frac: float = 0.0    # fraction of indexer-key rows that are exact copies of an earlier row
+    d_model: int = 2560      # hidden size of the states the projections read (the paper's 4B-scale model)
 
     def replace(self, **kw) -> "Config":
         return dataclasses.replace(self, **kw)
@@ -195,6 +198,40 @@ class Workload:
         n = c.num_seqs * c.q_per_seq * c.num_q_heads * c.head_dim
         return g.Stream(c.seed, TID_Q_LAYER0 + layer).host_range(0, n).reshape(
             c.num_seqs, c.q_per_seq, c.num_q_heads, c.head_dim)
+
+    # ------------------------------------------------------------------ projection inputs (Eq. 2)
+    def weight_shape(self, which: str):
+        c = self.cfg
+        return (c.idx_dim if which in ("q_idx", "k_idx") else c.num_kv_heads * c.head_dim, c.d_model)
+
+    def hidden_bits(self) -> np.ndarray:
+        """[B, T, d_model] hidden states of the query tokens, N(0,1)."""
+        c = self.cfg
+        return g.Stream(c.seed, TID_H).host_range(0, c.num_seqs * c.q_per_seq * c.d_model).reshape(
+            c.num_seqs, c.q_per_seq, c.d_model)
+
+    def weight_bits(self, which: str) -> np.ndarray:
+        """[n_out, d_model] projection weights (one output feature per row), N(0,1) * 2^-WEIGHT_SHIFT."""
+        tid = {"q_idx": TID_W_QIDX, "k_idx": TID_W_KIDX, "k": TID_W_K, "v": TID_W_V}[which]
+        n_out, d = self.weight_shape(which)
+        raw = g.Stream(self.cfg.seed, tid).host_range(0, n_out * d).reshape(n_out, d)
+        return g.f64_to_bf16_bits(g.bf16_bits_to_f64(raw) * 2.0 ** -WEIGHT_SHIFT)
+
+    def projection_to_device(self, device="cuda"):
+        """dict(h, w_q_idx, w_k_idx, w_k, w_v) as bf16 torch tensors, bit-identical to the host versions."""
+        import torch
+
+        c = self.cfg
+        dev = torch.device(device)
+        out = {}
+        h = torch.empty((c.num_seqs, c.q_per_seq, c.d_model), dtype=torch.bfloat16, device=dev)
+        g.Stream(c.seed, TID_H).device_fill(h)
+        out["h"] = h
+        for which, tid in (("q_idx", TID_W_QIDX), ("k_idx", TID_W_KIDX), ("k", TID_W_K), ("v", TID_W_V)):
+            t = torch.empty(self.weight_shape(which), dtype=torch.bfloat16, device=dev)
+            g.Stream(c.seed, tid).device_fill(t)
+            out["w_" + which] = t.mul_(2.0 ** -WEIGHT_SHIFT)  # a power of two: exact
+        return out
 
     def host_kidx_cache(self) -> np.ndarray:
         """Full [total_rows, idx_dim] indexer-key cache on the host."""
