@@ -147,6 +147,26 @@ CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, c
                              void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
                              size_t workspace_bytes, clsa_stream stream);
 
+/* The step immediately before the path (Eq. 2 and the append of the new tokens' cache rows): for query token t
+ * of sequence b, at position s = seq_len[b] - T + t (the sequence's newest tokens, whose rows this call fills),
+ *   q_idx_out[b][t][:]        = h[b][t][:] W^Q_idx                     (Eq. 2)
+ *   K_idx cache row of (b,s)  = h[b][t][:] W^K_idx                     (Eq. 2)
+ *   K and V cache rows of (b,s), laid out [Hkv][D] = h W^K, h W^V      (the shared cache built from the same states)
+ * bf16 operands, fp32 accumulation, one round-to-nearest-even to bf16. No normalisation, bias or rotation.
+ *   d_model  hidden size, a multiple of 32 (otherwise CLSA_ERR_UNSUPPORTED)
+ *   h        bf16 [B][T][d_model], 16-byte aligned
+ *   w_q_idx, w_k_idx  bf16 [d_idx][d_model]: one OUTPUT feature per row (y[o] = sum_j h[j] * w[o][j]), 16-byte aligned
+ *   w_k, w_v bf16 [Hkv*D][d_model], feature g*D + d is element d of KV head g; both NULL = indexer branch only
+ *   q_idx_out bf16 [B][T][d_idx], 16-byte aligned
+ * THIS CALL WRITES the caches named by p (idx_k_cache, and k_cache/v_cache when w_k is given) although clsa_params
+ * declares them const: exactly the rows above, nothing else. seq_len must already count the new tokens. Calls that
+ * follow on the same stream (clsa_index_scores, clsa_decode_step) see the appended rows. A sequence with
+ * seq_len < T or > max_seq_len is skipped and flags CLSA_DEV_BAD_SEQLEN. Built for decoding (B*T up to a few
+ * dozen rows, where the op is a stream of the weights); larger B*T works but re-reads the weights per 64 rows. */
+CLSA_API clsa_status clsa_project_append(const clsa_params* p, int32_t d_model, const void* h, const void* w_q_idx,
+                                         const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,
+                                         void* workspace, size_t workspace_bytes, clsa_stream stream);
+
 /* The same step as clsa_decode_step for callers that cannot allocate device memory. (The paper has
  * no counterpart: this is a convenience of the library.) Some callers have no way to obtain a
  * workspace: code that runs inside a region where cudaMalloc is forbidden or would synchronise the

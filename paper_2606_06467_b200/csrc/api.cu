@@ -200,7 +200,6 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
   if (err != cudaSuccess) return CLSA_ERR_CUDA;
   for (int l = 0; l < p->num_layers; ++l) {
     // alternate the sweep direction so that a layer starts on the rows its predecessor touched last
-    // alternate the sweep direction so that a layer starts on the rows its predecessor touched last
     // Layer 0 follows the top-k kernel and must wait for its index; every later layer reads only what
     // was complete before its predecessor started (the index, the caches, the caller's queries), so it
     // may overlap its predecessor's tail.
@@ -209,6 +208,27 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
     if (err != cudaSuccess) return CLSA_ERR_CUDA;
   }
   return CLSA_OK;
+}
+
+clsa_status clsa_project_append(const clsa_params* p, int32_t d_model, const void* h, const void* w_q_idx,
+                                const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,
+                                void* workspace, size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  CLSA_TRY(check_idx_cache(p));
+  if (h == nullptr || w_q_idx == nullptr || w_k_idx == nullptr || q_idx_out == nullptr) return CLSA_ERR_INVALID_ARG;
+  if ((w_k == nullptr) != (w_v == nullptr)) return CLSA_ERR_INVALID_ARG;
+  if (!aligned(h, 16) || !aligned(w_q_idx, 16) || !aligned(w_k_idx, 16) || !aligned(w_k, 16) || !aligned(w_v, 16) ||
+      !aligned(q_idx_out, 16))
+    return CLSA_ERR_INVALID_ARG;
+  if (d_model < 32) return CLSA_ERR_INVALID_ARG;
+  if (d_model % 32 != 0) return CLSA_ERR_UNSUPPORTED;
+  if (w_k != nullptr) CLSA_TRY(check_kv_cache(p));
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  return from_cuda(launch_project_append(*p, d_model, h, w_q_idx, w_k_idx, w_k, w_v, q_idx_out,
+                                         static_cast<uint32_t*>(workspace), dev, static_cast<cudaStream_t>(stream)));
 }
 
 // ---- entry point that allocates nothing -----------------------------------------------------------

@@ -60,6 +60,10 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
                                float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
                                const DeviceInfo& dev, cudaStream_t stream);
 
+cudaError_t launch_project_append(const clsa_params& p, int d_model, const void* h, const void* w_q_idx,
+                                  const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,
+                                  uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+
 // ---------------------------------------------------------------------------------------------
 // Device helpers
 // ---------------------------------------------------------------------------------------------
