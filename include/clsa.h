@@ -113,8 +113,8 @@ CLSA_API clsa_status clsa_workspace_bytes(const clsa_params* p, size_t* bytes);
  *   scores fp32 [B][T][score_stride], score_stride >= max_seq_len
  * T == 1 streams the indexer-key cache once (HBM-bound); T > 1 is a tensor-core GEMM (tcgen05, operands staged by
  * TMA), which needs p->num_cache_rows and, for 32-byte vector stores, a 32-byte aligned `scores` with
- * score_stride % 8 == 0 (otherwise it falls back to scalar stores of the same values). Paged caches are supported for
- * T == 1 only (T > 1 with a block table returns CLSA_ERR_UNSUPPORTED). */
+ * score_stride % 8 == 0 (otherwise it falls back to scalar stores of the same values). Both paths accept paged
+ * caches (T > 1 fetches one tiled copy per cache block; num_cache_rows is then the extent of the paged row space). */
 CLSA_API clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* scores, int64_t score_stride,
                               void* workspace, size_t workspace_bytes, clsa_stream stream);
 

@@ -126,7 +126,6 @@ clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* sc
   CLSA_TRY(check_idx_cache(p));
   if (q_idx == nullptr || scores == nullptr || !aligned(q_idx, 16) || !aligned(scores, 4)) return CLSA_ERR_INVALID_ARG;
   if (score_stride < p->max_seq_len) return CLSA_ERR_INVALID_ARG;
-  if (p->q_per_seq > 1 && p->block_table != nullptr) return CLSA_ERR_UNSUPPORTED;  // the GEMM path reads contiguous key tiles
   if (p->q_per_seq > 1) {
     // the GEMM path addresses rows through 32-bit TMA coordinates and needs the extent of the cache
     if (p->num_cache_rows < 1 || p->num_cache_rows > 0x7fffffffLL) return CLSA_ERR_INVALID_ARG;

@@ -8,8 +8,11 @@
 //
 // One persistent block per SM walks output tiles of 128 queries x 256 keys (query block fastest,
 // so neighbouring SMs share a key tile in L2). Warp roles:
-//   warp 0, one lane : TMA producer. Per tile, 2 + 2 tiled bulk copies (128-byte swizzle) bring the
-//                      128 x d_idx query tile and the 256 x d_idx key tile into a 2-stage ring.
+//   warp 0           : TMA producer. Per tile, 2 + 2 tiled bulk copies (128-byte swizzle) bring the
+//                      128 x d_idx query tile and the 256 x d_idx key tile into a 2-stage ring. With a
+//                      paged key cache the key tile is assembled from one box per cache block (blocks of
+//                      16..128 rows; every box starts on a 1024-byte swizzle atom, so the assembled tile
+//                      has the layout of a single 256-row box).
 //   warp 1, one lane : MMA issuer. d_idx/16 tcgen05.mma (M128 N256 K16, kind::f16, bf16 inputs, fp32
 //                      accumulate) per tile into one of two 256-column TMEM accumulators;
 //                      tcgen05.commit frees the smem stage and publishes the accumulator.
@@ -47,6 +50,10 @@ struct GemmArgs {
   int num_seqs, q_per_seq, causal, max_seq_len, idx_dim;
   int m_blocks, n_tiles;
   int vec_ok;  // rows of `scores` are 32-byte aligned: 256-bit stores allowed
+  // paged key cache: a 256-key tile is fetched as key_boxes boxes of box_rows rows, one per cache block
+  // (block_size < 256), or as one box inside a block (block_size >= 256). Contiguous: one box, no table.
+  const int32_t* block_table;
+  int block_size, max_blocks_per_seq, box_rows, key_boxes;
 };
 
 // ---- PTX wrappers ----------------------------------------------------------------------------------
@@ -176,24 +183,45 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-    if (lane == 0) {
-      uint32_t it = 0;
-      for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
-        const TileCoord c = tile_coord(a, id);
-        if (!c.valid) continue;
-        const int s = it % kStages;
-        const uint32_t ph = (it / kStages) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) break;
-        const uint32_t st = base + s * kStageBytes;
-        mbar_expect_tx(full_bar(s), (uint32_t)kblocks * (kABytes + kBBytes));
-        const int qrow = c.b * a.q_per_seq + c.mb * kBM;
-        const int krow = (int)(a.seq_start[c.b] + (int64_t)c.nt * kBN);
-        for (int kb = 0; kb < kblocks; ++kb) {
-          tma_load_2d(st + kb * kABytes, &map_q, kb * kBK, qrow, full_bar(s));
-          tma_load_2d(st + 2 * kABytes + kb * kBBytes, &map_k, kb * kBK, krow, full_bar(s));
+    // Lane 0 owns the barriers and the query tile; key boxes are spread over the lanes (lane i fetches box i),
+    // so that a tile made of sixteen 16-row cache blocks does not queue 32 copies behind one thread.
+    uint32_t it = 0;
+    for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
+      const TileCoord c = tile_coord(a, id);
+      if (!c.valid) continue;
+      const int s = it % kStages;
+      const uint32_t ph = (it / kStages) & 1u;
+      // first cache row of this lane's key box (looked up before the wait, used after it)
+      int krow = 0, boxes = 1;
+      if (a.block_table == nullptr) {
+        krow = (int)(a.seq_start[c.b] + (int64_t)c.nt * kBN);
+      } else {
+        const int32_t* tab = a.block_table + (int64_t)c.b * a.max_blocks_per_seq;
+        const int pos0 = c.nt * kBN;
+        if (a.block_size >= kBN) {
+          krow = tab[pos0 / a.block_size] * a.block_size + pos0 % a.block_size;
+        } else {
+          // only blocks that hold positions of the sequence: entries past them need not be valid
+          boxes = min(a.key_boxes, (c.n - pos0 + a.block_size - 1) / a.block_size);
+          if (lane < boxes) krow = tab[pos0 / a.block_size + lane] * a.block_size;
         }
-        ++it;
       }
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const uint32_t st = base + s * kStageBytes;
+      const uint32_t box_bytes = (uint32_t)a.box_rows * kBK * 2;
+      if (lane == 0) {
+        mbar_expect_tx(full_bar(s), (uint32_t)kblocks * (kABytes + (uint32_t)boxes * box_bytes));
+        const int qrow = c.b * a.q_per_seq + c.mb * kBM;
+        for (int kb = 0; kb < kblocks; ++kb) tma_load_2d(st + kb * kABytes, &map_q, kb * kBK, qrow, full_bar(s));
+      }
+      __syncwarp();  // the expected byte count is posted before any key box can complete
+      if (lane < boxes)  // rows of boxes that are not fetched keep stale bits: their columns are never stored
+        for (int kb = 0; kb < kblocks; ++kb)
+          tma_load_2d(st + 2 * kABytes + kb * kBBytes + lane * box_bytes, &map_k, kb * kBK, krow, full_bar(s));
+      ++it;
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
@@ -321,9 +349,17 @@ cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, fl
   CUtensorMap map_q, map_k;
   const uint64_t q_rows = (uint64_t)p.num_seqs * p.q_per_seq;
   if (!make_map(&map_q, q_idx, q_rows, (uint64_t)p.idx_dim, (uint64_t)p.idx_dim, kBM)) return cudaErrorInvalidValue;
-  if (!make_map(&map_k, p.idx_k_cache, (uint64_t)p.num_cache_rows, (uint64_t)p.idx_dim, (uint64_t)p.idx_token_stride, kBN))
+  const bool paged = p.block_table != nullptr;
+  const int box_rows = paged && p.block_size < kBN ? p.block_size : kBN;
+  if (!make_map(&map_k, p.idx_k_cache, (uint64_t)p.num_cache_rows, (uint64_t)p.idx_dim, (uint64_t)p.idx_token_stride,
+                (uint32_t)box_rows))
     return cudaErrorInvalidValue;
   GemmArgs a;
+  a.block_table = p.block_table;
+  a.block_size = paged ? p.block_size : 0;
+  a.max_blocks_per_seq = p.max_blocks_per_seq;
+  a.box_rows = box_rows;
+  a.key_boxes = kBN / box_rows;
   a.seq_start = p.seq_start;
   a.seq_len = p.seq_len;
   a.scores = scores;

@@ -69,8 +69,8 @@ def test_paged_arguments_are_validated():
         clsa.clsa_topk(g.params, s, g.score_stride, g.idx, g.count, g.ws)
     assert e.value.status == clsa.CLSA_ERR_INVALID_ARG
     g.params.max_blocks_per_seq = g.t["block_table"].shape[1]
-    g.params.q_per_seq = 4                    # chunked scores on a paged cache are not built
-    g.params.num_cache_rows = g.t["idx_k_cache"].shape[0]
+    g.params.q_per_seq = 4                    # chunked scores need the extent of the (paged) row space
+    g.params.num_cache_rows = 0
     with pytest.raises(clsa.ClsaError) as e:
         clsa.clsa_index_scores(g.params, g.t["q_idx"], s, g.score_stride, g.ws)
-    assert e.value.status == clsa.CLSA_ERR_UNSUPPORTED
+    assert e.value.status == clsa.CLSA_ERR_INVALID_ARG

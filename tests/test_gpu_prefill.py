@@ -50,6 +50,31 @@ def test_chunk_scores_topk_attention(B, T, n, d_idx, causal, ragged):
     assert g.status() == 0
 
 
+@pytest.mark.parametrize("B,T,n,d_idx,causal,ragged,bs", [
+    (2, 200, 3000, 128, 1, 0, 16), (1, 300, 2500, 64, 1, 0, 64), (3, 150, 2000, 128, 1, 500, 128),
+    (2, 77, 1111, 128, 0, 0, 256), (1, 260, 5000, 128, 1, 0, 1024), (2, 130, 300, 64, 1, 0, 32)])
+def test_chunk_on_paged_caches(B, T, n, d_idx, causal, ragged, bs):
+    """Paging changes addresses only: the chunk's scores are bit-identical to the contiguous run, and the rest of
+    the chunk path (top-k, attention through the block table) agrees with the oracle."""
+    base = MID if d_idx == 128 else TINY
+    cfg = base.replace(num_seqs=B, ctx=n, q_per_seq=T, causal=causal, top_k=96, num_layers=1, seed=700 + T + n + bs,
+                       ragged_min=ragged, num_short=0)
+    w = Workload(cfg)
+    flat, g = GpuProblem(w), GpuProblem(w, block_size=bs)
+    prob = _full_oracle(w)
+    ref_scores = prob.index_scores(w.q_idx_bits())
+    gs = g.index_scores()
+    torch.cuda.synchronize()
+    assert g.status() == 0
+    check_scores(gs, ref_scores, w)
+    assert torch.equal(gs.nan_to_num(7.0), flat.index_scores().nan_to_num(7.0))
+    gi, gc = g.topk(gs)
+    check_topk_exact_on_gpu_scores(prob, gs, gi, gc, w)
+    out, lse = g.sparse_attn(0)
+    check_attention(prob, w, 0, out, lse, gi.cpu().numpy().copy(), gc.cpu().numpy().copy())
+    assert g.status() == 0
+
+
 def test_gemm_row_equals_decode_gemv():
     """Row t of the chunk GEMM is the decode kernel's result for the same query against the same keys."""
     w = Workload(MID.replace(num_seqs=1, ctx=4096, q_per_seq=256, causal=0, top_k=64, num_layers=1, seed=31))
