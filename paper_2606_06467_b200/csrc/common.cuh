@@ -56,6 +56,9 @@ cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, fl
                                      uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,
                         uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx,
+                                  int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream,
+                                  int* launched);
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
                                const DeviceInfo& dev, cudaStream_t stream);

@@ -162,27 +162,21 @@ __device__ __forceinline__ void radix_pass(Shared& sh, cg::cluster_group& cluste
   k_rem = sh.k_rem;
 }
 
+// One (sequence, query) row, by the calling cluster (one block when the cluster has one).
 template <bool CACHED>
-__global__ void __launch_bounds__(kThreads, 1)
-topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const int32_t* __restrict__ seq_len,
-                  int q_per_seq, int causal, int top_k, int max_seq_len, int32_t* __restrict__ idx_out,
-                  int32_t* __restrict__ count_out, uint32_t* status) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ __forceinline__ void topk_row(const int row, const float* __restrict__ scores, int64_t score_stride,
+                                         const int32_t* __restrict__ seq_len, int q_per_seq, int causal, int top_k,
+                                         int max_seq_len, int32_t* __restrict__ idx_out, int32_t* __restrict__ count_out,
+                                         uint32_t* status, unsigned char* smem_raw) {
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Shared));
 
   cg::cluster_group cluster = cg::this_cluster();
   const int nblk = (int)cluster.num_blocks();
   const int rank = (int)cluster.block_rank();
-  const int row = blockIdx.x / nblk;
   const int b = row / q_per_seq, t = row % q_per_seq;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  // Programmatic dependent launch: this grid may have been scheduled before the kernel that writes
-  // the scores has finished; wait for it here, before the first global read, and let the kernel
-  // after this one be scheduled early in turn.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // Everything up to the first cluster.sync() is uniform over the cluster (same row, same lengths).
   const int n = seq_len[b];
   int v = causal ? n - q_per_seq + t + 1 : n;
@@ -483,6 +477,46 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
   cluster_wait();  // no block may exit while a neighbour can still read its shared memory (arrived earlier)
 }
 
+constexpr int kPendingRowsPerBlock = 16;  // rows a block of the pending-only launch looks after (all pending: still >= 148 blocks for 2400 rows)
+
+template <bool CACHED>
+__global__ void __launch_bounds__(kThreads, 1)
+topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const int32_t* __restrict__ seq_len,
+                  int q_per_seq, int causal, int top_k, int max_seq_len, int pending_rows,
+                  int32_t* __restrict__ idx_out, int32_t* __restrict__ count_out, uint32_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  // Programmatic dependent launch: this grid may have been scheduled before the kernel that writes
+  // the scores has finished; wait for it here, before the first global read, and let the kernel
+  // after this one be scheduled early in turn.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (pending_rows == 0) {
+    const int nblk = (int)cg::this_cluster().num_blocks();
+    topk_row<CACHED>(blockIdx.x / nblk, scores, score_stride, seq_len, q_per_seq, causal, top_k, max_seq_len, idx_out,
+                     count_out, status, smem_raw);
+    return;
+  }
+  // Second kernel of the many-rows route (one block per kPendingRowsPerBlock rows, no clusters): the one-sweep
+  // kernel before this one has done every row it could and left count = -1 on the others. All marks of this
+  // block's rows are read in one round trip; the usual outcome is that none is set.
+  __shared__ int pending[kPendingRowsPerBlock];
+  const int first = blockIdx.x * kPendingRowsPerBlock;
+  int mine = 0;
+  if (threadIdx.x < kPendingRowsPerBlock) {
+    const int row = first + threadIdx.x;
+    mine = (row < pending_rows && count_out[row] == -1) ? 1 : 0;
+    pending[threadIdx.x] = mine;
+  }
+  if (__syncthreads_or(mine) == 0) return;
+  for (int j = 0; j < kPendingRowsPerBlock; ++j) {
+    if (pending[j]) {
+      topk_row<CACHED>(first + j, scores, score_stride, seq_len, q_per_seq, causal, top_k, max_seq_len, idx_out,
+                       count_out, status, smem_raw);
+      __syncthreads();  // the next row reuses this block's shared memory
+    }
+  }
+}
+
 }  // namespace
 
 TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev) {
@@ -518,11 +552,20 @@ cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score
                         uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
   const TopkPlan plan = make_topk_plan(p, dev);
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
+  // Many long rows (a prefill chunk): a one-sweep kernel takes every row it can finish exactly and marks the
+  // rest; the general kernel below then runs for the marked rows only.
+  int pending_only = 0;
+  if (plan.cluster == 1) {
+    const cudaError_t pre = launch_topk_prefilter(p, scores, score_stride, idx, count, status, dev, stream, &pending_only);
+    if (pre != cudaSuccess) return pre;
+  }
+  const int pending_rows = pending_only ? (int)rows : 0;
+  const int64_t blocks = pending_only ? (rows + kPendingRowsPerBlock - 1) / kPendingRowsPerBlock : rows * plan.cluster;
   auto kernel = plan.slice_cap > 0 ? topk_radix_kernel<true> : topk_radix_kernel<false>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(rows * plan.cluster), 1, 1);
+  cfg.gridDim = dim3((unsigned)blocks, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
@@ -536,7 +579,7 @@ cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, scores, score_stride, p.seq_len, (int)p.q_per_seq, (int)p.causal,
-                            (int)p.top_k, (int)p.max_seq_len, idx, count, status);
+                            (int)p.top_k, (int)p.max_seq_len, pending_rows, idx, count, status);
 }
 
 }  // namespace clsa
