@@ -53,9 +53,11 @@ struct alignas(16) Shared {  // the keys follow it in shared memory and are writ
   uint32_t rank_gt[kMaxCluster], rank_eq[kMaxCluster];  // per block of the cluster: candidates above / equal to the threshold
   uint32_t digit, k_rem, bin_count;
   uint32_t out_base, eq_base;
+  uint32_t eq_n, use_bitmap, pad_[2];
 };
 
 // Split cluster barrier: arrive early, wait late, so the barrier's latency hides behind independent work.
+static_assert(kWarps == 32, "lane l reads warp l's total");
 static_assert(sizeof(Shared) % 16 == 0, "the key array behind Shared must stay 16-byte aligned");
 
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
@@ -273,6 +275,12 @@ __device__ __forceinline__ void topk_row(const int row, const float* __restrict_
   const int c_lo = min(cnt, warp * chunk), c_hi = min(cnt, c_lo + chunk);
   uint32_t thr, need_eq;
 
+  // Short path only: selected positions of this slice as a bitmap (the first histogram copy is free again after
+  // its scan cleared it), so that the last step is a prefix count over at most 4096 words instead of a third
+  // sweep over the keys.
+  uint32_t* bitmap = sh.cluster_hist[0];
+  const bool use_bitmap = in_bin <= (uint32_t)kCandCap && cnt <= kMaxBins * 32;
+  bool emitted = false;
   if (in_bin <= (uint32_t)kCandCap) {
     // ---- short path: sweep 2 counts keys above the bin per warp and collects the bin's keys ----------
     uint2* cand = reinterpret_cast<uint2*>(sh.cluster_hist[1]);  // (key, slice position), unordered
@@ -288,7 +296,10 @@ __device__ __forceinline__ void topk_row(const int row, const float* __restrict_
       for (int u = 0; u < 4; ++u) {
         const int i = i0 + 32 * u + lane;
         const uint32_t top = key[u] >> 20;
-        gt += (i < c_hi && top > digit0) ? 1u : 0u;
+        // keys above the threshold's bin are certainly selected: their ballot is the position bitmap's word
+        const uint32_t gtb = __ballot_sync(0xffffffffu, i < c_hi && top > digit0);
+        if (use_bitmap && lane == 0 && i0 + 32 * u < c_hi) bitmap[(i0 + 32 * u) >> 5] = gtb;
+        gt += (uint32_t)__popc(gtb);  // the same on every lane
         const bool is_c = i < c_hi && top == digit0;
         const uint32_t cb = __ballot_sync(0xffffffffu, is_c);
         if (cb != 0u) {
@@ -299,8 +310,6 @@ __device__ __forceinline__ void topk_row(const int row, const float* __restrict_
         }
       }
     }
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) gt += __shfl_xor_sync(0xffffffffu, gt, d);
     if (lane == 0) { sh.warp_gt[warp] = gt; sh.warp_eq[warp] = 0; atomicAdd(&sh.block_gt0, gt); }
     cluster.sync();  // every block's candidate list, candidate count and above-the-bin count are complete
     // gather the row's candidates (keys only) into local_hist[0..in_bin)
@@ -356,11 +365,13 @@ __device__ __forceinline__ void topk_row(const int row, const float* __restrict_
     need_eq = k_rem;
     // per-warp counts of this block: keys above the bin (already counted) plus candidates above / equal to thr
     const uint32_t my_n = sh.cand_count;
-    for (uint32_t i = tid; i < my_n; i += kThreads) {
-      const uint2 c = cand[i];
-      const int w = (int)c.y / chunk;
-      if (c.x > thr) atomicAdd(&sh.warp_gt[w], 1u);
-      else if (c.x == thr) atomicAdd(&sh.warp_eq[w], 1u);
+    if (!use_bitmap) {  // only the ordered sweep at the end needs them
+      for (uint32_t i = tid; i < my_n; i += kThreads) {
+        const uint2 c = cand[i];
+        const int w = (int)c.y / chunk;
+        if (c.x > thr) atomicAdd(&sh.warp_gt[w], 1u);
+        else if (c.x == thr) atomicAdd(&sh.warp_eq[w], 1u);
+      }
     }
     // the same two counts for every block of the cluster, from the gathered candidates (grouped by block):
     // with them each block derives its output offset alone, without another exchange
@@ -385,9 +396,64 @@ __device__ __forceinline__ void topk_row(const int row, const float* __restrict_
         sel_before += gr + take;
         eq_before += er;
       }
-      if (lane == 0) { sh.out_base = sel_before; sh.eq_base = eq_before; }
+      if (lane == 0) { sh.out_base = sel_before; sh.eq_base = eq_before; sh.eq_n = 0u; }
     }
     __syncthreads();
+    if (use_bitmap) {
+      // threshold-equal candidates of this block that are taken: the lowest positions, after those of lower blocks
+      const uint32_t my_eq = sh.rank_eq[rank];
+      const uint32_t quota = sh.eq_base >= need_eq ? 0u : min(my_eq, need_eq - sh.eq_base);
+      uint32_t* eq_pos = sh.local_hist;  // the gathered candidates and their histogram are dead by now
+      const bool partial = quota != 0u && quota != my_eq;  // my_eq <= kCandCap entries: they fit eq_pos
+      {
+        for (uint32_t i = tid; i < my_n; i += kThreads) {
+          const uint2 c = cand[i];
+          if (c.x > thr || (c.x == thr && quota == my_eq)) atomicOr(&bitmap[c.y >> 5], 1u << (c.y & 31u));
+          else if (c.x == thr && partial) eq_pos[atomicAdd(&sh.eq_n, 1u)] = c.y;
+        }
+        __syncthreads();
+        if (partial) {
+          for (uint32_t i = tid; i < my_eq; i += kThreads) {
+            const uint32_t mine = eq_pos[i];
+            uint32_t lower = 0;
+            for (uint32_t j = 0; j < my_eq; ++j) lower += eq_pos[j] < mine;
+            if (lower < quota) atomicOr(&bitmap[mine >> 5], 1u << (mine & 31u));
+          }
+          __syncthreads();
+        }
+        // prefix count over the bitmap words, then every thread writes the positions of its own words
+        const int words = (cnt + 31) >> 5;
+        const int wpt = (words + kThreads - 1) / kThreads;
+        const int w_lo = min(words, tid * wpt), w_hi = min(words, w_lo + wpt);
+        uint32_t mine = 0;
+        for (int w = w_lo; w < w_hi; ++w) mine += __popc(bitmap[w]);
+        uint32_t incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
+          if (lane >= d) incl += up;
+        }
+        if (lane == 31) sh.warp_tot[warp] = incl;
+        __syncthreads();
+        uint32_t tot = sh.warp_tot[lane];  // kWarps == 32: lane l holds warp l's total
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t up = __shfl_up_sync(0xffffffffu, tot, d);
+          if (lane >= d) tot += up;
+        }
+        const uint32_t below = __shfl_sync(0xffffffffu, tot, (warp + 31) & 31);
+        uint32_t off = sh.out_base + (warp == 0 ? 0u : below) + incl - mine;
+        for (int w = w_lo; w < w_hi; ++w) {
+          uint32_t bits = bitmap[w];
+          while (bits != 0u) {
+            if (off < (uint32_t)kk) out[off] = lo + w * 32 + __ffs(bits) - 1;
+            ++off;
+            bits &= bits - 1u;
+          }
+        }
+        emitted = true;
+      }
+    }
   } else {
     // ---- long path: two more cluster-wide radix passes, then a counting sweep ------------------------
     uint32_t prefix = digit0 << 20, prefix_mask = 0xfff00000u;
@@ -436,7 +502,11 @@ __device__ __forceinline__ void topk_row(const int row, const float* __restrict_
     cluster_arrive();  // pairs with the wait at the very end
   }
 
-  // ---- index-ordered compaction ----------------------------------------------------------------------
+  if (emitted) {
+    cluster_wait();  // no block may exit while a neighbour can still read its shared memory (arrived earlier)
+    return;
+  }
+  // ---- index-ordered compaction (long path, and short-path slices the bitmap route does not take) ------------
   // offsets of this warp: selected / threshold-equal keys in lower warps of this block
   uint32_t out_pos = sh.out_base, eq_rank = sh.eq_base;
   for (int w = 0; w < warp; ++w) {
