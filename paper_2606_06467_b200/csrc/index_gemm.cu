@@ -17,9 +17,11 @@
 //                      accumulate) per tile into one of two 256-column TMEM accumulators;
 //                      tcgen05.commit frees the smem stage and publishes the accumulator.
 //   warp 2           : allocates / frees the 512 TMEM columns.
-//   warps 4..7       : epilogue. Each warp owns 32 TMEM lanes (= 32 query rows): tcgen05.ld 32
-//                      columns at a time, then 32-byte vector stores of the visible part of the row
-//                      (causal limit per query), so the epilogue of tile i overlaps the MMAs of tile i+1.
+//   warps 4..11      : epilogue. Two warps per 32 TMEM lanes (= 32 query rows), 128 columns each: tcgen05.ld 32
+//                      columns at a time (double-buffered), a transposition through shared memory, then
+//                      32-byte vector stores, four lanes per row, of the visible part of each row (causal
+//                      limit per query): whole 128-byte lines per store instruction. The epilogue of tile i
+//                      overlaps the MMAs of tile i+1.
 // Tiles that lie entirely above the causal diagonal are skipped by every role alike.
 // Every mbarrier wait is bounded: on expiry the block raises CLSA_DEV_TIMEOUT in the status word,
 // all roles leave their loops, in-flight copies are given time to land, TMEM is freed, and the
@@ -33,12 +35,14 @@ namespace {
 
 constexpr int kBM = 128, kBN = 256, kBK = 64;  // tile; kBK bf16 = one 128-byte swizzle row
 constexpr int kStages = 2, kAccBufs = 2;
-constexpr int kThreads = 256;
+constexpr int kEpiWarps = 8;                     // two per TMEM lane quadrant, 128 columns each
+constexpr int kThreads = (4 + kEpiWarps) * 32;
 constexpr int kABytes = kBM * kBK * 2;          // one k-block of the query tile (16 KiB)
 constexpr int kBBytes = kBN * kBK * 2;          // one k-block of the key tile (32 KiB)
 constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;  // up to two k-blocks each (96 KiB)
 constexpr int kBarrierBytes = 128;
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+constexpr int kEpiTileBytes = kEpiWarps * 32 * 33 * 4;  // one padded 32 x 32 fp32 transposition tile per epilogue warp
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + kBarrierBytes + kEpiTileBytes + 1024;  // + alignment slack
 constexpr uint32_t kSpinLimit = 1u << 22;       // polls with back-off: a few seconds at most
 
 struct GemmArgs {
@@ -168,7 +172,7 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int i = 0; i < kAccBufs; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 4); }
+    for (int i = 0; i < kAccBufs; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), kEpiWarps); }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -254,7 +258,8 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     }
   } else if (warp >= 4) {
     // ---------------- epilogue: TMEM -> registers -> global ----------------
-    const int quad = warp & 3;  // TMEM lanes 32*quad .. 32*quad+31
+    const int quad = warp & 3;          // TMEM lanes 32*quad .. 32*quad+31 (a warp may only touch its own quadrant)
+    const int half = (warp - 4) >> 2;   // which 128 of the tile's 256 columns
     uint32_t it = 0;
     for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
       const TileCoord c = tile_coord(a, id);
@@ -266,32 +271,62 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       const int t = c.mb * kBM + quad * 32 + lane;       // query of this thread's row
       const bool row_ok = t < a.q_per_seq;
       const int v = row_ok ? (a.causal ? c.n - a.q_per_seq + t + 1 : c.n) : 0;  // visible keys of this query
-      float* orow = a.scores + ((int64_t)c.b * a.q_per_seq + t) * a.score_stride;
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kBN);
-#pragma unroll 1
-      for (int c0 = 0; c0 < kBN; c0 += 32) {
-        const int s0 = c.nt * kBN + c0;
-        if (__all_sync(0xffffffffu, s0 >= v)) break;     // the rest of the tile is above the diagonal for this warp
-        uint32_t r[32];
-        tc_ld32(taddr + (uint32_t)c0, r);
-        tc_ld_wait();
+      // 32 columns at a time through two register buffers (the TMEM load of the next 32 columns is in flight
+      // while the current 32 are stored). A TMEM load leaves a lane with 32 columns of ONE row; stored as they
+      // come, a warp instruction would scatter 32-byte pieces over 32 rows. They go through a padded
+      // shared-memory tile instead and come back with four lanes per row, so that every store instruction writes
+      // eight complete 128-byte lines.
+      float* tile = reinterpret_cast<float*>(base_ptr + kStages * kStageBytes + kBarrierBytes) + (warp - 4) * (32 * 33);
+      const int t0 = c.mb * kBM + quad * 32;  // first query row of this warp
+      auto store32 = [&](const uint32_t (&r)[32], int s0) {
+        __syncwarp();  // the previous chunk's reads of the tile are done
 #pragma unroll
-        for (int j = 0; j < 32; j += 8) {
-          const int s = s0 + j;
-          if (a.vec_ok && s + 8 <= v) {
-            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(orow + s), "r"(r[j]), "r"(r[j + 1]),
-                         "r"(r[j + 2]), "r"(r[j + 3]), "r"(r[j + 4]), "r"(r[j + 5]), "r"(r[j + 6]), "r"(r[j + 7])
+        for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = __uint_as_float(r[j]);  // bank (lane + j) % 32: no conflicts
+        __syncwarp();
+        const int s = s0 + (lane & 3) * 8;  // this lane's 8 columns
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int row = k * 8 + (lane >> 2);
+          const int tq = t0 + row;
+          const int vr = tq < a.q_per_seq ? (a.causal ? c.n - a.q_per_seq + tq + 1 : c.n) : 0;
+          if (s >= vr) continue;
+          const float* src = tile + row * 33 + (lane & 3) * 8;  // bank (row + 8 * (lane & 3) + e) % 32: no conflicts
+          float w[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) w[e] = src[e];
+          float* dst = a.scores + ((int64_t)c.b * a.q_per_seq + tq) * a.score_stride + s;
+          if (a.vec_ok && s + 8 <= vr) {
+            asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "f"(w[0]), "f"(w[1]), "f"(w[2]),
+                         "f"(w[3]), "f"(w[4]), "f"(w[5]), "f"(w[6]), "f"(w[7])
                          : "memory");
           } else {
 #pragma unroll
             for (int e = 0; e < 8; ++e)
-              if (s + e < v) orow[s + e] = __uint_as_float(r[j + e]);
+              if (s + e < vr) dst[e] = w[e];
           }
+        }
+      };
+      // columns this warp has to drain: up to the last one any of its 32 queries can see (a multiple of 32)
+      const int v_warp = __reduce_max_sync(0xffffffffu, v) - c.nt * kBN;
+      const int c_begin = half * (kBN / 2);
+      const int c_end = min(c_begin + kBN / 2, (max(v_warp, 0) + 31) & ~31);
+      uint32_t ra[32], rb[32];
+      if (c_end > c_begin) tc_ld32(taddr + (uint32_t)c_begin, ra);
+#pragma unroll 1
+      for (int c0 = c_begin; c0 < c_end; c0 += 64) {
+        tc_ld_wait();
+        if (c0 + 32 < c_end) tc_ld32(taddr + (uint32_t)(c0 + 32), rb);
+        store32(ra, c.nt * kBN + c0);
+        if (c0 + 32 < c_end) {
+          tc_ld_wait();
+          if (c0 + 64 < c_end) tc_ld32(taddr + (uint32_t)(c0 + 64), ra);
+          store32(rb, c.nt * kBN + c0 + 32);
         }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));        // 4 arrivals (one per epilogue warp) free the accumulator
+      if (lane == 0) mbar_arrive(tempty_bar(acc));        // one arrival per epilogue warp frees the accumulator
       ++it;
     }
   }
