@@ -136,3 +136,38 @@ def test_many_rows_misaligned_rows_and_non_finite_scores_keep_the_contract():
     sub = Workload(MID.replace(num_seqs=1, ctx=n, q_per_seq=len(finite_rows), causal=0, top_k=k, num_layers=1))
     check_topk_exact_on_gpu_scores(oracle.problem_from_workload(sub), sc2[:, finite_rows], g2.idx[:, finite_rows],
                                    g2.count[:, finite_rows], sub)
+
+
+def test_many_sequences_one_query_each():
+    """The same route when the rows are 640 sequences of different lengths (a large decode batch), not the queries
+    of one chunk: selection only, on random scores, against the oracle's sort."""
+    B, k, n_max = ROWS, 800, 16000
+    rng = np.random.default_rng(99)
+    lens = rng.integers(500, n_max + 1, B).astype(np.int32)
+    lens[:3] = (n_max, 799, 6145)                      # longest, shorter than k, just above the candidate list's capacity
+    dev = torch.device("cuda:0")
+    stride = (n_max + 63) // 64 * 64
+    sc_host = (rng.standard_normal((B, 1, stride)) * 11.3).astype(np.float32)
+    sc = torch.from_numpy(sc_host).to(dev)
+    seq_len = torch.from_numpy(lens).to(dev)
+    seq_start = torch.zeros(B, dtype=torch.int64, device=dev)
+    kv = torch.zeros((8, 8, 128), dtype=torch.bfloat16, device=dev)
+    ik = torch.zeros((8, 128), dtype=torch.bfloat16, device=dev)
+    p = clsa.make_params(num_seqs=B, q_per_seq=1, num_q_heads=32, num_kv_heads=8, head_dim=128, idx_dim=128, top_k=k,
+                         num_layers=1, max_seq_len=n_max, sm_scale=0.1, seq_start=seq_start, seq_len=seq_len, k_cache=kv,
+                         v_cache=kv, idx_k_cache=ik)
+    ws = torch.zeros(clsa.clsa_workspace_bytes(p), dtype=torch.uint8, device=dev)
+    idx = torch.full((B, 1, k), -7, dtype=torch.int32, device=dev)
+    cnt = torch.full((B, 1), -7, dtype=torch.int32, device=dev)
+    clsa.clsa_topk(p, sc, stride, idx, cnt, ws)
+    torch.cuda.synchronize()
+    assert clsa.clsa_device_status(ws) == 0
+    prob = oracle.Problem(num_seqs=B, q_per_seq=1, num_q_heads=32, num_kv_heads=8, head_dim=128, idx_dim=128, top_k=k,
+                          sm_scale=0.1, seq_start=np.zeros(B, np.int64), seq_len=lens)
+    ref_idx, ref_cnt = prob.topk(sc_host.astype(np.float64))
+    gi, gc = idx.cpu().numpy(), cnt.cpu().numpy()
+    np.testing.assert_array_equal(gc, ref_cnt)
+    for b in range(B):
+        c = gc[b, 0]
+        np.testing.assert_array_equal(gi[b, 0, :c], np.sort(ref_idx[b, 0, :c]))
+        assert (gi[b, 0, c:] == -1).all()
