@@ -179,6 +179,13 @@ __device__ __forceinline__ void topk_row(const int row, const float* __restrict_
   const int b = row / q_per_seq, t = row % q_per_seq;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+  // Shared-memory state first: it needs nothing from global memory, so it is cleared while the kernel that
+  // produces the scores may still be running (programmatic dependent launch); only then wait for that kernel.
+  for (int i = tid; i < kMaxBins; i += kThreads) { sh.local_hist[i] = 0; sh.cluster_hist[0][i] = 0; }
+  if (tid < kMaxCluster) { sh.rank_gt[tid] = 0; sh.rank_eq[tid] = 0; }
+  if (tid == 0) { sh.cand_count = 0; sh.block_gt0 = 0; }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
   // Everything up to the first cluster.sync() is uniform over the cluster (same row, same lengths).
   const int n = seq_len[b];
   int v = causal ? n - q_per_seq + t + 1 : n;
@@ -202,9 +209,6 @@ __device__ __forceinline__ void topk_row(const int row, const float* __restrict_
   const float* src = scores + (int64_t)row * score_stride + lo;
   auto key_at = [&](int i) -> uint32_t { return CACHED ? keys[i] : score_key(src[i]); };
 
-  for (int i = tid; i < kMaxBins; i += kThreads) { sh.local_hist[i] = 0; sh.cluster_hist[0][i] = 0; }
-  if (tid < kMaxCluster) { sh.rank_gt[tid] = 0; sh.rank_eq[tid] = 0; }
-  if (tid == 0) { sh.cand_count = 0; sh.block_gt0 = 0; }
   __syncthreads();
   // Remote adds may land in this block's histogram copy only after it has been cleared: every block arrives
   // here and waits just before it starts adding, with the whole first sweep in between.
@@ -555,10 +559,9 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
                   int q_per_seq, int causal, int top_k, int max_seq_len, int pending_rows,
                   int32_t* __restrict__ idx_out, int32_t* __restrict__ count_out, uint32_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // Programmatic dependent launch: this grid may have been scheduled before the kernel that writes
-  // the scores has finished; wait for it here, before the first global read, and let the kernel
-  // after this one be scheduled early in turn.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Programmatic dependent launch: this grid may have been scheduled before the kernel that writes the scores
+  // has finished. The kernel after this one may be scheduled early in turn (it waits for this grid itself);
+  // this grid's own wait sits in topk_row, after the shared-memory clears and before the first global access.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (pending_rows == 0) {
     const int nblk = (int)cg::this_cluster().num_blocks();
@@ -569,6 +572,7 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
   // Second kernel of the many-rows route (one block per kPendingRowsPerBlock rows, no clusters): the one-sweep
   // kernel before this one has done every row it could and left count = -1 on the others. All marks of this
   // block's rows are read in one round trip; the usual outcome is that none is set.
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the marks come from the kernel just before this one
   __shared__ int pending[kPendingRowsPerBlock];
   const int first = blockIdx.x * kPendingRowsPerBlock;
   int mine = 0;
