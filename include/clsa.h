@@ -147,6 +147,17 @@ CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, c
                              void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
                              size_t workspace_bytes, clsa_stream stream);
 
+/* Eq. 4 for all L layers that share one index (Sec. 2.1): the attention half of clsa_decode_step on its own, for a
+ * caller that has the index already (from clsa_index_scores + clsa_topk) -- for instance to let the layers' queries
+ * arrive on another stream while the routing runs, making `stream` wait on that upload just before this call.
+ *   q_layers / out_layers  HOST arrays of L device pointers, each bf16 [B][T][Hq][D], 16-byte aligned
+ *   idx, count             as written by clsa_topk (read only)
+ * Bit for bit the L calls of clsa_sparse_attn with sweep = (p->sweep + l) & 1 and lse = NULL, launched so that a
+ * layer may start while its predecessor's last blocks finish (which is why the calls are offered as one). */
+CLSA_API clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* const* q_layers, const int32_t* idx,
+                                             const int32_t* count, void* const* out_layers, void* workspace,
+                                             size_t workspace_bytes, clsa_stream stream);
+
 /* The step immediately before the path (Eq. 2 and the append of the new tokens' cache rows): for query token t
  * of sequence b, at position s = seq_len[b] - T + t (the sequence's newest tokens, whose rows this call fills),
  *   q_idx_out[b][t][:]        = h[b][t][:] W^Q_idx                     (Eq. 2)

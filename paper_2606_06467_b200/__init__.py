@@ -49,6 +49,7 @@ _lib.clsa_topk.argtypes = [_P, _vp, _i64, _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_sparse_attn.argtypes = [_P, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_decode_step.argtypes = [_P, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_decode_step_static.argtypes = [_P, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _vp, _vp, _vp]
+_lib.clsa_sparse_attn_layers.argtypes = [_P, ctypes.POINTER(_vp), _vp, _vp, ctypes.POINTER(_vp), _vp, _sz, _vp]
 _lib.clsa_project_append.argtypes = [_P, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_clear_status.argtypes = [_vp, _sz, _vp]
 _lib.clsa_device_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32), _vp]
@@ -56,11 +57,13 @@ _lib.clsa_status_string.argtypes = [ctypes.c_int]
 _lib.clsa_status_string.restype = ctypes.c_char_p
 _lib.clsa_version.restype = ctypes.c_int
 for _name in ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_decode_step",
-              "clsa_decode_step_static", "clsa_project_append", "clsa_clear_status", "clsa_device_status"):
+              "clsa_decode_step_static", "clsa_sparse_attn_layers", "clsa_project_append", "clsa_clear_status",
+              "clsa_device_status"):
     getattr(_lib, _name).restype = ctypes.c_int
 
 EXPORTS = ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_decode_step",
-           "clsa_decode_step_static", "clsa_project_append", "clsa_clear_status", "clsa_device_status",
+           "clsa_decode_step_static", "clsa_sparse_attn_layers", "clsa_project_append", "clsa_clear_status",
+           "clsa_device_status",
            "clsa_status_string", "clsa_version")
 
 
@@ -175,6 +178,17 @@ def clsa_decode_step_static(p, q_idx, q_layers, out_layers, idx, count, dev_stat
     outs = (_vp * L)(*[_ptr(t) for t in out_layers])
     _check(_lib.clsa_decode_step_static(ctypes.byref(p), _ptr(q_idx), qs, outs, _ptr(idx), _ptr(count),
                                         _ptr(dev_status), _stream(stream)), "clsa_decode_step_static")
+
+
+def clsa_sparse_attn_layers(p, q_layers, idx, count, out_layers, workspace, workspace_bytes=None, stream=None) -> None:
+    """The L attention launches of clsa_decode_step on an index that already exists (idx, count from clsa_topk)."""
+    L = p.num_layers
+    if len(q_layers) != L or len(out_layers) != L:
+        raise ValueError("q_layers and out_layers must have num_layers entries")
+    qs = (_vp * L)(*[_ptr(t) for t in q_layers])
+    outs = (_vp * L)(*[_ptr(t) for t in out_layers])
+    _check(_lib.clsa_sparse_attn_layers(ctypes.byref(p), qs, _ptr(idx), _ptr(count), outs, _ptr(workspace),
+                                        _nbytes(workspace, workspace_bytes), _stream(stream)), "clsa_sparse_attn_layers")
 
 
 def clsa_project_append(p, d_model, h, w_q_idx, w_k_idx, w_k, w_v, q_idx_out, workspace, workspace_bytes=None,

@@ -103,6 +103,20 @@ clsa_status check_workspace(const void* ws, size_t ws_bytes, size_t need) {
 
 clsa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? CLSA_OK : CLSA_ERR_CUDA; }
 
+// The L attention launches that share one index. Layer l walks the selected set in direction (sweep + l) & 1, so a
+// layer starts on the rows its predecessor touched last. Layer 0 follows whatever produced the index and must wait
+// for it; every later layer reads only what was complete before its predecessor started (the index, the caches,
+// the caller's queries), so it may overlap its predecessor's tail.
+cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, void* const* out_layers, const int32_t* idx,
+                          const int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t s) {
+  for (int l = 0; l < p.num_layers; ++l) {
+    const cudaError_t err = launch_sparse_attn(p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p.sweep + l) & 1,
+                                               l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0, dev, s);
+    if (err != cudaSuccess) return err;
+  }
+  return cudaSuccess;
+}
+
 }  // namespace
 }  // namespace clsa
 
@@ -197,16 +211,26 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
   if (err != cudaSuccess) return CLSA_ERR_CUDA;
   err = launch_topk(*p, scores, w.score_stride, idx, count, status, dev, s);
   if (err != cudaSuccess) return CLSA_ERR_CUDA;
-  for (int l = 0; l < p->num_layers; ++l) {
-    // alternate the sweep direction so that a layer starts on the rows its predecessor touched last
-    // Layer 0 follows the top-k kernel and must wait for its index; every later layer reads only what
-    // was complete before its predecessor started (the index, the caches, the caller's queries), so it
-    // may overlap its predecessor's tail.
-    err = launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p->sweep + l) & 1,
-                             l == 0 ? 1 : 0, l + 1 < p->num_layers ? 1 : 0, dev, s);
-    if (err != cudaSuccess) return CLSA_ERR_CUDA;
-  }
+  if (launch_layers(*p, q_layers, out_layers, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
   return CLSA_OK;
+}
+
+clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* const* q_layers, const int32_t* idx,
+                                    const int32_t* count, void* const* out_layers, void* workspace,
+                                    size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  CLSA_TRY(check_kv_cache(p));
+  if (q_layers == nullptr || out_layers == nullptr || idx == nullptr || count == nullptr) return CLSA_ERR_INVALID_ARG;
+  if (!aligned(idx, 4) || !aligned(count, 4)) return CLSA_ERR_INVALID_ARG;
+  for (int l = 0; l < p->num_layers; ++l)
+    if (q_layers[l] == nullptr || out_layers[l] == nullptr || !aligned(q_layers[l], 16) || !aligned(out_layers[l], 16))
+      return CLSA_ERR_INVALID_ARG;
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  return from_cuda(launch_layers(*p, q_layers, out_layers, idx, count, static_cast<uint32_t*>(workspace), dev,
+                                 static_cast<cudaStream_t>(stream)));
 }
 
 clsa_status clsa_project_append(const clsa_params* p, int32_t d_model, const void* h, const void* w_q_idx,
@@ -287,10 +311,7 @@ clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, con
   auto scores = reinterpret_cast<float*>(base + kStatusBytes);
   if (launch_index_scores_decode(*p, q_idx, scores, stride, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
   if (launch_topk(*p, scores, stride, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
-  for (int l = 0; l < p->num_layers; ++l)
-    if (launch_sparse_attn(*p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p->sweep + l) & 1,
-                           l == 0 ? 1 : 0, l + 1 < p->num_layers ? 1 : 0, dev, s) != cudaSuccess)
-      return CLSA_ERR_CUDA;
+  if (launch_layers(*p, q_layers, out_layers, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
   return CLSA_OK;
 }
 

@@ -30,7 +30,7 @@ def _declared_functions():
 
 def test_every_declared_symbol_is_exported(clsa):
     names = _declared_functions()
-    assert len(names) == 11 and set(names) == set(clsa.EXPORTS)
+    assert len(names) == 12 and set(names) == set(clsa.EXPORTS)
     lib = ctypes.CDLL(clsa.LIB_PATH)
     for n in names:
         assert hasattr(lib, n), n
@@ -100,6 +100,9 @@ def test_bad_arguments_are_refused_on_the_host(clsa):
     outs = (ctypes.c_void_p * L)(0x80000, None)
     assert raw.clsa_decode_step(P(good), 0x50000, qs, outs, 0x60000, 0x70000, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
     assert raw.clsa_decode_step(P(good), 0x50000, None, outs, 0x60000, 0x70000, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_sparse_attn_layers(P(good), qs, 0x60000, 0x70000, outs, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG  # null out
+    assert raw.clsa_sparse_attn_layers(P(good), qs, None, 0x70000, qs, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_sparse_attn_layers(P(good), qs, 0x60000, 0x70000, qs, None, wsb, st) == clsa.CLSA_ERR_WORKSPACE
     # projections + append
     h, wq, wk, wkk, wv, qo = 0x90000, 0xA0000, 0xB0000, 0xC0000, 0xD0000, 0xE0000
     assert raw.clsa_project_append(P(good), 2560, None, wq, wk, wkk, wv, qo, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG

@@ -54,6 +54,13 @@ def _run_all(w, layers=None, check_lse=True):
     np.testing.assert_array_equal(g.count.cpu().numpy(), cnt_np)
     for l in range(g.L):
         assert torch.equal(outs[l].view(torch.int16), singles[l].view(torch.int16)), f"layer {l}: chain != separate call"
+    # the attention half of the chain on its own, fed the index that is already there
+    layer_outs = [g.new_out() for _ in range(g.L)]
+    clsa.clsa_sparse_attn_layers(g.params, [g.t["q_layers"][l] for l in range(g.L)], g.idx, g.count, layer_outs, g.ws)
+    torch.cuda.synchronize()
+    for l in range(g.L):
+        assert torch.equal(layer_outs[l].view(torch.int16), singles[l].view(torch.int16)), f"layer {l}: layers call"
+    np.testing.assert_array_equal(g.idx.cpu().numpy(), idx_np)  # the shared index is read, never written
     assert g.status() == 0
     return g, prob
 
