@@ -20,10 +20,17 @@
 // equal scores): two more full radix passes (12 + 8 bits) with the same cluster-wide histograms.
 //
 // Either way the exact threshold key and the number of threshold-equal keys still needed are
-// known, and the last sweep is an index-ordered compaction: a block's output offset is the number
-// of selected keys in lower-ranked blocks, a warp's offset the number selected in lower warps, so
-// positions come out ascending and, among keys equal to the threshold, the lowest positions win.
+// known, and a block's output offset is the number of selected keys in lower-ranked blocks. Common
+// case: the ballots of the second sweep (keys above the threshold's bin) were kept as a position
+// bitmap of the slice; the selected candidates add their bits, and a prefix count over the bitmap
+// words writes the positions in ascending order -- no third sweep over the keys. Rare case: an
+// index-ordered compaction sweep (a warp's offset is the number selected in lower warps). In both,
+// among keys equal to the threshold the lowest positions win.
 // No atomics touch global memory and nothing spins.
+//
+// Launches with thousands of rows (a prefill chunk) first go through the one-sweep kernel in
+// topk_filter.cu; this kernel then runs once more, one block per 16 rows, for the rows that kernel
+// marked as unfinished (count = -1).
 #include <cooperative_groups.h>
 
 #include "common.cuh"
