@@ -41,12 +41,12 @@ namespace clsa {
 namespace {
 
 // 1024 threads per block for latency hiding (the sweeps are chains of votes and shared-memory atomics), clusters
-// of at most 4: a block then fills an SM, and 33 clusters of 4 are resident at once on a B200, whereas only 15
-// clusters of 8 one-per-SM blocks fit its GPCs (16 rows would run in two waves).
+// of at most 4 (8 for launches of up to 8 rows): a block then fills an SM, and 33 clusters of 4 are resident at once on
+// a B200, whereas only 15 clusters of 8 one-per-SM blocks fit its GPCs (16 rows would run in two waves).
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxBins = 4096;
-constexpr int kMaxCluster = 4;
+constexpr int kMaxCluster = 8;       // 8 only for launches of at most 8 rows (see make_topk_plan)
 constexpr int kCandCap = 2048;  // candidates (row-wide) the short path handles
 
 struct alignas(16) Shared {  // the keys follow it in shared memory and are written 16 bytes at a time
@@ -605,11 +605,13 @@ TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev) {
   // One block per 32K visible scores, capped at kMaxCluster and rounded to a power of two; when there are few
   // rows, spread each over more blocks (down to 2K scores per block).
   int c = (p.max_seq_len + 32767) / 32768;
-  if (c > kMaxCluster) c = kMaxCluster;
+  if (c > 4) c = 4;
   int pow2 = 1;
   while (pow2 < c) pow2 <<= 1;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
-  while (pow2 < kMaxCluster && rows * pow2 * 2 <= dev.sm_count && p.max_seq_len / (pow2 * 2) >= 2048) pow2 <<= 1;
+  while (pow2 < 4 && rows * pow2 * 2 <= dev.sm_count && p.max_seq_len / (pow2 * 2) >= 2048) pow2 <<= 1;
+  // a handful of rows (small-batch decoding): clusters of 8, all of which are resident at once up to 8 rows
+  if (pow2 == 4 && rows <= 8 && p.max_seq_len / 8 >= 2048) pow2 = 8;
   // Many more rows than SMs (a prefill chunk): throughput matters, not the latency of one row. One block per
   // row needs no cluster barriers and keeps more rows in flight; its keys are re-read from global memory in
   // each of the three sweeps when they do not fit in shared memory.
