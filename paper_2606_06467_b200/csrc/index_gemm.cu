@@ -41,7 +41,7 @@ constexpr int kABytes = kBM * kBK * 2;          // one k-block of the query tile
 constexpr int kBBytes = kBN * kBK * 2;          // one k-block of the key tile (32 KiB)
 constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;  // up to two k-blocks each (96 KiB)
 constexpr int kBarrierBytes = 128;
-constexpr int kEpiTileBytes = kEpiWarps * 32 * 33 * 4;  // one padded 32 x 32 fp32 transposition tile per epilogue warp
+constexpr int kEpiTileBytes = kEpiWarps * 4096;  // one 32 x 32 fp32 tile (128-byte rows, 128-byte swizzle) per epilogue warp
 constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + kBarrierBytes + kEpiTileBytes + 1024;  // + alignment slack
 constexpr uint32_t kSpinLimit = 1u << 22;       // polls with back-off: a few seconds at most
 
@@ -53,7 +53,7 @@ struct GemmArgs {
   uint32_t* status;
   int num_seqs, q_per_seq, causal, max_seq_len, idx_dim;
   int m_blocks, n_tiles;
-  int vec_ok;  // rows of `scores` are 32-byte aligned: 256-bit stores allowed
+  int vec_ok;  // rows of `scores` are 32-byte aligned: 256-bit stores and tiled bulk stores allowed
   // paged key cache: a 256-key tile is fetched as key_boxes boxes of box_rows rows, one per cache block
   // (block_size < 256), or as one box inside a block (block_size >= 256). Contiguous: one box, no table.
   const int32_t* block_table;
@@ -153,18 +153,19 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmArgs& a, int64_t id) {
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const GemmArgs a) {
+index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                         const __grid_constant__ CUtensorMap map_s, const GemmArgs a) {
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t raw = smem_u32(smem_dyn);
   const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle wants 1024-byte aligned tiles
   unsigned char* base_ptr = smem_dyn + (base - raw);
-  const uint32_t bars = base + kStages * kStageBytes;
+  const uint32_t bars = base + kStages * kStageBytes + kEpiTileBytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 16u + 8u * s; };
   auto tfull_bar = [&](int i) { return bars + 32u + 8u * i; };
   auto tempty_bar = [&](int i) { return bars + 48u + 8u * i; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + 64);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + 68);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kEpiTileBytes + 64);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kEpiTileBytes + 68);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.idx_dim / kBK;  // 1 or 2
@@ -277,12 +278,34 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       // come, a warp instruction would scatter 32-byte pieces over 32 rows. They go through a padded
       // shared-memory tile instead and come back with four lanes per row, so that every store instruction writes
       // eight complete 128-byte lines.
-      float* tile = reinterpret_cast<float*>(base_ptr + kStages * kStageBytes + kBarrierBytes) + (warp - 4) * (32 * 33);
+      // The staging tile holds 32 rows x 128 bytes in the 128-byte-swizzle layout of the tensor maps: the 16-byte
+      // chunk c of row r sits at r * 128 + ((c ^ (r & 7)) << 4). Written a row per lane and read back four lanes per
+      // row, both without bank conflicts; a chunk that is visible to all 32 queries leaves as ONE tiled bulk store
+      // (the copy engine writes whole lines and the warp does not wait for them), the others -- on the causal
+      // diagonal, at the end of a sequence -- as masked 32-byte stores.
+      unsigned char* tile = base_ptr + kStages * kStageBytes + (warp - 4) * 4096;
+      const uint32_t tile_u32 = smem_u32(tile);
       const int t0 = c.mb * kBM + quad * 32;  // first query row of this warp
+      // every key below v_all is visible to all 32 rows (under the causal rule the first row sees the fewest)
+      const int v_all = (t0 + 31 < a.q_per_seq) ? (a.causal ? c.n - a.q_per_seq + t0 + 1 : c.n) : 0;
       auto store32 = [&](const uint32_t (&r)[32], int s0) {
-        __syncwarp();  // the previous chunk's reads of the tile are done
+        // the copy engine must have finished reading the tile's previous contents; so must the other lanes
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = __uint_as_float(r[j]);  // bank (lane + j) % 32: no conflicts
+        for (int ch = 0; ch < 8; ++ch)
+          *reinterpret_cast<uint4*>(tile + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
+              make_uint4(r[4 * ch], r[4 * ch + 1], r[4 * ch + 2], r[4 * ch + 3]);
+        if (a.vec_ok && s0 + 32 <= v_all) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the copy engine
+          __syncwarp();
+          if (lane == 0) {
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(&map_s), "r"(s0), "r"(c.b * a.q_per_seq + t0), "r"(tile_u32) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+          return;
+        }
         __syncwarp();
         const int s = s0 + (lane & 3) * 8;  // this lane's 8 columns
 #pragma unroll
@@ -291,10 +314,10 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
           const int tq = t0 + row;
           const int vr = tq < a.q_per_seq ? (a.causal ? c.n - a.q_per_seq + tq + 1 : c.n) : 0;
           if (s >= vr) continue;
-          const float* src = tile + row * 33 + (lane & 3) * 8;  // bank (row + 8 * (lane & 3) + e) % 32: no conflicts
-          float w[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) w[e] = src[e];
+          const int ch = (lane & 3) * 2;
+          const float4 w0 = *reinterpret_cast<const float4*>(tile + row * 128 + ((ch ^ (row & 7)) << 4));
+          const float4 w1 = *reinterpret_cast<const float4*>(tile + row * 128 + (((ch + 1) ^ (row & 7)) << 4));
+          const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
           float* dst = a.scores + ((int64_t)c.b * a.q_per_seq + tq) * a.score_stride + s;
           if (a.vec_ok && s + 8 <= vr) {
             asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "f"(w[0]), "f"(w[1]), "f"(w[2]),
@@ -329,6 +352,7 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       if (lane == 0) mbar_arrive(tempty_bar(acc));        // one arrival per epilogue warp frees the accumulator
       ++it;
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // this warp's bulk stores have landed
   }
 
   tc_fence_before();
@@ -377,6 +401,18 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 [rows][row_stride] (all row_stride columns addressable), box = 32 columns x 32 rows, 128-byte swizzle.
+bool make_map_f32(CUtensorMap* map, void* ptr, uint64_t rows, uint64_t row_stride) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {row_stride, rows};
+  const cuuint64_t strides[1] = {row_stride * 4};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
@@ -389,6 +425,11 @@ cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, fl
   if (!make_map(&map_k, p.idx_k_cache, (uint64_t)p.num_cache_rows, (uint64_t)p.idx_dim, (uint64_t)p.idx_token_stride,
                 (uint32_t)box_rows))
     return cudaErrorInvalidValue;
+  // fp32 scores [B*T][score_stride], box = 32 columns x 32 rows, for the epilogue's tiled bulk stores (only when the
+  // rows are 32-byte aligned; otherwise the map is a valid dummy over the key cache and is never used)
+  const bool vec_ok = score_stride % 8 == 0 && reinterpret_cast<uintptr_t>(scores) % 32 == 0;
+  CUtensorMap map_s = map_k;
+  if (vec_ok && !make_map_f32(&map_s, scores, q_rows, (uint64_t)score_stride)) return cudaErrorInvalidValue;
   GemmArgs a;
   a.block_table = p.block_table;
   a.block_size = paged ? p.block_size : 0;
@@ -407,12 +448,12 @@ cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, fl
   a.idx_dim = p.idx_dim;
   a.m_blocks = (p.q_per_seq + kBM - 1) / kBM;
   a.n_tiles = (p.max_seq_len + kBN - 1) / kBN;
-  a.vec_ok = (score_stride % 8 == 0 && reinterpret_cast<uintptr_t>(scores) % 32 == 0) ? 1 : 0;
+  a.vec_ok = vec_ok ? 1 : 0;
   cudaError_t err = cudaFuncSetAttribute(index_scores_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (err != cudaSuccess) return err;
   const int64_t tiles = (int64_t)p.num_seqs * a.m_blocks * a.n_tiles;
   const int grid = (int)(tiles < dev.sm_count ? tiles : dev.sm_count);
-  index_scores_gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, a);
+  index_scores_gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_s, a);
   return cudaGetLastError();
 }
 
