@@ -18,10 +18,10 @@
 //                      tcgen05.commit frees the smem stage and publishes the accumulator.
 //   warp 2           : allocates / frees the 512 TMEM columns.
 //   warps 4..11      : epilogue. Two warps per 32 TMEM lanes (= 32 query rows), 128 columns each: tcgen05.ld 32
-//                      columns at a time (double-buffered), a transposition through shared memory, then
-//                      32-byte vector stores, four lanes per row, of the visible part of each row (causal
-//                      limit per query): whole 128-byte lines per store instruction. The epilogue of tile i
-//                      overlaps the MMAs of tile i+1.
+//                      columns at a time (double-buffered) into a swizzled shared-memory tile; chunks that
+//                      every query of the warp may see leave as one tiled bulk store, the others (causal
+//                      diagonal, end of a sequence) as masked 32-byte stores, four lanes per row. The
+//                      epilogue of tile i overlaps the MMAs of tile i+1.
 // Tiles that lie entirely above the causal diagonal are skipped by every role alike.
 // Every mbarrier wait is bounded: on expiry the block raises CLSA_DEV_TIMEOUT in the status word,
 // all roles leave their loops, in-flight copies are given time to land, TMEM is freed, and the
