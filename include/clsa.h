@@ -80,6 +80,12 @@ typedef struct {
   float sm_scale;       /* softmax scale of Eq. 4's Attn; 1/sqrt(head_dim) in the benchmarks */
   int32_t sweep;        /* 0 or 1: direction in which clsa_sparse_attn walks the selected set; a cache-locality
                            hint only (results agree to rounding). clsa_decode_step uses (sweep + l) & 1 for layer l */
+  int32_t attn_plan;    /* launch shape of clsa_sparse_attn. 0: the whole GPU on this one launch (shortest time for a
+                           launch that has to finish before anything else can run -- a layer whose output feeds the
+                           next kernel). 1: a few large blocks per launch (about 32), for launches that run side by
+                           side with their neighbours on the stream, as the L layers of clsa_decode_step and
+                           clsa_sparse_attn_layers do (they always use 1, whatever this field says). Results of the
+                           two shapes agree to rounding (different split of the selected set), not bit for bit. */
   const int64_t* seq_start; /* [B] first cache row of each sequence */
   const int32_t* seq_len;   /* [B] valid tokens n_b >= T, including the T query tokens */
   const void* k_cache;      /* bf16 [rows][Hkv][D]; element (r,g,d) at r*kv_token_stride + g*kv_head_stride + d */
@@ -142,7 +148,9 @@ CLSA_API clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const
  *   q_layers   HOST array of L device pointers, each bf16 [B][T][Hq][D]
  *   out_layers HOST array of L device pointers, each bf16 [B][T][Hq][D]
  * Equivalent, bit for bit, to clsa_index_scores, clsa_topk and L calls of clsa_sparse_attn made one
- * after another with sweep = (p->sweep + l) & 1 for layer l. T > 1 is not chained here. */
+ * after another with sweep = (p->sweep + l) & 1 and attn_plan = 1 for layer l. The layers do not wait for one
+ * another (each reads only the index, the caches and its own queries), so several of them are in flight at once and
+ * find each other's rows in L2. T > 1 is not chained here. */
 CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
                              void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
                              size_t workspace_bytes, clsa_stream stream);
@@ -152,8 +160,8 @@ CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, c
  * arrive on another stream while the routing runs, making `stream` wait on that upload just before this call.
  *   q_layers / out_layers  HOST arrays of L device pointers, each bf16 [B][T][Hq][D], 16-byte aligned
  *   idx, count             as written by clsa_topk (read only)
- * Bit for bit the L calls of clsa_sparse_attn with sweep = (p->sweep + l) & 1 and lse = NULL, launched so that a
- * layer may start while its predecessor's last blocks finish (which is why the calls are offered as one). */
+ * Bit for bit the L calls of clsa_sparse_attn with sweep = (p->sweep + l) & 1, attn_plan = 1 and lse = NULL, launched
+ * so that a layer does not wait for its predecessor (which is why the calls are offered as one). */
 CLSA_API clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* const* q_layers, const int32_t* idx,
                                              const int32_t* count, void* const* out_layers, void* workspace,
                                              size_t workspace_bytes, clsa_stream stream);

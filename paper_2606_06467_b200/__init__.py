@@ -33,6 +33,7 @@ class clsa_params(ctypes.Structure):
         ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("idx_dim", ctypes.c_int32),
         ("top_k", ctypes.c_int32), ("num_layers", ctypes.c_int32), ("causal", ctypes.c_int32),
         ("max_seq_len", ctypes.c_int32), ("sm_scale", ctypes.c_float), ("sweep", ctypes.c_int32),
+        ("attn_plan", ctypes.c_int32),
         ("seq_start", ctypes.c_void_p), ("seq_len", ctypes.c_void_p),
         ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
         ("kv_token_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64),
@@ -104,7 +105,7 @@ def _nbytes(ws, ws_bytes):
 
 
 def make_params(*, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim=128, idx_dim, top_k, num_layers=1,
-                causal=0, max_seq_len, sm_scale, sweep=0, seq_start=None, seq_len=None, k_cache=None, v_cache=None,
+                causal=0, max_seq_len, sm_scale, sweep=0, attn_plan=0, seq_start=None, seq_len=None, k_cache=None, v_cache=None,
                 kv_token_stride=None, kv_head_stride=None, idx_k_cache=None, idx_token_stride=None,
                 num_cache_rows=None, block_table=None, block_size=0, max_blocks_per_seq=None) -> clsa_params:
     """Fill a clsa_params. Tensor arguments contribute their device address (and, for the caches, their strides
@@ -112,7 +113,7 @@ def make_params(*, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim=12
     p = clsa_params()
     p.num_seqs, p.q_per_seq, p.num_q_heads, p.num_kv_heads = num_seqs, q_per_seq, num_q_heads, num_kv_heads
     p.head_dim, p.idx_dim, p.top_k, p.num_layers, p.causal = head_dim, idx_dim, top_k, num_layers, causal
-    p.max_seq_len, p.sm_scale, p.sweep = max_seq_len, sm_scale, sweep
+    p.max_seq_len, p.sm_scale, p.sweep, p.attn_plan = max_seq_len, sm_scale, sweep, attn_plan
     p.seq_start, p.seq_len = _ptr(seq_start), _ptr(seq_len)
     p.k_cache, p.v_cache, p.idx_k_cache = _ptr(k_cache), _ptr(v_cache), _ptr(idx_k_cache)
     if kv_token_stride is None and k_cache is not None and not isinstance(k_cache, int):

@@ -54,6 +54,7 @@ clsa_status check_shape(const clsa_params* p) {
   if (p->num_q_heads % p->num_kv_heads != 0) return CLSA_ERR_INVALID_ARG;
   if (p->causal != 0 && p->causal != 1) return CLSA_ERR_INVALID_ARG;
   if (p->sweep != 0 && p->sweep != 1) return CLSA_ERR_INVALID_ARG;
+  if (p->attn_plan != 0 && p->attn_plan != 1) return CLSA_ERR_INVALID_ARG;
   if (p->max_seq_len < p->q_per_seq) return CLSA_ERR_INVALID_ARG;
   if (!isfinite(p->sm_scale)) return CLSA_ERR_INVALID_ARG;
   if ((int64_t)p->num_seqs * p->q_per_seq > (int64_t)1 << 30) return CLSA_ERR_INVALID_ARG;
@@ -111,7 +112,7 @@ cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, voi
                           const int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t s) {
   for (int l = 0; l < p.num_layers; ++l) {
     const cudaError_t err = launch_sparse_attn(p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p.sweep + l) & 1,
-                                               l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0, dev, s);
+                                               l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0, 1, dev, s);
     if (err != cudaSuccess) return err;
   }
   return cudaSuccess;
@@ -180,7 +181,8 @@ clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t*
   CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
-  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, 1, 0, dev,
+  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, 1, 0,
+                                      p->attn_plan, dev,
                                       static_cast<cudaStream_t>(stream)));
 }
 

@@ -31,7 +31,8 @@ struct AttnPlan {
   int head_groups;      // ceil(Hkv / HC): grid.y
   size_t smem_bytes;
 };
-AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev);
+// throughput != 0: a few large blocks (the launch shares the GPU with its neighbours on the stream)
+AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int throughput);
 
 struct TopkPlan {
   int cluster;      // blocks per (sequence, query) row, a thread-block cluster
@@ -61,7 +62,7 @@ cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int
                                   int* launched);
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
-                               const DeviceInfo& dev, cudaStream_t stream);
+                               int throughput_plan, const DeviceInfo& dev, cudaStream_t stream);
 
 cudaError_t launch_project_append(const clsa_params& p, int d_model, const void* h, const void* w_q_idx,
                                   const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,

@@ -481,38 +481,52 @@ static int max_resident_blocks(int cluster, size_t smem_bytes) {
 
 }  // namespace
 
-AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev) {
+AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int throughput) {
   AttnPlan plan;
   plan.smem_bytes = (size_t)kAttnWarps * kWarpRingBytes + kAttnWarps * kAttnStages * sizeof(uint32_t);
   const int hkv = p.num_kv_heads;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
-  // Heads per block: as few as it takes for all blocks to be resident at once (more blocks, and the
-  // split over tokens then stays inside a block); all 8 warps on different heads once there are
-  // more rows than SMs.
   int hc_max = 1;
   while (hc_max * 2 <= kAttnWarps && hc_max * 2 <= hkv) hc_max *= 2;
-  int hc = 1;
-  while (hc < hc_max && rows * ((hkv + hc - 1) / hc) > dev.sm_count) hc *= 2;
+  int hc, c = 1;
+  if (throughput) {
+    // The launch shares the GPU with the launches next to it on the stream (the layers of one step: each reads
+    // only the index, the caches and its own queries, so none waits for its predecessor). What counts then is the
+    // work per block, not how many SMs one launch covers: as many KV heads per block as leave about 32 blocks
+    // per launch, no clusters. Four or five layers are then in flight at once over the same selected rows, and
+    // find most of them in L2 (measured: 32 blocks per layer beat 16, 64 and 128 at every batch size tried).
+    hc = hc_max;
+    while (hc > 1 && rows * ((hkv + hc - 1) / hc) < 32) hc /= 2;
+  } else {
+    // Heads per block: as few as it takes for all blocks to be resident at once (more blocks, and the
+    // split over tokens then stays inside a block); all 8 warps on different heads once there are
+    // more rows than SMs.
+    hc = 1;
+    while (hc < hc_max && rows * ((hkv + hc - 1) / hc) > dev.sm_count) hc *= 2;
+  }
   // every token range should hold at least one 16-token stage
   while (hc < hc_max && (int64_t)(kAttnWarps / hc) * kAttnStageTokens > p.top_k) hc *= 2;
   plan.heads_per_block = hc;
   plan.subs = kAttnWarps / hc;
   plan.head_groups = (hkv + hc - 1) / hc;
-  // Cluster: the largest power of two that still keeps every block resident at once.
-  int c = 1;
-  const int64_t blocks = rows * plan.head_groups;
-  while (c < 8 && blocks * (c * 2) <= max_resident_blocks(c * 2, plan.smem_bytes) &&
-         (int64_t)(c * 2) * plan.subs * kAttnStageTokens <= p.top_k)
-    c *= 2;
+  if (throughput) {
+    // a handful of (row, KV head) pairs (batch of one): split each over a small cluster until there are 16 blocks
+    while (c < 8 && rows * plan.head_groups * c < 16 && (int64_t)(c * 2) * plan.subs * kAttnStageTokens <= p.top_k) c *= 2;
+  } else {
+    // Cluster: the largest power of two that still keeps every block resident at once.
+    const int64_t blocks = rows * plan.head_groups;
+    while (c < 8 && blocks * (c * 2) <= max_resident_blocks(c * 2, plan.smem_bytes) &&
+           (int64_t)(c * 2) * plan.subs * kAttnStageTokens <= p.top_k)
+      c *= 2;
+  }
   plan.cluster = c;
-  (void)dev;
   return plan;
 }
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
-                               const DeviceInfo& dev, cudaStream_t stream) {
-  const AttnPlan plan = make_attn_plan(p, dev);
+                               int throughput_plan, const DeviceInfo& dev, cudaStream_t stream) {
+  const AttnPlan plan = make_attn_plan(p, dev, throughput_plan);
   AttnArgs a;
   a.q = static_cast<const uint16_t*>(q);
   a.kc = static_cast<const uint16_t*>(p.k_cache);

@@ -69,14 +69,14 @@ class GpuProblem:
         clsa.clsa_topk(self.params, scores, scores.shape[-1], self.idx, self.count, self.ws)
         return self.idx, self.count
 
-    def sparse_attn(self, layer, idx=None, count=None, lse=True, sweep=0):
+    def sparse_attn(self, layer, idx=None, count=None, lse=True, sweep=0, plan=0):
         c = self.cfg
         out = self.new_out()
         l = torch.full((c.num_seqs, c.q_per_seq, c.num_q_heads), float("nan"), dtype=torch.float32, device=self.dev) if lse else None
-        self.params.sweep = sweep
+        self.params.sweep, self.params.attn_plan = sweep, plan
         clsa.clsa_sparse_attn(self.params, self.t["q_layers"][layer], self.idx if idx is None else idx,
                               self.count if count is None else count, out, l, self.ws)
-        self.params.sweep = 0
+        self.params.sweep, self.params.attn_plan = 0, 0
         return out, l
 
     def decode_step(self):
