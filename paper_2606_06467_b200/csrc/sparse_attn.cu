@@ -16,11 +16,14 @@
 // the cluster synchronises once, and the (KV head, query head) outputs are dealt round-robin to
 // the warps of the cluster, each reading the C * S partials it needs through distributed shared
 // memory and combining them by log-sum-exp. Nothing goes through global memory, nothing spins.
-// The launch shape is chosen per call so that all blocks are resident at once where possible:
-// HC shrinks (down to one KV head per block, its 8 warps splitting the tokens) until
-// rows * Hkv / HC fits the SM count, then C grows while the clusters still fit. Decoding a batch of
-// 16 with 8 KV heads runs 128 single-block clusters whose merge never leaves the block; a prefill
-// chunk runs one block per query row with nothing to merge.
+// Two launch shapes. A launch on its own (its output feeds the next kernel) gets the whole GPU: HC shrinks
+// (down to one KV head per block, its 8 warps splitting the tokens) until rows * Hkv / HC fits the SM
+// count, then C grows while all clusters stay resident at once. Decoding a batch of 16 with 8 KV heads
+// runs 128 single-block clusters whose merge never leaves the block; a prefill chunk runs one block per
+// query row with nothing to merge. The layers of one decode step, which do not wait for one another,
+// are launched side by side instead: about 32 large blocks per layer (as many KV heads per block as that
+// allows), so that four or five layers are in flight at once over the same selected rows and meet them
+// in L2.
 // `reverse` flips the order in which a warp walks its range; alternating it between consecutive
 // layers makes layer l+1 start on the rows layer l touched last, which are the ones still in L2.
 #include <cooperative_groups.h>
