@@ -1,7 +1,6 @@
 """Paged caches (block tables): the CUDA path on scattered blocks against the oracle on contiguous sequences.
 Paging changes addresses only, so scores, indices and outputs must agree exactly as in the contiguous case --
 and byte for byte with the CUDA path's own contiguous run."""
-import numpy as np
 import pytest
 
 torch = pytest.importorskip("torch")

@@ -14,7 +14,7 @@ entry._load_build_module().build()
 import oracle
 import paper_2606_06467_b200 as clsa
 from _harness import GpuProblem, check_attention, check_scores, check_topk_band, check_topk_exact_on_gpu_scores
-from workloads import MID, PREFILL, TINY, Workload
+from workloads import MID, TINY, Workload
 
 pytestmark = pytest.mark.gpu
 

@@ -8,7 +8,6 @@ through the C ABI twice in a row (the second call finds the first call's scores 
 and checks both results against the ordinary entry point; it also checks that a shape beyond the
 array's fixed capacity is refused before anything runs. This file sorts last on purpose.
 """
-import numpy as np
 import pytest
 
 torch = pytest.importorskip("torch")
