@@ -149,8 +149,8 @@ CLSA_API clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const
  *   out_layers HOST array of L device pointers, each bf16 [B][T][Hq][D]
  * Equivalent, bit for bit, to clsa_index_scores, clsa_topk and L calls of clsa_sparse_attn made one
  * after another with sweep = (p->sweep + l) & 1 and attn_plan = 1 for layer l. The layers do not wait for one
- * another (each reads only the index, the caches and its own queries), so several of them are in flight at once and
- * find each other's rows in L2. T > 1 is not chained here. */
+ * another (each reads only the index, the caches and its own queries), so several of them are in flight at once.
+ * T > 1 is not chained here. */
 CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
                              void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
                              size_t workspace_bytes, clsa_stream stream);

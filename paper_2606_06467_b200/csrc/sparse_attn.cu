@@ -22,8 +22,8 @@
 // runs 128 single-block clusters whose merge never leaves the block; a prefill chunk runs one block per
 // query row with nothing to merge. The layers of one decode step, which do not wait for one another,
 // are launched side by side instead: about 32 large blocks per layer (as many KV heads per block as that
-// allows), so that four or five layers are in flight at once over the same selected rows and meet them
-// in L2.
+// allows), so that four or five layers are in flight at once: every SM stays busy and the per-block
+// fixed costs are paid 32 instead of 128 times per layer.
 // `reverse` flips the order in which a warp walks its range; alternating it between consecutive
 // layers makes layer l+1 start on the rows layer l touched last, which are the ones still in L2.
 #include <cooperative_groups.h>
@@ -496,8 +496,8 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
     // The launch shares the GPU with the launches next to it on the stream (the layers of one step: each reads
     // only the index, the caches and its own queries, so none waits for its predecessor). What counts then is the
     // work per block, not how many SMs one launch covers: as many KV heads per block as leave about 32 blocks
-    // per launch, no clusters. Four or five layers are then in flight at once over the same selected rows, and
-    // find most of them in L2 (measured: 32 blocks per layer beat 16, 64 and 128 at every batch size tried).
+    // per launch, no clusters. Four or five layers are then in flight at once and keep every SM busy
+    // (measured: 32 blocks per layer beat 16, 64 and 128 at every batch size tried).
     hc = hc_max;
     while (hc > 1 && rows * ((hkv + hc - 1) / hc) < 32) hc /= 2;
   } else {
