@@ -94,8 +94,10 @@ typedef struct {
   int64_t kv_head_stride;   /* multiple of 8 */
   const void* idx_k_cache;  /* bf16 [rows][d_idx]; element (r,j) at r*idx_token_stride + j */
   int64_t idx_token_stride; /* multiple of 8 */
-  int64_t num_cache_rows;   /* rows of the cache row space (the extent of idx_k_cache); required when q_per_seq > 1,
-                               where tiled bulk copies need the bound; ignored (may be 0) when q_per_seq == 1 */
+  int64_t num_cache_rows;   /* rows of the cache row space (the extent of k_cache, v_cache and idx_k_cache); required when
+                               q_per_seq > 1, where tiled bulk copies need the bound. Optional (0 = unknown) otherwise; when
+                               given, clsa_sparse_attn computes row addresses in 32 bits where the caches allow it and treats
+                               a row at or beyond the extent like an index outside its sequence (skipped and flagged) */
   /* Paged caches (optional). With block_table == NULL sequence b occupies the contiguous rows starting at
    * seq_start[b]. Otherwise the row space is cut into blocks of block_size rows and position s of sequence b is
    * cache row  block_table[b * max_blocks_per_seq + s / block_size] * block_size + s % block_size  (the same

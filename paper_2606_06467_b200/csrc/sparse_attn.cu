@@ -63,6 +63,8 @@ struct AttnArgs {
   int q_per_seq, num_q_heads, num_kv_heads, group, top_k;
   int heads_per_block, subs, reverse;
   int wait_prior;  // 1: inputs may come from the kernel launched just before this one (wait for it first)
+  int off32;          // every row offset of the caches fits 32 bits when counted in 16-byte units
+  int64_t rows_max;   // extent of the cache row space (off32 only): rows at or beyond it are refused like bad indices
   int keep_permille;  // share of each warp's sweep (its end) whose rows are asked to stay in L2 for the next layer
   float scale_log2;
 };
@@ -237,27 +239,51 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
     const uint64_t pol_keep = l2_policy_evict_last();
     const uint64_t pol_stream = a.keep_permille > 0 ? l2_policy_evict_first() : l2_policy_evict_normal();
     const int keep_from = nstages - (nstages * a.keep_permille + 500) / 1000;  // steps >= keep_from are kept
+    // Per-lane constants of the copies: where in a stage buffer this lane's 16-byte chunk of token j = 2*it + lane/16
+    // goes (XOR swizzle), and the lane's byte offset inside a row.
+    uint32_t sw[8];
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      const int j = it * 2 + (lane >> 4);
+      sw[it] = (uint32_t)(j * 256 + (((lane & 15) ^ (j & 7)) << 4));
+    }
+    const char* kbytes = reinterpret_cast<const char*>(kbase);
+    const char* vbytes = reinterpret_cast<const char*>(vbase);
+    const uint32_t stride16 = (uint32_t)(a.tok_stride >> 3);  // row stride in 16-byte units (the stride is a multiple of 8)
     auto issue = [&](int i, int raw, int blk) {
       if (i < nstages) {
         const uint64_t pol = i >= keep_from ? pol_keep : pol_stream;
         const int buf = i % kAttnStages;
         const uint32_t kdst = ring_u32 + buf * kStageBytes, vdst = kdst + kStageBytes / 2;
-        const bool in_range = raw >= 0 && raw < n;
         // cache row relative to s0: the position itself, or its place inside its block
         const int my_idx = paged ? (blk << a.block_shift) + (raw & ((1 << a.block_shift) - 1)) : raw;
+        const bool in_range = raw >= 0 && raw < n && (!a.off32 || (uint64_t)(s0 + my_idx) < (uint64_t)a.rows_max);
         const uint32_t okmask = __ballot_sync(0xffffffffu, in_range) & 0xffffu;
         const bool bad = lane < kAttnStageTokens && !in_range && (stage_t0(i) + lane) < t_hi;
         if (bad) flag_status(a.status, CLSA_DEV_BAD_INDEX);
         if (lane == 0) stage_mask[buf] = okmask;
+        if (a.off32) {
+          // the whole cache spans fewer than 2^32 16-byte units: a row's offset is one 32-bit number, computed once
+          // by the lane that holds the position and widened with the base pointer in one multiply-add per copy
+          const uint32_t my_off16 = in_range ? ((uint32_t)s0 + (uint32_t)my_idx) * stride16 : 0u;
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int j = it * 2 + (lane >> 4);  // token of the stage this lane helps fetch
-          const int tok = __shfl_sync(0xffffffffu, my_idx, j);
-          const bool ok = (okmask >> j) & 1u;
-          const int64_t off = (s0 + (ok ? tok : 0)) * a.tok_stride;
-          const uint32_t sw = (uint32_t)(j * 256 + (((lane & 15) ^ (j & 7)) << 4));
-          cp_async16(kdst + sw, kbase + off, ok, pol);
-          cp_async16(vdst + sw, vbase + off, ok, pol);
+          for (int it = 0; it < 8; ++it) {
+            const int j = it * 2 + (lane >> 4);  // token of the stage this lane helps fetch
+            const uint32_t off16 = __shfl_sync(0xffffffffu, my_off16, j);
+            const bool ok = (okmask >> j) & 1u;
+            cp_async16(kdst + sw[it], kbytes + (uint64_t)off16 * 16u, ok, pol);
+            cp_async16(vdst + sw[it], vbytes + (uint64_t)off16 * 16u, ok, pol);
+          }
+        } else {
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int j = it * 2 + (lane >> 4);
+            const int tok = __shfl_sync(0xffffffffu, my_idx, j);
+            const bool ok = (okmask >> j) & 1u;
+            const int64_t off = (s0 + (ok ? tok : 0)) * a.tok_stride;
+            cp_async16(kdst + sw[it], kbase + off, ok, pol);
+            cp_async16(vdst + sw[it], vbase + off, ok, pol);
+          }
         }
       }
       cp_async_commit();
@@ -564,6 +590,9 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
     a.keep_permille = keep_for_next ? (int)(share * 1000.0) : 0;
   }
   a.scale_log2 = p.sm_scale * kLog2e;
+  // With the extent of the row space known (num_cache_rows) and below 2^32 16-byte units, row offsets are 32-bit.
+  a.rows_max = p.num_cache_rows;
+  a.off32 = (a.rows_max > 0 && (double)a.rows_max * (double)(p.kv_token_stride >> 3) < 4294967296.0) ? 1 : 0;
   auto kernel = a.group <= 8 ? (p.block_table ? sparse_attn_kernel<1, true> : sparse_attn_kernel<1, false>)
                              : (p.block_table ? sparse_attn_kernel<2, true> : sparse_attn_kernel<2, false>);
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
