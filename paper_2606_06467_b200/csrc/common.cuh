@@ -19,15 +19,17 @@ struct DeviceInfo {
 bool device_info(DeviceInfo* out);
 
 constexpr size_t kStatusBytes = 256;   // status word + padding at the start of the workspace
-constexpr int kAttnWarps = 8;          // warps per attention block, each an autonomous worker
+constexpr int kAttnWarpsNarrow = 12;    // warps per attention block (groups of up to 8 query heads per KV head), each an autonomous worker
+constexpr int kAttnWarpsWide = 8;      // the same for groups of 9..16 query heads (more registers per thread)
 constexpr int kAttnStageTokens = 16;   // tokens per pipeline stage (one PV MMA k-step)
-constexpr int kAttnStages = 3;         // cp.async ring depth per warp
+constexpr int kAttnStages = 2;         // cp.async ring depth per warp: one stage computed, one in flight
 
 // Launch shape of the sparse-attention kernel.
 struct AttnPlan {
+  int warps;            // warps per block: 12 (query-head groups up to 8) or 8
   int cluster;          // C: blocks per query row (a thread-block cluster), 1/2/4/8
-  int heads_per_block;  // HC = min(Hkv, 8): KV heads served by one block, one warp each
-  int subs;             // S = 8 / HC: token ranges per block
+  int heads_per_block;  // HC: KV heads served by one block (a power of two that divides the warps)
+  int subs;             // S = warps / HC: token ranges per block
   int head_groups;      // ceil(Hkv / HC): grid.y
   size_t smem_bytes;
 };

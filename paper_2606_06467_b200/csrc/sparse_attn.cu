@@ -37,8 +37,7 @@ namespace cg = cooperative_groups;
 namespace clsa {
 namespace {
 
-constexpr int kThreads = kAttnWarps * 32;
-static_assert(kAttnStages == 3, "the position pipeline in the kernel is written for a 3-deep ring");
+static_assert(kAttnStages == 2, "the position pipeline in the kernel is written for a 2-deep ring");
 constexpr int kStageBytes = kAttnStageTokens * 256 * 2;  // 16 K rows + 16 V rows of 256 bytes
 constexpr int kWarpRingBytes = kAttnStages * kStageBytes;
 constexpr int kPartialStride = 132;                      // floats per head of a partial: 128 outputs, max, sum, pad
@@ -122,8 +121,9 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
 }
 
 // NT = number of 8-head tiles that hold the query heads of one KV head (1 for groups up to 8, 2 up to 16).
-template <int NT, bool PAGED>
-__global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs a) {
+// WARPS = warps per block: 12 for NT = 1 (about 165 registers per thread), 8 for NT = 2.
+template <int NT, bool PAGED, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   cg::cluster_group cluster = cg::this_cluster();
   const int C = (int)cluster.num_blocks();
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
 
   unsigned char* ring = smem + warp * kWarpRingBytes;
   const uint32_t ring_u32 = smem_u32(ring);
-  uint32_t* stage_mask = reinterpret_cast<uint32_t*>(smem + kAttnWarps * kWarpRingBytes) + warp * kAttnStages;
+  uint32_t* stage_mask = reinterpret_cast<uint32_t*>(smem + WARPS * kWarpRingBytes) + warp * kAttnStages;
 
   // Fragment coordinates. The products are formed transposed, tokens along M:
   //   S^T[16 tokens x 8 heads] = K[16 x 128] Q^T,   O^T[128 x 8 heads] += V^T[128 x 16 tokens] P^T
@@ -169,14 +169,14 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   const int32_t* table = paged ? a.block_table + (int64_t)b * a.max_blocks : nullptr;
   const int n = a.seq_len[b];
   // Positions are fetched two pipeline steps before they are used and (paged caches) their block numbers one
-  // step before, so that no load is consumed in the step that issued it. The first four steps' positions are
+  // step before, so that no load is consumed in the step that issued it. The first three steps' positions are
   // fetched here, speculatively for a range that lies entirely below the row's count (entries past the count
   // are never used).
   const int nst_full = (slot_hi - slot_lo + kAttnStageTokens - 1) / kAttnStageTokens;
-  int spec_raw[4] = {-1, -1, -1, -1};
+  int spec_raw[3] = {-1, -1, -1};
   if (active && lane < kAttnStageTokens) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 3; ++i) {
       const int tt = slot_lo + (a.reverse ? nst_full - 1 - i : i) * kAttnStageTokens + lane;
       if (i < nst_full && tt < slot_hi) spec_raw[i] = row_idx[tt];
     }
@@ -289,19 +289,17 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
       cp_async_commit();
     };
 
-    // prologue: stages 0 and 1 in flight; positions of steps 2 and 3 (and step 2's block numbers) in registers
-    int r0 = spec_raw[0], r1 = spec_raw[1], rawA = spec_raw[2], rawB = spec_raw[3];
+    // prologue: stage 0 in flight; positions of steps 1 and 2 (and step 1's block numbers) in registers
+    int r0 = spec_raw[0], rawA = spec_raw[1], rawB = spec_raw[2];
     if (t_hi != slot_hi) {  // the count cuts this range short: fetch the real first positions
-      r0 = load_raw(0); r1 = load_raw(1); rawA = load_raw(2); rawB = load_raw(3);
+      r0 = load_raw(0); rawA = load_raw(1); rawB = load_raw(2);
     }
+    int blkA;
     {
-      const int b0 = load_blk(r0), b1 = load_blk(r1);
-      int blkA_init = load_blk(rawA);
+      const int b0 = load_blk(r0);
+      blkA = load_blk(rawA);
       issue(0, r0, b0);
-      issue(1, r1, b1);
-      r0 = blkA_init;  // reuse the register: block numbers of step 2
     }
-    int blkA = r0;
 #pragma unroll 1
     for (int i = 0; i < nstages; ++i) {
       {  // refill the buffer freed by step i-1, then advance the position pipeline
@@ -419,7 +417,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
   const int heads_here = min(HC, a.num_kv_heads - (int)blockIdx.y * HC);
   const int njobs = heads_here * G;
   const uint32_t smem_base = smem_u32(smem);
-  for (int job = crank + C * warp; job < njobs; job += C * kAttnWarps) {
+  for (int job = crank + C * warp; job < njobs; job += C * WARPS) {
     const int jg = job / G, hh = job - jg * G;   // local KV head, query head within the group
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f, M = -INFINITY;
@@ -483,17 +481,19 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_attn_kernel(const AttnArgs
 
 // Blocks of `cluster` that can be resident at once on the current device (cached per device and cluster size;
 // 0 if the query fails).
-static int max_resident_blocks(int cluster, size_t smem_bytes) {
+static int max_resident_blocks(int cluster, size_t smem_bytes, int warps) {
   static std::mutex mu;
-  static int cache[64][9] = {};
+  static int cache[64][9][2] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 0; }
+  const int which = warps == kAttnWarpsNarrow ? 0 : 1;
   std::lock_guard<std::mutex> lock(mu);
-  if (cache[dev][cluster] != 0) return cache[dev][cluster];
-  cudaFuncSetAttribute(sparse_attn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  if (cache[dev][cluster][which] != 0) return cache[dev][cluster][which];
+  auto kernel = which == 0 ? sparse_attn_kernel<1, false, kAttnWarpsNarrow> : sparse_attn_kernel<2, false, kAttnWarpsWide>;
+  cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)cluster * 64, 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.blockDim = dim3((unsigned)warps * 32, 1, 1);
   cfg.dynamicSmemBytes = smem_bytes;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -503,20 +503,25 @@ static int max_resident_blocks(int cluster, size_t smem_bytes) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, sparse_attn_kernel<1, false>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-  cache[dev][cluster] = n * cluster;
-  return cache[dev][cluster];
+  if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+  cache[dev][cluster][which] = n * cluster;
+  return cache[dev][cluster][which];
 }
 
 }  // namespace
 
 AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int throughput) {
   AttnPlan plan;
-  plan.smem_bytes = (size_t)kAttnWarps * kWarpRingBytes + kAttnWarps * kAttnStages * sizeof(uint32_t);
+  // 12 warps per block where the registers allow it (query-head groups up to 8: one 8-column tile per warp); the
+  // main loop is a dependent chain per warp, so warps per SM, not bytes in flight, set the pace once the rows come
+  // from L2.
+  plan.warps = p.num_q_heads / p.num_kv_heads <= 8 ? kAttnWarpsNarrow : kAttnWarpsWide;
+  plan.smem_bytes = (size_t)plan.warps * kWarpRingBytes + plan.warps * kAttnStages * sizeof(uint32_t);
   const int hkv = p.num_kv_heads;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
+  // heads per block: a power of two that divides the warps (1, 2, 4 of 12; 1, 2, 4, 8 of 8) and does not exceed Hkv
   int hc_max = 1;
-  while (hc_max * 2 <= kAttnWarps && hc_max * 2 <= hkv) hc_max *= 2;
+  while (hc_max * 2 <= hkv && plan.warps % (hc_max * 2) == 0) hc_max *= 2;
   int hc, c = 1;
   if (throughput) {
     // The launch shares the GPU with the launches next to it on the stream (the layers of one step: each reads
@@ -528,15 +533,14 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
     while (hc > 1 && rows * ((hkv + hc - 1) / hc) < 32) hc /= 2;
   } else {
     // Heads per block: as few as it takes for all blocks to be resident at once (more blocks, and the
-    // split over tokens then stays inside a block); all 8 warps on different heads once there are
-    // more rows than SMs.
+    // split over tokens then stays inside a block); as many as possible once there are more rows than SMs.
     hc = 1;
     while (hc < hc_max && rows * ((hkv + hc - 1) / hc) > dev.sm_count) hc *= 2;
   }
   // every token range should hold at least one 16-token stage
-  while (hc < hc_max && (int64_t)(kAttnWarps / hc) * kAttnStageTokens > p.top_k) hc *= 2;
+  while (hc < hc_max && (int64_t)(plan.warps / hc) * kAttnStageTokens > p.top_k) hc *= 2;
   plan.heads_per_block = hc;
-  plan.subs = kAttnWarps / hc;
+  plan.subs = plan.warps / hc;
   plan.head_groups = (hkv + hc - 1) / hc;
   if (throughput) {
     // a handful of (row, KV head) pairs (batch of one): split each over a small cluster until there are 16 blocks
@@ -544,7 +548,7 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   } else {
     // Cluster: the largest power of two that still keeps every block resident at once.
     const int64_t blocks = rows * plan.head_groups;
-    while (c < 8 && blocks * (c * 2) <= max_resident_blocks(c * 2, plan.smem_bytes) &&
+    while (c < 8 && blocks * (c * 2) <= max_resident_blocks(c * 2, plan.smem_bytes, plan.warps) &&
            (int64_t)(c * 2) * plan.subs * kAttnStageTokens <= p.top_k)
       c *= 2;
   }
@@ -593,14 +597,14 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   // With the extent of the row space known (num_cache_rows) and below 2^32 16-byte units, row offsets are 32-bit.
   a.rows_max = p.num_cache_rows;
   a.off32 = (a.rows_max > 0 && (double)a.rows_max * (double)(p.kv_token_stride >> 3) < 4294967296.0) ? 1 : 0;
-  auto kernel = a.group <= 8 ? (p.block_table ? sparse_attn_kernel<1, true> : sparse_attn_kernel<1, false>)
-                             : (p.block_table ? sparse_attn_kernel<2, true> : sparse_attn_kernel<2, false>);
+  auto kernel = a.group <= 8 ? (p.block_table ? sparse_attn_kernel<1, true, kAttnWarpsNarrow> : sparse_attn_kernel<1, false, kAttnWarpsNarrow>)
+                             : (p.block_table ? sparse_attn_kernel<2, true, kAttnWarpsWide> : sparse_attn_kernel<2, false, kAttnWarpsWide>);
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(rows * plan.cluster), (unsigned)plan.head_groups, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.blockDim = dim3((unsigned)plan.warps * 32, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
