@@ -77,7 +77,7 @@ typedef struct {
   int32_t num_layers;   /* L >= 1; read by clsa_decode_step and clsa_workspace_bytes only */
   int32_t causal;       /* 0 or 1, see "Visibility" */
   int32_t max_seq_len;  /* host-known upper bound of seq_len[], used for grid sizing (no device read-back) */
-  float sm_scale;       /* softmax scale of Eq. 4's Attn; 1/sqrt(head_dim) in the benchmarks */
+  float sm_scale;       /* softmax scale of Eq. 4's Attn, > 0; 1/sqrt(head_dim) in the benchmarks */
   int32_t sweep;        /* 0 or 1: direction in which clsa_sparse_attn walks the selected set; a cache-locality
                            hint only (results agree to rounding). clsa_decode_step uses (sweep + l) & 1 for layer l */
   int32_t attn_plan;    /* launch shape of clsa_sparse_attn. 0: the whole GPU on this one launch (shortest time for a

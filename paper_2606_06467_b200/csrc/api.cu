@@ -56,7 +56,7 @@ clsa_status check_shape(const clsa_params* p) {
   if (p->sweep != 0 && p->sweep != 1) return CLSA_ERR_INVALID_ARG;
   if (p->attn_plan != 0 && p->attn_plan != 1) return CLSA_ERR_INVALID_ARG;
   if (p->max_seq_len < p->q_per_seq) return CLSA_ERR_INVALID_ARG;
-  if (!isfinite(p->sm_scale)) return CLSA_ERR_INVALID_ARG;
+  if (!isfinite(p->sm_scale) || !(p->sm_scale > 0.f)) return CLSA_ERR_INVALID_ARG;  // the kernels take maxima before scaling
   if ((int64_t)p->num_seqs * p->q_per_seq > (int64_t)1 << 30) return CLSA_ERR_INVALID_ARG;
   if (p->head_dim != 128) return CLSA_ERR_UNSUPPORTED;
   if (p->idx_dim != 64 && p->idx_dim != 128) return CLSA_ERR_UNSUPPORTED;

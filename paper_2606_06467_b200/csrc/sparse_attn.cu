@@ -74,6 +74,10 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool v
   asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;\n"
                ::"r"(dst), "l"(src), "r"(bytes), "l"(policy) : "memory");
 }
+// The same without the source-size operand (the whole 16 bytes are copied).
+__device__ __forceinline__ void cp_async16_full(uint32_t dst, const void* src, uint64_t policy) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "l"(policy) : "memory");
+}
 __device__ __forceinline__ uint64_t l2_policy_evict_last() {
   uint64_t p;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
@@ -189,9 +193,12 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
 
   float o[NT][8][4];                   // O^T: [head tile][16-wide slice of D][c0..c3]
   float mA[NT], mB[NT], lA[NT], lB[NT];  // running max / sum of heads hcol and hcol+1 (log2 domain)
+  float lacc[NT][4];                   // the sums as an MMA accumulator: ones[16 x 16] . P^T puts a head's sum over the stage's
+                                       // 16 tokens in every row of its column (c0: head hcol, c1: head hcol + 1)
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     mA[nt] = -INFINITY; mB[nt] = -INFINITY; lA[nt] = 0.f; lB[nt] = 0.f;
+    lacc[nt][0] = 0.f; lacc[nt][1] = 0.f; lacc[nt][2] = 0.f; lacc[nt][3] = 0.f;
 #pragma unroll
     for (int j = 0; j < 8; ++j) { o[nt][j][0] = 0.f; o[nt][j][1] = 0.f; o[nt][j][2] = 0.f; o[nt][j][3] = 0.f; }
   }
@@ -266,13 +273,22 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
           // the whole cache spans fewer than 2^32 16-byte units: a row's offset is one 32-bit number, computed once
           // by the lane that holds the position and widened with the base pointer in one multiply-add per copy
           const uint32_t my_off16 = in_range ? ((uint32_t)s0 + (uint32_t)my_idx) * stride16 : 0u;
+          if (okmask == 0xffffu) {  // the usual stage: all 16 positions valid, plain copies
 #pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int j = it * 2 + (lane >> 4);  // token of the stage this lane helps fetch
-            const uint32_t off16 = __shfl_sync(0xffffffffu, my_off16, j);
-            const bool ok = (okmask >> j) & 1u;
-            cp_async16(kdst + sw[it], kbytes + (uint64_t)off16 * 16u, ok, pol);
-            cp_async16(vdst + sw[it], vbytes + (uint64_t)off16 * 16u, ok, pol);
+            for (int it = 0; it < 8; ++it) {
+              const uint32_t off16 = __shfl_sync(0xffffffffu, my_off16, it * 2 + (lane >> 4));
+              cp_async16_full(kdst + sw[it], kbytes + (uint64_t)off16 * 16u, pol);
+              cp_async16_full(vdst + sw[it], vbytes + (uint64_t)off16 * 16u, pol);
+            }
+          } else {
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+              const int j = it * 2 + (lane >> 4);  // token of the stage this lane helps fetch
+              const uint32_t off16 = __shfl_sync(0xffffffffu, my_off16, j);
+              const bool ok = (okmask >> j) & 1u;
+              cp_async16(kdst + sw[it], kbytes + (uint64_t)off16 * 16u, ok, pol);
+              cp_async16(vdst + sw[it], vbytes + (uint64_t)off16 * 16u, ok, pol);
+            }
           }
         } else {
 #pragma unroll
@@ -328,46 +344,54 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) mma_bf16(s[nt], kf, qb[nt][ks][0], qb[nt][ks][1]);
       }
-      // online softmax over tokens (rows), per head (columns), exp2 domain; masked tokens get -inf
+      // online softmax over tokens (rows), per head (columns), exp2 domain; masked tokens get -inf. The maxima are
+      // taken over the raw dot products (the scale is positive) and the scale rides in the multiply-add of the exponent.
+      const bool full = okmask == 0xffffu;  // the usual stage: nothing to mask
       const bool ok_lo = (okmask >> rowq) & 1u, ok_hi = (okmask >> (rowq + 8)) & 1u;
       uint32_t pb0[NT], pb1[NT];
       bool rescale = false;
       float alphaA[NT], alphaB[NT];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        const float s0v = ok_lo ? s[nt][0] * a.scale_log2 : -INFINITY;   // token rowq,   head hcol
-        const float s1v = ok_lo ? s[nt][1] * a.scale_log2 : -INFINITY;   // token rowq,   head hcol+1
-        const float s2v = ok_hi ? s[nt][2] * a.scale_log2 : -INFINITY;   // token rowq+8, head hcol
-        const float s3v = ok_hi ? s[nt][3] * a.scale_log2 : -INFINITY;   // token rowq+8, head hcol+1
-        float mxA = fmaxf(s0v, s2v), mxB = fmaxf(s1v, s3v);
+        float r0 = s[nt][0], r1 = s[nt][1], r2 = s[nt][2], r3 = s[nt][3];  // tokens rowq (r0, r1) and rowq + 8; heads hcol, hcol + 1
+        if (!full) {
+          r0 = ok_lo ? r0 : -INFINITY; r1 = ok_lo ? r1 : -INFINITY;
+          r2 = ok_hi ? r2 : -INFINITY; r3 = ok_hi ? r3 : -INFINITY;
+        }
+        float mxA = fmaxf(r0, r2), mxB = fmaxf(r1, r3);
 #pragma unroll
         for (int d = 4; d <= 16; d <<= 1) {
           mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, d));
           mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, d));
         }
-        const float mnA = fmaxf(mA[nt], mxA), mnB = fmaxf(mB[nt], mxB);
+        const float mnA = fmaxf(mA[nt], mxA * a.scale_log2), mnB = fmaxf(mB[nt], mxB * a.scale_log2);
         const float muA = mnA == -INFINITY ? 0.f : mnA, muB = mnB == -INFINITY ? 0.f : mnB;
         alphaA[nt] = fast_exp2(mA[nt] - muA);
         alphaB[nt] = fast_exp2(mB[nt] - muB);
         rescale = rescale || mnA != mA[nt] || mnB != mB[nt];
         mA[nt] = mnA;
         mB[nt] = mnB;
-        const uint32_t p_lo = pack_bf16x2(fast_exp2(s0v - muA), fast_exp2(s1v - muB));  // token rowq
-        const uint32_t p_hi = pack_bf16x2(fast_exp2(s2v - muA), fast_exp2(s3v - muB));  // token rowq + 8
-        // the denominators use the same bf16-rounded weights as the numerators
-        lA[nt] = lA[nt] * alphaA[nt] + (bf16_lo(p_lo) + bf16_lo(p_hi));
-        lB[nt] = lB[nt] * alphaB[nt] + (bf16_hi(p_lo) + bf16_hi(p_hi));
+        const uint32_t p_lo = pack_bf16x2(fast_exp2(fmaf(r0, a.scale_log2, -muA)), fast_exp2(fmaf(r1, a.scale_log2, -muB)));
+        const uint32_t p_hi = pack_bf16x2(fast_exp2(fmaf(r2, a.scale_log2, -muA)), fast_exp2(fmaf(r3, a.scale_log2, -muB)));
         // P is held [token][head]; the PV product wants P^T as its B operand: transpose the two 8x8 halves
         pb0[nt] = movmatrix_trans(p_lo);
         pb1[nt] = movmatrix_trans(p_hi);
       }
       if (__any_sync(0xffffffffu, rescale)) {  // the running max moved for some head: rescale the accumulators
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             o[nt][j][0] *= alphaA[nt]; o[nt][j][1] *= alphaB[nt]; o[nt][j][2] *= alphaA[nt]; o[nt][j][3] *= alphaB[nt];
           }
+          lacc[nt][0] *= alphaA[nt]; lacc[nt][1] *= alphaB[nt]; lacc[nt][2] *= alphaA[nt]; lacc[nt][3] *= alphaB[nt];
+        }
+      }
+      // the denominators: the same bf16-rounded weights as the numerators, summed over the stage's tokens by one MMA
+      {
+        const uint32_t ones[4] = {0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u};
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(lacc[nt], ones, pb0[nt], pb1[nt]);
       }
       // O^T += V^T P^T: A = V^T (transposing ldmatrix of the [token][d] tile), 8 slices of 16 output dimensions
 #pragma unroll
@@ -383,12 +407,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
     cp_async_wait<0>();
 
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int d = 4; d <= 16; d <<= 1) {
-        lA[nt] += __shfl_xor_sync(0xffffffffu, lA[nt], d);
-        lB[nt] += __shfl_xor_sync(0xffffffffu, lB[nt], d);
-      }
+    for (int nt = 0; nt < NT; ++nt) { lA[nt] = lacc[nt][0]; lB[nt] = lacc[nt][1]; }
   }
 
   // ---- split-K merge through (distributed) shared memory --------------------------------------------
