@@ -332,17 +332,25 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
       const uint32_t kbuf = ring_u32 + buf * kStageBytes, vbuf = kbuf + kStageBytes / 2;
       const uint32_t okmask = stage_mask[buf];
 
-      // S^T = K Q^T for 16 tokens: A = K rows (tokens) from shared memory, B = Q^T from registers
-      float s[NT][4];
+      // S^T = K Q^T for 16 tokens: A = K rows (tokens) from shared memory, B = Q^T from registers. Two accumulators
+      // (even and odd 16-wide slices of D) halve the chain of dependent MMAs.
+      float s[NT][4], s_odd[NT][4];
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) { s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f; }
+      for (int nt = 0; nt < NT; ++nt) {
+        s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f;
+        s_odd[nt][0] = 0.f; s_odd[nt][1] = 0.f; s_odd[nt][2] = 0.f; s_odd[nt][3] = 0.f;
+      }
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const int tok = (lane & 7) + 8 * ((lane >> 3) & 1), chunk = 2 * ks + (lane >> 4);
         uint32_t kf[4];
         ldmatrix_x4(kf, kbuf + tok * 256 + ((chunk ^ (tok & 7)) << 4));
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) mma_bf16(s[nt], kf, qb[nt][ks][0], qb[nt][ks][1]);
+        for (int nt = 0; nt < NT; ++nt) mma_bf16((ks & 1) ? s_odd[nt] : s[nt], kf, qb[nt][ks][0], qb[nt][ks][1]);
+      }
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        s[nt][0] += s_odd[nt][0]; s[nt][1] += s_odd[nt][1]; s[nt][2] += s_odd[nt][2]; s[nt][3] += s_odd[nt][3];
       }
       // online softmax over tokens (rows), per head (columns), exp2 domain; masked tokens get -inf. The maxima are
       // taken over the raw dot products (the scale is positive) and the scale rides in the multiply-add of the exponent.
