@@ -6,10 +6,10 @@
 // packed into the 8 columns of one tile -- far below tensor-pipe capacity.
 //
 // Decomposition. One thread-block cluster of C blocks serves one query row (sequence, query
-// token); its selected tokens are cut into C * S contiguous ranges. A block has 8 autonomous
-// warps: warp w serves KV head w % HC of token range w / HC (HC heads per block, S = 8 / HC
-// ranges per block). A warp streams
-// its range in 16-token stages through a private 3-deep cp.async ring (16-byte chunks,
+// token); its selected tokens are cut into C * S contiguous ranges. A block has 12 autonomous
+// warps (8 for query-head groups above 8): warp w serves KV head w % HC of token range w / HC (HC
+// heads per block, S = warps / HC ranges per block). A warp streams
+// its range in 16-token stages through a private 2-deep cp.async ring (16-byte chunks,
 // XOR-swizzled for conflict-free ldmatrix), runs S = Q K^T, an online softmax in the exp2 domain
 // and O += P V per stage; there is no block-level barrier in the main loop. Split-K merge: every
 // warp leaves its unnormalised partial (O, running max, running sum) in its own shared memory,
@@ -17,7 +17,7 @@
 // the warps of the cluster, each reading the C * S partials it needs through distributed shared
 // memory and combining them by log-sum-exp. Nothing goes through global memory, nothing spins.
 // Two launch shapes. A launch on its own (its output feeds the next kernel) gets the whole GPU: HC shrinks
-// (down to one KV head per block, its 8 warps splitting the tokens) until rows * Hkv / HC fits the SM
+// (down to one KV head per block, its warps splitting the tokens) until rows * Hkv / HC fits the SM
 // count, then C grows while all clusters stay resident at once. Decoding a batch of 16 with 8 KV heads
 // runs 128 single-block clusters whose merge never leaves the block; a prefill chunk runs one block per
 // query row with nothing to merge. The layers of one decode step, which do not wait for one another,
