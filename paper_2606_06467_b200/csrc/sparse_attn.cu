@@ -543,6 +543,12 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   // main loop is a dependent chain per warp, so warps per SM, not bytes in flight, set the pace once the rows come
   // from L2.
   plan.warps = p.num_q_heads / p.num_kv_heads <= 8 ? kAttnWarpsNarrow : kAttnWarpsWide;
+  const int64_t rows_ = (int64_t)p.num_seqs * p.q_per_seq;
+  // Side by side, 32 to 63 rows of 8 or more KV heads: 8 warps can take all 8 heads of a row (32 to 63 blocks per
+  // launch, the shape that works best), which 12 warps cannot (4 heads per block, twice the blocks). Measured at
+  // 32 rows: 631 against 736 us per step.
+  if (throughput && p.num_kv_heads >= 8 && rows_ * ((p.num_kv_heads + 7) / 8) >= 32 && rows_ * ((p.num_kv_heads + 7) / 8) < 64)
+    plan.warps = kAttnWarpsWide;
   plan.smem_bytes = (size_t)plan.warps * kWarpRingBytes + plan.warps * kAttnStages * sizeof(uint32_t);
   const int hkv = p.num_kv_heads;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
@@ -624,8 +630,13 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   // With the extent of the row space known (num_cache_rows) and below 2^32 16-byte units, row offsets are 32-bit.
   a.rows_max = p.num_cache_rows;
   a.off32 = (a.rows_max > 0 && (double)a.rows_max * (double)(p.kv_token_stride >> 3) < 4294967296.0) ? 1 : 0;
-  auto kernel = a.group <= 8 ? (p.block_table ? sparse_attn_kernel<1, true, kAttnWarpsNarrow> : sparse_attn_kernel<1, false, kAttnWarpsNarrow>)
-                             : (p.block_table ? sparse_attn_kernel<2, true, kAttnWarpsWide> : sparse_attn_kernel<2, false, kAttnWarpsWide>);
+  void (*kernel)(const AttnArgs);
+  if (a.group > 8)
+    kernel = p.block_table ? sparse_attn_kernel<2, true, kAttnWarpsWide> : sparse_attn_kernel<2, false, kAttnWarpsWide>;
+  else if (plan.warps == kAttnWarpsNarrow)
+    kernel = p.block_table ? sparse_attn_kernel<1, true, kAttnWarpsNarrow> : sparse_attn_kernel<1, false, kAttnWarpsNarrow>;
+  else
+    kernel = p.block_table ? sparse_attn_kernel<1, true, kAttnWarpsWide> : sparse_attn_kernel<1, false, kAttnWarpsWide>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
