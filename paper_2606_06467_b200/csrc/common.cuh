@@ -29,7 +29,8 @@ struct AttnPlan {
   int warps;            // warps per block: 12 (query-head groups up to 8) or 8
   int cluster;          // C: blocks per query row (a thread-block cluster), 1/2/4/8
   int heads_per_block;  // HC: KV heads served by one block (a power of two that divides the warps)
-  int subs;             // S = warps / HC: token ranges per block
+  int rows_per_block;   // RB: query rows served by one block (1 unless a chunk launch has short per-warp ranges)
+  int subs;             // S = warps / HC / RB: token ranges of one row per block
   int head_groups;      // ceil(Hkv / HC): grid.y
   size_t smem_bytes;
 };

@@ -19,8 +19,8 @@
 // Two launch shapes. A launch on its own (its output feeds the next kernel) gets the whole GPU: HC shrinks
 // (down to one KV head per block, its warps splitting the tokens) until rows * Hkv / HC fits the SM
 // count, then C grows while all clusters stay resident at once. Decoding a batch of 16 with 8 KV heads
-// runs 128 single-block clusters whose merge never leaves the block; a prefill chunk runs one block per
-// query row with nothing to merge. The layers of one decode step, which do not wait for one another,
+// runs 128 single-block clusters whose merge never leaves the block; a launch with far more rows than SMs
+// (a prefill chunk) puts several rows in a block, up to one warp per (row, KV head) with nothing to merge. The layers of one decode step, which do not wait for one another,
 // are launched side by side instead: about 32 large blocks per layer (as many KV heads per block as that
 // allows), so that four or five layers are in flight at once: every SM stays busy and the per-block
 // fixed costs are paid 32 instead of 128 times per layer.
@@ -60,7 +60,8 @@ struct AttnArgs {
   float* lse;
   uint32_t* status;
   int q_per_seq, num_q_heads, num_kv_heads, group, top_k;
-  int heads_per_block, subs, reverse;
+  int heads_per_block, subs, rows_per_block, reverse;
+  int64_t num_rows;
   int wait_prior;  // 1: inputs may come from the kernel launched just before this one (wait for it first)
   int off32;          // every row offset of the caches fits 32 bits when counted in 16-byte units
   int64_t rows_max;   // extent of the cache row space (off32 only): rows at or beyond it are refused like bad indices
@@ -126,18 +127,24 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
 
 // NT = number of 8-head tiles that hold the query heads of one KV head (1 for groups up to 8, 2 up to 16).
 // WARPS = warps per block: 12 for NT = 1 (about 165 registers per thread), 8 for NT = 2.
-template <int NT, bool PAGED, int WARPS>
+// MULTI: a block serves several query rows (rows_per_block > 1); the single-row instances keep the row uniform
+// over the block.
+template <int NT, bool PAGED, int WARPS, bool MULTI>
 __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   cg::cluster_group cluster = cg::this_cluster();
   const int C = (int)cluster.num_blocks();
   const int crank = (int)cluster.block_rank();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t r = blockIdx.x / C;                 // query row
   const int HC = a.heads_per_block, S = a.subs, G = a.group;
-  const int g_local = warp % HC, sub = warp / HC;
+  const int g_local = warp % HC;
+  const int RB = MULTI ? a.rows_per_block : 1;
+  const int row_local = MULTI ? (warp / HC) / S : 0;  // which of the block's rows
+  const int sub = (warp / HC) - row_local * S;       // which of that row's token ranges
+  const int64_t r_true = (int64_t)(blockIdx.x / C) * RB + row_local;
   const int g = blockIdx.y * HC + g_local;          // KV head of this warp
-  const bool active = sub < S && g < a.num_kv_heads;
+  const bool active = sub < S && row_local < RB && r_true < a.num_rows && g < a.num_kv_heads;
+  const int64_t r = (!MULTI || r_true < a.num_rows) ? r_true : a.num_rows - 1;  // query row (clamped past the last row)
   const int nsplit = C * S;                         // token ranges of the row
 
   unsigned char* ring = smem + warp * kWarpRingBytes;
@@ -186,7 +193,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
     }
   }
   if (cnt < 0 || cnt > a.top_k) {
-    if (threadIdx.x == 0 && crank == 0 && blockIdx.y == 0) flag_status(a.status, CLSA_DEV_BAD_COUNT);
+    if (lane == 0 && sub == 0 && g_local == 0 && crank == 0 && blockIdx.y == 0 && active) flag_status(a.status, CLSA_DEV_BAD_COUNT);
     cnt = cnt < 0 ? 0 : a.top_k;
   }
   const int t_lo = min(cnt, slot_lo), t_hi = active ? min(cnt, slot_hi) : t_lo;
@@ -442,13 +449,18 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
 
   // Output jobs (KV head of this block's group, query head of the group) dealt over the cluster's warps.
   const int heads_here = min(HC, a.num_kv_heads - (int)blockIdx.y * HC);
-  const int njobs = heads_here * G;
+  const int jobs_per_row = heads_here * G;
+  const int njobs = RB * jobs_per_row;
   const uint32_t smem_base = smem_u32(smem);
   for (int job = crank + C * warp; job < njobs; job += C * WARPS) {
-    const int jg = job / G, hh = job - jg * G;   // local KV head, query head within the group
+    const int rl = MULTI ? job / jobs_per_row : 0;  // which of the block's rows
+    const int64_t r_job = (int64_t)(blockIdx.x / C) * RB + rl;
+    if (MULTI && r_job >= a.num_rows) continue;
+    const int jrow = job - rl * jobs_per_row;
+    const int jg = jrow / G, hh = jrow - jg * G;   // local KV head, query head within the group
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f, M = -INFINITY;
-    // Partial p = (block p / S, range p % S) was left by warp (p % S) * HC + jg of block p / S. Lane p of each
+    // Partial p = (block p / S, range p % S) of row rl was left by warp (rl * S + p % S) * HC + jg of block p / S. Lane p of each
     // 32-partial chunk resolves that partial's shared::cluster address once; everyone then reads through it.
     for (int p0 = 0; p0 < nsplit; p0 += 32) {
       const int p = p0 + lane;
@@ -456,7 +468,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
       float2 ml = make_float2(-INFINITY, 0.f);
       if (p < nsplit) {
         const int c2 = p / S, sub2 = p - c2 * S;
-        const uint32_t local = smem_base + (uint32_t)((sub2 * HC + jg) * kWarpRingBytes + hh * kPartialStride * 4);
+        const uint32_t local = smem_base + (uint32_t)(((rl * S + sub2) * HC + jg) * kWarpRingBytes + hh * kPartialStride * 4);
         asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(src) : "r"(local), "r"(c2));
         asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(ml.x), "=f"(ml.y) : "r"(src + 512u) : "memory");
       }
@@ -496,7 +508,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
       }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
-    const int64_t item = r * a.num_q_heads + (int64_t)(blockIdx.y * HC + jg) * G + hh;
+    const int64_t item = r_job * a.num_q_heads + (int64_t)(blockIdx.y * HC + jg) * G + hh;
     uint2 packed;
     packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
     packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
@@ -516,7 +528,7 @@ static int max_resident_blocks(int cluster, size_t smem_bytes, int warps) {
   const int which = warps == kAttnWarpsNarrow ? 0 : 1;
   std::lock_guard<std::mutex> lock(mu);
   if (cache[dev][cluster][which] != 0) return cache[dev][cluster][which];
-  auto kernel = which == 0 ? sparse_attn_kernel<1, false, kAttnWarpsNarrow> : sparse_attn_kernel<2, false, kAttnWarpsWide>;
+  auto kernel = which == 0 ? sparse_attn_kernel<1, false, kAttnWarpsNarrow, false> : sparse_attn_kernel<2, false, kAttnWarpsWide, false>;
   cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)cluster * 64, 1, 1);
@@ -578,15 +590,30 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   // every token range should hold at least one 16-token stage
   while (hc < hc_max && (int64_t)(plan.warps / hc) * kAttnStageTokens > p.top_k) hc *= 2;
   plan.heads_per_block = hc;
-  plan.subs = plan.warps / hc;
   plan.head_groups = (hkv + hc - 1) / hc;
+  // Rows per block. With many more (row, head group) pairs than the launch needs blocks, a block takes several
+  // rows: every warp then walks a longer range (up to a whole row of one KV head: no split, nothing to merge), and
+  // the ramp of its pipeline and the merge are paid less often. Kept: at least 2 blocks per SM for a launch on its
+  // own, about 32 blocks for one that runs side by side with its neighbours.
+  plan.rows_per_block = 1;
+  {
+    const int per_block = plan.warps / hc;  // (row, range) slots of a block
+    const int64_t want_blocks = throughput ? 32 : 2 * (int64_t)dev.sm_count;
+    for (int rb = per_block; rb > 1; --rb) {
+      if (per_block % rb != 0) continue;
+      if ((rows + rb - 1) / rb * plan.head_groups >= want_blocks) { plan.rows_per_block = rb; break; }
+    }
+  }
+  plan.subs = plan.warps / hc / plan.rows_per_block;
   if (throughput) {
     // a handful of (row, KV head) pairs (batch of one): split each over a small cluster until there are 16 blocks
-    while (c < 8 && rows * plan.head_groups * c < 16 && (int64_t)(c * 2) * plan.subs * kAttnStageTokens <= p.top_k) c *= 2;
+    while (plan.rows_per_block == 1 && c < 8 && rows * plan.head_groups * c < 16 &&
+           (int64_t)(c * 2) * plan.subs * kAttnStageTokens <= p.top_k)
+      c *= 2;
   } else {
     // Cluster: the largest power of two that still keeps every block resident at once.
     const int64_t blocks = rows * plan.head_groups;
-    while (c < 8 && blocks * (c * 2) <= max_resident_blocks(c * 2, plan.smem_bytes, plan.warps) &&
+    while (plan.rows_per_block == 1 && c < 8 && blocks * (c * 2) <= max_resident_blocks(c * 2, plan.smem_bytes, plan.warps) &&
            (int64_t)(c * 2) * plan.subs * kAttnStageTokens <= p.top_k)
       c *= 2;
   }
@@ -622,6 +649,8 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.top_k = p.top_k;
   a.heads_per_block = plan.heads_per_block;
   a.subs = plan.subs;
+  a.rows_per_block = plan.rows_per_block;
+  a.num_rows = (int64_t)p.num_seqs * p.q_per_seq;
   a.reverse = reverse;
   a.wait_prior = wait_prior;
   {
@@ -636,17 +665,19 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.rows_max = p.num_cache_rows;
   a.off32 = (a.rows_max > 0 && (double)a.rows_max * (double)(p.kv_token_stride >> 3) < 4294967296.0) ? 1 : 0;
   void (*kernel)(const AttnArgs);
-  if (a.group > 8)
-    kernel = p.block_table ? sparse_attn_kernel<2, true, kAttnWarpsWide> : sparse_attn_kernel<2, false, kAttnWarpsWide>;
-  else if (plan.warps == kAttnWarpsNarrow)
-    kernel = p.block_table ? sparse_attn_kernel<1, true, kAttnWarpsNarrow> : sparse_attn_kernel<1, false, kAttnWarpsNarrow>;
-  else
-    kernel = p.block_table ? sparse_attn_kernel<1, true, kAttnWarpsWide> : sparse_attn_kernel<1, false, kAttnWarpsWide>;
+  const bool multi = plan.rows_per_block > 1, pg = p.block_table != nullptr;
+#define CLSA_ATTN_PICK(NT_, W_)                                                                      \
+  (multi ? (pg ? sparse_attn_kernel<NT_, true, W_, true> : sparse_attn_kernel<NT_, false, W_, true>) \
+         : (pg ? sparse_attn_kernel<NT_, true, W_, false> : sparse_attn_kernel<NT_, false, W_, false>))
+  if (a.group > 8) kernel = CLSA_ATTN_PICK(2, kAttnWarpsWide);
+  else if (plan.warps == kAttnWarpsNarrow) kernel = CLSA_ATTN_PICK(1, kAttnWarpsNarrow);
+  else kernel = CLSA_ATTN_PICK(1, kAttnWarpsWide);
+#undef CLSA_ATTN_PICK
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(rows * plan.cluster), (unsigned)plan.head_groups, 1);
+  cfg.gridDim = dim3((unsigned)((rows + plan.rows_per_block - 1) / plan.rows_per_block * plan.cluster), (unsigned)plan.head_groups, 1);
   cfg.blockDim = dim3((unsigned)plan.warps * 32, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
