@@ -26,7 +26,8 @@ def _full_oracle(w):
 
 @pytest.mark.parametrize("B,T,n,d_idx,causal,ragged", [
     (1, 128, 1024, 128, 1, 0), (2, 200, 3000, 128, 1, 0), (1, 300, 2500, 64, 1, 0), (2, 77, 1111, 128, 0, 0),
-    (3, 150, 2000, 128, 1, 500), (1, 513, 700, 64, 1, 0)])
+    (3, 150, 2000, 128, 1, 500), (1, 513, 700, 64, 1, 0),
+    (2, 401, 2500, 128, 1, 0), (1, 650, 1500, 64, 0, 0)])   # the last two: several query rows per attention block, with a tail
 def test_chunk_scores_topk_attention(B, T, n, d_idx, causal, ragged):
     base = MID if d_idx == 128 else TINY
     cfg = base.replace(num_seqs=B, ctx=n, q_per_seq=T, causal=causal, top_k=96, num_layers=2, seed=900 + T + n,
@@ -52,7 +53,8 @@ def test_chunk_scores_topk_attention(B, T, n, d_idx, causal, ragged):
 
 @pytest.mark.parametrize("B,T,n,d_idx,causal,ragged,bs", [
     (2, 200, 3000, 128, 1, 0, 16), (1, 300, 2500, 64, 1, 0, 64), (3, 150, 2000, 128, 1, 500, 128),
-    (2, 77, 1111, 128, 0, 0, 256), (1, 260, 5000, 128, 1, 0, 1024), (2, 130, 300, 64, 1, 0, 32)])
+    (2, 77, 1111, 128, 0, 0, 256), (1, 260, 5000, 128, 1, 0, 1024), (2, 130, 300, 64, 1, 0, 32),
+    (2, 333, 2100, 128, 1, 0, 16)])
 def test_chunk_on_paged_caches(B, T, n, d_idx, causal, ragged, bs):
     """Paging changes addresses only: the chunk's scores are bit-identical to the contiguous run, and the rest of
     the chunk path (top-k, attention through the block table) agrees with the oracle."""
