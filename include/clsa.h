@@ -79,7 +79,7 @@ typedef struct {
   int32_t max_seq_len;  /* host-known upper bound of seq_len[], used for grid sizing (no device read-back) */
   float sm_scale;       /* softmax scale of Eq. 4's Attn, > 0; 1/sqrt(head_dim) in the benchmarks */
   int32_t sweep;        /* 0 or 1: direction in which clsa_sparse_attn walks the selected set; a cache-locality
-                           hint only (results agree to rounding). clsa_decode_step uses (sweep + l) & 1 for layer l */
+                           hint only (results agree to rounding). clsa_decode_step walks every layer in this direction */
   int32_t attn_plan;    /* launch shape of clsa_sparse_attn. 0: the whole GPU on this one launch (shortest time for a
                            launch that has to finish before anything else can run -- a layer whose output feeds the
                            next kernel). 1: a few large blocks per launch (about 32), for launches that run side by
@@ -150,7 +150,7 @@ CLSA_API clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const
  *   q_layers   HOST array of L device pointers, each bf16 [B][T][Hq][D]
  *   out_layers HOST array of L device pointers, each bf16 [B][T][Hq][D]
  * Equivalent, bit for bit, to clsa_index_scores, clsa_topk and L calls of clsa_sparse_attn made one
- * after another with sweep = (p->sweep + l) & 1 and attn_plan = 1 for layer l. The layers do not wait for one
+ * after another with attn_plan = 1 (and the same p->sweep for every layer). The layers do not wait for one
  * another (each reads only the index, the caches and its own queries), so several of them are in flight at once.
  * T > 1 is not chained here. */
 CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
@@ -162,7 +162,7 @@ CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, c
  * arrive on another stream while the routing runs, making `stream` wait on that upload just before this call.
  *   q_layers / out_layers  HOST arrays of L device pointers, each bf16 [B][T][Hq][D], 16-byte aligned
  *   idx, count             as written by clsa_topk (read only)
- * Bit for bit the L calls of clsa_sparse_attn with sweep = (p->sweep + l) & 1, attn_plan = 1 and lse = NULL, launched
+ * Bit for bit the L calls of clsa_sparse_attn with attn_plan = 1, the same p->sweep and lse = NULL, launched
  * so that a layer does not wait for its predecessor (which is why the calls are offered as one). */
 CLSA_API clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* const* q_layers, const int32_t* idx,
                                              const int32_t* count, void* const* out_layers, void* workspace,

@@ -104,14 +104,15 @@ clsa_status check_workspace(const void* ws, size_t ws_bytes, size_t need) {
 
 clsa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? CLSA_OK : CLSA_ERR_CUDA; }
 
-// The L attention launches that share one index. Layer l walks the selected set in direction (sweep + l) & 1, so a
-// layer starts on the rows its predecessor touched last. Layer 0 follows whatever produced the index and must wait
-// for it; every later layer reads only what was complete before its predecessor started (the index, the caches,
-// the caller's queries), so it may overlap its predecessor's tail.
+// The L attention launches that share one index. Layer 0 follows whatever produced the index and must wait for it;
+// every later layer reads only what was complete before its predecessor started (the index, the caches, the caller's
+// queries), so it does not wait, and several layers are in flight at once. All of them walk the selected set in the
+// same direction (p.sweep): a layer then trails its predecessor by a few microseconds over the same rows and finds
+// them in L2 (measured at the headline: 286 us per step against 320 us with alternating directions).
 cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, void* const* out_layers, const int32_t* idx,
                           const int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t s) {
   for (int l = 0; l < p.num_layers; ++l) {
-    const cudaError_t err = launch_sparse_attn(p, q_layers[l], idx, count, out_layers[l], nullptr, status, (p.sweep + l) & 1,
+    const cudaError_t err = launch_sparse_attn(p, q_layers[l], idx, count, out_layers[l], nullptr, status, p.sweep & 1,
                                                l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0, 1, dev, s);
     if (err != cudaSuccess) return err;
   }

@@ -24,8 +24,8 @@
 // are launched side by side instead: about 32 large blocks per layer (as many KV heads per block as that
 // allows), so that four or five layers are in flight at once: every SM stays busy and the per-block
 // fixed costs are paid 32 instead of 128 times per layer.
-// `reverse` flips the order in which a warp walks its range; alternating it between consecutive
-// layers makes layer l+1 start on the rows layer l touched last, which are the ones still in L2.
+// `reverse` flips the order in which a warp walks its range (a locality hint for callers that issue
+// dependent layers one by one; the chained layers of a step all walk the same way).
 #include <cooperative_groups.h>
 
 #include <mutex>
@@ -65,7 +65,7 @@ struct AttnArgs {
   int wait_prior;  // 1: inputs may come from the kernel launched just before this one (wait for it first)
   int off32;          // every row offset of the caches fits 32 bits when counted in 16-byte units
   int64_t rows_max;   // extent of the cache row space (off32 only): rows at or beyond it are refused like bad indices
-  int keep_permille;  // share of each warp's sweep (its end) whose rows are asked to stay in L2 for the next layer
+  int keep;           // 1: the rows are fetched with the L2 evict_last priority (launches behind this one read them again)
   float scale_log2;
 };
 
@@ -245,14 +245,11 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
       if (!paged || raw < 0 || raw >= n) return 0;
       return __ldg(table + (raw >> a.block_shift));
     };
-    // L2 residency across layers: consecutive layers walk the same rows in opposite directions, so
-    // the rows a warp reads LAST are the ones the next layer reads FIRST. Those are fetched with the
-    // evict_last priority; everything else (including their re-read by the next layer, which
-    // demotes them again) with evict_first, so that the protected share of the gathered set fits L2.
-    // (A launch that protects nothing leaves the replacement policy alone.)
-    const uint64_t pol_keep = l2_policy_evict_last();
-    const uint64_t pol_stream = a.keep_permille > 0 ? l2_policy_evict_first() : l2_policy_evict_normal();
-    const int keep_from = nstages - (nstages * a.keep_permille + 500) / 1000;  // steps >= keep_from are kept
+    // L2 residency across layers: the layers of a step walk the same rows in the same direction a few microseconds
+    // apart, so what one layer fetches the next ones find in L2. Such launches fetch with the evict_last priority
+    // (other traffic through L2 does not push the rows out in between); a launch on its own leaves the replacement
+    // policy alone.
+    const uint64_t pol = a.keep ? l2_policy_evict_last() : l2_policy_evict_normal();
     // Per-lane constants of the copies: where in a stage buffer this lane's 16-byte chunk of token j = 2*it + lane/16
     // goes (XOR swizzle), and the lane's byte offset inside a row.
     uint32_t sw[8];
@@ -266,7 +263,6 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
     const uint32_t stride16 = (uint32_t)(a.tok_stride >> 3);  // row stride in 16-byte units (the stride is a multiple of 8)
     auto issue = [&](int i, int raw, int blk) {
       if (i < nstages) {
-        const uint64_t pol = i >= keep_from ? pol_keep : pol_stream;
         const int buf = i % kAttnStages;
         const uint32_t kdst = ring_u32 + buf * kStageBytes, vdst = kdst + kStageBytes / 2;
         // cache row relative to s0: the position itself, or its place inside its block
@@ -653,13 +649,10 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.num_rows = (int64_t)p.num_seqs * p.q_per_seq;
   a.reverse = reverse;
   a.wait_prior = wait_prior;
-  {
-    // protect at most about half of L2 with the tail of this layer's sweep
-    const double gathered = (double)p.num_seqs * p.q_per_seq * (double)p.top_k * p.num_kv_heads * 512.0;
-    double share = 0.5 * (double)dev.l2_bytes / gathered;
-    if (share > 1.0) share = 1.0;
-    a.keep_permille = keep_for_next ? (int)(share * 1000.0) : 0;
-  }
+  // L2 priority of the gathered rows. A launch with a successor that will read the same rows (the chained layers)
+  // fetches all of them with evict_last, so that scores, indices and outputs passing through L2 do not push them
+  // out before the layers behind it arrive; a launch on its own leaves the replacement policy alone.
+  a.keep = keep_for_next ? 1 : 0;
   a.scale_log2 = p.sm_scale * kLog2e;
   // With the extent of the row space known (num_cache_rows) and below 2^32 16-byte units, row offsets are 32-bit.
   a.rows_max = p.num_cache_rows;
