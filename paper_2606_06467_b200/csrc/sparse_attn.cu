@@ -577,12 +577,12 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
     // split over tokens then stays inside a block); as many as possible once there are more rows than SMs.
     hc = 1;
     while (hc < hc_max && rows * ((hkv + hc - 1) / hc) > dev.sm_count) hc *= 2;
-    // A prefill chunk: the queries of a sequence all gather from the same cache, and blocks run head group by head
-    // group (rows fastest), so the rows of the head group in flight are what L2 has to hold: as few heads per
-    // block as it takes for them to fit in about 60 % of it (a 128K-token cache: one head, 66 MB).
-    if (p.q_per_seq > 1)
-      while (hc > 1 && (double)hc * p.max_seq_len * 512.0 > 0.6 * (double)dev.l2_bytes) hc /= 2;
   }
+  // A prefill chunk: the queries of a sequence all gather from the same cache, and blocks run head group by head
+  // group (rows fastest), so the rows of the head group in flight are what L2 has to hold: as few heads per
+  // block as it takes for them to fit in about 60 % of it (a 128K-token cache: one head, 66 MB).
+  if (p.q_per_seq > 1 && rows > dev.sm_count)
+    while (hc > 1 && (double)hc * p.max_seq_len * 512.0 > 0.6 * (double)dev.l2_bytes) hc /= 2;
   // every token range should hold at least one 16-token stage
   while (hc < hc_max && (int64_t)(plan.warps / hc) * kAttnStageTokens > p.top_k) hc *= 2;
   plan.heads_per_block = hc;
