@@ -259,3 +259,20 @@ def test_non_finite_scores_never_fault_and_keep_the_index_contract():
     # attention on those indices still runs and stays finite (the caches are finite)
     out, _ = g.sparse_attn(0)
     assert torch.isfinite(out.float()).all()
+
+
+def test_rows_beyond_the_declared_cache_extent_are_refused_not_read():
+    """num_cache_rows is the extent of the cache row space; a selected position that maps beyond it is treated like
+    an index outside its sequence: skipped and flagged, never dereferenced."""
+    w = Workload(MID.replace(num_seqs=2, ctx=1000, top_k=64, num_layers=1))
+    g = GpuProblem(w, layers=1)
+    g.topk(g.index_scores())
+    base, _ = g.sparse_attn(0)
+    assert g.status() == 0
+    g.params.num_cache_rows = 1500          # the second sequence (rows 1000..1999) now reaches past the extent
+    out, _ = g.sparse_attn(0)
+    torch.cuda.synchronize()
+    assert g.status() & clsa.CLSA_DEV_BAD_INDEX
+    assert torch.equal(out[0].view(torch.int16), base[0].view(torch.int16))      # the first sequence is untouched
+    assert torch.isfinite(out.float()).all()
+    clsa.clsa_clear_status(g.ws)
