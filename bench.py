@@ -53,6 +53,9 @@ def parse():
                     help="also time the upstream step (Eq. 2 projections of the new tokens + cache append, "
                          "clsa_project_append) on the same workload; reported under \"projection\", not part of the step")
     ap.add_argument("--block-size", type=int, default=0, help="page the caches into scattered blocks of this many rows")
+    ap.add_argument("--e2e-out", default="mapped", choices=["mapped", "copy"],
+                    help="end-to-end leg, decode: the layers store their outputs straight into pinned host memory "
+                         "(mapped) or into HBM followed by one device-to-host copy (copy)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-breakdown", action="store_true", help="skip the per-kernel instrumented loop")
     return ap.parse_args()
@@ -499,8 +502,12 @@ def run_ours(args):
     d_qidx = d_in[:n_qidx].view(t["q_idx"].shape)
     d_q = [d_in[n_qidx + l * n_q: n_qidx + (l + 1) * n_q].view(q_layers[l].shape) for l in range(L)]
     d_out = torch.empty((L,) + tuple(outs[0].shape), dtype=torch.bfloat16, device=dev)
-    e2e_outs = [d_out[l] for l in range(L)]
     h_out = torch.empty(d_out.shape, dtype=torch.bfloat16).pin_memory()
+    # A decode step's outputs are small (L x B x H x D bf16): the attention kernels can store them straight into the
+    # pinned host buffer, which the device addresses through the unified address space, instead of into HBM followed
+    # by a copy. The bytes that cross to the host are the same; the copy's launch and its wait for the last layer go.
+    mapped_out = T == 1 and args.e2e_out == "mapped"
+    e2e_outs = [(h_out if mapped_out else d_out)[l] for l in range(L)]
 
     # The routing needs only q_idx (a few KB). It goes up first on the launch stream; the L query tensors follow on a
     # second stream while the index scores and the top-k run, and the launch stream waits for them just before the
@@ -527,7 +534,8 @@ def run_ours(args):
         clsa.clsa_topk(p, e2e_scores, stride, idx, cnt, ws, stream=None)
         stream.wait_event(q_ready)
         clsa.clsa_sparse_attn_layers(p, d_q, idx, cnt, e2e_outs, ws, stream=None)
-        h_out.copy_(d_out, non_blocking=True)
+        if not mapped_out:
+            h_out.copy_(d_out, non_blocking=True)
 
     for _ in range(3):
         flush.zero_()
@@ -547,6 +555,8 @@ def run_ours(args):
     e2e_value = aggregate_value(world, alg_bytes, e2e_ms / K)
     h2d = h_in.numel() * 2
     d2h = h_out.numel() * 2
+    for l in range(L):  # the host copy of the last end-to-end step equals the device-resident step's outputs
+        assert torch.equal(h_out[l].view(torch.int16), outs[l].cpu().view(torch.int16)), f"end-to-end output {l} differs"
 
     # ---- per-kernel durations: the same launches issued as separate ABI calls with events between -------
     breakdown = None
@@ -641,7 +651,8 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms / K,
                     "note": "per-step inputs from pinned host memory (q_idx on the launch stream, the L query tensors on a "
-                            "second stream while the routing runs) and all L outputs back (one copy), through "
+                            "second stream while the routing runs) and all L outputs back ("
+                            + ("stored by the layers straight into pinned host memory" if mapped_out else "one copy") + "), through "
                             "clsa_index_scores + clsa_topk + clsa_sparse_attn_layers; the KV and indexer-key caches are "
                             "decoder state and stay resident"},
             "gpu_launches": K * (2 + L),

@@ -12,7 +12,11 @@
  * Conventions shared by every entry point
  * ---------------------------------------
  * Pointers: every pointer is a DEVICE pointer unless its comment says HOST. The clsa_params struct
- *   itself lives in host memory and is read during the call only.
+ *   itself lives in host memory and is read during the call only. "Device pointer" means any address
+ *   the device can dereference: the attention outputs, which are written once with plain stores, may
+ *   for example live in pinned host memory mapped into the unified address space (a decode step's
+ *   outputs then reach the host without a copy). Inputs that many blocks read (q_idx, the caches, the
+ *   index) belong in device memory: the kernels' traffic assumptions hold only there.
  * Ownership: the caller owns every buffer (inputs, outputs, workspace). The library allocates
  *   nothing, frees nothing, keeps no state between calls except cached device properties, and only
  *   enqueues work on the given stream. No entry point synchronises except clsa_device_status.

@@ -276,3 +276,22 @@ def test_rows_beyond_the_declared_cache_extent_are_refused_not_read():
     assert torch.equal(out[0].view(torch.int16), base[0].view(torch.int16))      # the first sequence is untouched
     assert torch.isfinite(out.float()).all()
     clsa.clsa_clear_status(g.ws)
+
+
+def test_outputs_may_live_in_pinned_host_memory():
+    """The attention outputs are written once with plain stores, so any address the device can reach serves: the
+    layers of a decode step store straight into pinned host memory and the host reads the same bits that a device
+    buffer would have held (single-block and cluster-merged epilogues both: B = 1 takes the cluster path)."""
+    for cfg in (MID.replace(num_seqs=6, ctx=2500, top_k=256, num_layers=3),
+                MID.replace(num_seqs=1, ctx=5000, top_k=1024, num_layers=2)):
+        w = Workload(cfg)
+        g = GpuProblem(w)
+        dev_outs = g.decode_step()
+        torch.cuda.synchronize()
+        host = torch.full((g.L,) + tuple(dev_outs[0].shape), float("nan"), dtype=torch.bfloat16).pin_memory()
+        clsa.clsa_sparse_attn_layers(g.params, [g.t["q_layers"][l] for l in range(g.L)], g.idx, g.count,
+                                     [host[l] for l in range(g.L)], g.ws)
+        torch.cuda.synchronize()
+        assert g.status() == 0
+        for l in range(g.L):
+            assert torch.equal(host[l].view(torch.int16), dev_outs[l].cpu().view(torch.int16)), l
