@@ -56,6 +56,9 @@ def parse():
     ap.add_argument("--e2e-out", default="mapped", choices=["mapped", "copy"],
                     help="end-to-end leg, decode: the layers store their outputs straight into pinned host memory "
                          "(mapped) or into HBM followed by one device-to-host copy (copy)")
+    ap.add_argument("--profile-range", action="store_true",
+                    help="bracket one extra step (after the warm-up, L2 flushed first) with cudaProfilerStart/Stop, so "
+                         "that a profiler in range mode sees the whole chained step with its layers in flight together")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-breakdown", action="store_true", help="skip the per-kernel instrumented loop")
     return ap.parse_args()
@@ -473,6 +476,13 @@ def run_ours(args):
             flush.zero_()
             step()
         sync_all()
+    if args.profile_range:
+        flush.zero_()
+        sync_all()
+        torch.cuda.profiler.start()
+        step()
+        torch.cuda.synchronize()
+        torch.cuda.profiler.stop()
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
     K = args.steps
