@@ -40,9 +40,11 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
 struct TopkPlan {
   int cluster;      // blocks per (sequence, query) row, a thread-block cluster
   int slice_cap;    // score slots each block keeps in shared memory (0 = re-read global memory each pass)
+  int one_sweep;    // the one-sweep kernel goes first; the general kernel then only finishes the rows it marks
   size_t smem_bytes;
 };
-TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev);
+// one_sweep_fits: whether the one-sweep kernel can take this launch (topk_prefilter_fits)
+TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev, bool one_sweep_fits);
 
 struct WorkspaceLayout {
   size_t scores_off, scores_bytes;  // fp32 score matrix of clsa_decode_step
@@ -60,9 +62,9 @@ cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, fl
                                      uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,
                         uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+bool topk_prefilter_fits(const clsa_params& p, const float* scores, int64_t score_stride, const DeviceInfo& dev);
 cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx,
-                                  int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream,
-                                  int* launched);
+                                  int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
                                int throughput_plan, const DeviceInfo& dev, cudaStream_t stream);

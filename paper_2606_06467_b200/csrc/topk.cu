@@ -28,10 +28,13 @@
 // among keys equal to the threshold the lowest positions win.
 // No atomics touch global memory and nothing spins.
 //
-// Launches with thousands of rows (a prefill chunk) first go through the one-sweep kernel in
-// topk_filter.cu; this kernel then runs once more, one block per 16 rows, for the rows that kernel
-// marked as unfinished (count = -1).
+// Launches with more rows than clusters that are resident at once (a prefill chunk's thousands of
+// rows, but also a decode batch of 34 or more 128K-token sequences) first go through the one-sweep
+// kernel in topk_filter.cu, if the shape fits it; this kernel then runs once more, one block per 16
+// rows, for the rows that kernel marked as unfinished (count = -1).
 #include <cooperative_groups.h>
+
+#include <mutex>
 
 #include "common.cuh"
 
@@ -600,7 +603,56 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
 
 }  // namespace
 
-TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev) {
+// Clusters of `cluster` blocks with `smem_bytes` of dynamic shared memory that are resident at once on the current
+// device (cached; a failed query falls back to one block per SM).
+static int resident_clusters(int cluster, size_t smem_bytes, bool cached, const DeviceInfo& dev) {
+  struct Entry { int dev, cluster, cached; size_t smem; int n; };
+  static std::mutex mu;
+  static Entry seen[16];
+  static int used = 0;
+  int d = 0;
+  if (cudaGetDevice(&d) != cudaSuccess) { cudaGetLastError(); return dev.sm_count / cluster; }
+  std::lock_guard<std::mutex> lock(mu);
+  for (int i = 0; i < used; ++i)
+    if (seen[i].dev == d && seen[i].cluster == cluster && seen[i].cached == (int)cached && seen[i].smem == smem_bytes) return seen[i].n;
+  auto kernel = cached ? topk_radix_kernel<true> : topk_radix_kernel<false>;
+  int n = 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)cluster * 64, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess ||
+      cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    n = dev.sm_count / cluster;
+  }
+  if (used < 16) seen[used++] = Entry{d, cluster, (int)cached, smem_bytes, n};
+  return n;
+}
+
+// Shared memory of a block whose slice of the row is `per` scores: the keys are kept there whenever they fit,
+// even if that leaves one block per SM and several waves (measured: 64 rows of 131072 in two waves of one block
+// per SM 41 us, in one wave of two blocks per SM that re-read their slices from L2 in every sweep 49 us).
+static void size_blocks(TopkPlan& plan, int max_seq_len, const DeviceInfo& dev) {
+  const int per = (((max_seq_len + plan.cluster - 1) / plan.cluster) + 3) & ~3;
+  const size_t want = sizeof(Shared) + (size_t)per * sizeof(uint32_t);
+  if (want <= (size_t)dev.max_smem_optin) {
+    plan.slice_cap = per;
+    plan.smem_bytes = want;
+  } else {
+    plan.slice_cap = 0;  // slice too long for shared memory: keys are recomputed from global memory in every sweep
+    plan.smem_bytes = sizeof(Shared);
+  }
+}
+
+TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev, bool one_sweep_fits) {
   TopkPlan plan;
   // One block per 32K visible scores, capped at kMaxCluster and rounded to a power of two; when there are few
   // rows, spread each over more blocks (down to 2K scores per block).
@@ -612,34 +664,34 @@ TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev) {
   while (pow2 < 4 && rows * pow2 * 2 <= dev.sm_count && p.max_seq_len / (pow2 * 2) >= 2048) pow2 <<= 1;
   // a handful of rows (small-batch decoding): clusters of 8, all of which are resident at once up to 8 rows
   if (pow2 == 4 && rows <= 8 && p.max_seq_len / 8 >= 2048) pow2 = 8;
-  // Many more rows than SMs (a prefill chunk): throughput matters, not the latency of one row. One block per
-  // row needs no cluster barriers and keeps more rows in flight; its keys are re-read from global memory in
-  // each of the three sweeps when they do not fit in shared memory.
-  if (rows >= 4 * (int64_t)dev.sm_count) pow2 = 1;
   plan.cluster = pow2;
-  const int per = (((p.max_seq_len + plan.cluster - 1) / plan.cluster) + 3) & ~3;
-  const size_t want = sizeof(Shared) + (size_t)per * sizeof(uint32_t);
-  // two blocks per SM: each may use half of the SM's shared memory less the per-block reservation
-  const size_t half_sm = ((size_t)dev.max_smem_optin + 1024) / 2 - 1024;
-  if (want <= half_sm || (want <= (size_t)dev.max_smem_optin && rows * plan.cluster <= dev.sm_count)) {
-    plan.slice_cap = per;
-    plan.smem_bytes = want;
-  } else {
-    plan.slice_cap = 0;  // slice too long for shared memory: keys are recomputed from global memory in every sweep
-    plan.smem_bytes = sizeof(Shared);
+  plan.one_sweep = 0;
+  size_blocks(plan, p.max_seq_len, dev);
+  // Many rows. Far more rows than SMs (a prefill chunk): throughput matters, not the latency of one row; one block
+  // per row needs no cluster barriers and keeps more rows in flight. And whenever the clusters of this launch would
+  // not all be resident at once, the one-sweep kernel (one block per row, two blocks per SM, one pass over the
+  // scores) is faster than a second wave of clusters, if the shape fits it: 64 rows of 131072 scores 41 -> 34 us,
+  // 200 rows 150 -> 48 us, 400 rows of 32768 68 -> 42 us; 33 rows of 131072, the most that one wave of clusters of 4
+  // holds, 32 us either way.
+  bool many = rows >= 4 * (int64_t)dev.sm_count;
+  if (!many && one_sweep_fits && rows > resident_clusters(plan.cluster, plan.smem_bytes, plan.slice_cap > 0, dev)) many = true;
+  if (many) {
+    plan.cluster = 1;
+    plan.one_sweep = one_sweep_fits ? 1 : 0;
+    size_blocks(plan, p.max_seq_len, dev);
   }
   return plan;
 }
 
 cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,
                         uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
-  const TopkPlan plan = make_topk_plan(p, dev);
+  const TopkPlan plan = make_topk_plan(p, dev, topk_prefilter_fits(p, scores, score_stride, dev));
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
-  // Many long rows (a prefill chunk): a one-sweep kernel takes every row it can finish exactly and marks the
-  // rest; the general kernel below then runs for the marked rows only.
-  int pending_only = 0;
-  if (plan.cluster == 1) {
-    const cudaError_t pre = launch_topk_prefilter(p, scores, score_stride, idx, count, status, dev, stream, &pending_only);
+  // Many rows: a one-sweep kernel takes every row it can finish exactly and marks the rest; the general kernel
+  // below then runs for the marked rows only.
+  const int pending_only = plan.one_sweep;
+  if (pending_only) {
+    const cudaError_t pre = launch_topk_prefilter(p, scores, score_stride, idx, count, status, dev, stream);
     if (pre != cudaSuccess) return pre;
   }
   const int pending_rows = pending_only ? (int)rows : 0;

@@ -1,5 +1,6 @@
 // Token-level top-k (Eq. 3, second half) for many long rows at once (a prefill chunk: thousands of
-// (sequence, query) rows of 10^5 scores each), where throughput matters and not the latency of one row.
+// (sequence, query) rows of 10^5 scores each; or a decode batch with more rows than the general kernel's
+// clusters can all be resident for), where throughput matters and not the latency of one row.
 //
 // The general kernel (topk.cu) reads a row three times and pays a vote and a shared-memory atomic per
 // score. Here a row is read ONCE at full width, and per score only a float compare is paid:
@@ -24,6 +25,8 @@
 // too long for the bitmap, misaligned for 16-byte loads, or holding NaNs that the float compare lets through
 // below the pivot -- is marked pending (count = -1) and is taken by the general kernel, launched right after for
 // pending rows only. Nothing is approximated.
+#include <cmath>
+
 #include "common.cuh"
 
 namespace clsa {
@@ -124,6 +127,15 @@ topk_prefilter_kernel(const float* __restrict__ scores, int64_t score_stride, co
   const int row = blockIdx.x;
   const int b = row / q_per_seq, t = row % q_per_seq;
   const int tid = threadIdx.x, lane = tid & 31;
+  // Programmatic dependent launch: the kernel behind this one may be scheduled early (it waits for this grid
+  // itself), and this grid may have been scheduled before the kernel that writes the scores has finished: shared
+  // memory is cleared meanwhile, and the wait comes before the first global access.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  for (int i = tid; i < 4096; i += kThreads) sh.hist[i] = 0u;
+  for (int i = tid; i < 1024; i += kThreads) sh.hist10[i] = 0u;
+  for (int i = tid; i < bitmap_words; i += kThreads) bitmap[i] = 0u;
+  if (tid == 0) { sh.cand_count = 0u; sh.cand_max = 0u; sh.small_count = 0u; sh.below_pivot = 0u; }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n = seq_len[b];
   int v = causal ? n - q_per_seq + t + 1 : n;
   if (n < q_per_seq || n > max_seq_len) {
@@ -145,18 +157,14 @@ topk_prefilter_kernel(const float* __restrict__ scores, int64_t score_stride, co
   const float4* src4 = reinterpret_cast<const float4*>(src);
   const int n4 = v >> 2;
 
-  // ---- 1. pivot from a sample (its loads are in flight while shared memory is cleared) ----------------------------
+  // ---- 1. pivot from a sample ------------------------------------------------------------------------------------
   constexpr int kPer = kSample / 4 / kThreads;  // 16-byte samples per thread, kept in registers
   float4 smp[kPer];
   if (v > kCandCap) {
 #pragma unroll
     for (int u = 0; u < kPer; ++u) smp[u] = src4[(int)(((int64_t)(tid + u * kThreads) * n4) / (kSample / 4))];
   }
-  for (int i = tid; i < 4096; i += kThreads) sh.hist[i] = 0u;
-  for (int i = tid; i < 1024; i += kThreads) sh.hist10[i] = 0u;
-  for (int i = tid; i < bitmap_words; i += kThreads) bitmap[i] = 0u;
-  if (tid == 0) { sh.cand_count = 0u; sh.cand_max = 0u; sh.small_count = 0u; sh.below_pivot = 0u; }
-  __syncthreads();
+  __syncthreads();  // the clears at the top
 
   uint32_t pivot = 0u;  // rows that fit the candidate list whole need none
   if (v > kCandCap) {
@@ -364,28 +372,48 @@ topk_prefilter_kernel(const float* __restrict__ scores, int64_t score_stride, co
 
 }  // namespace
 
-// Launches the one-sweep kernel when the shape suits it. *launched = 1 tells the caller to follow up with the
-// general kernel restricted to rows whose count is -1.
-cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx,
-                                  int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream,
-                                  int* launched) {
-  *launched = 0;
-  const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
-  if (rows < 4 * (int64_t)dev.sm_count) return cudaSuccess;        // few rows: the cluster kernel is the fast one
-  if (p.max_seq_len <= kCandCap) return cudaSuccess;               // short rows fit the general kernel's shared memory
-  if (p.top_k > kCandCap * 2 / 3) return cudaSuccess;              // the candidate list must hold k plus the pivot's margin
-  if (score_stride % 4 != 0 || reinterpret_cast<uintptr_t>(scores) % 16 != 0) return cudaSuccess;
+// Whether the one-sweep kernel can take this launch at all (the caller decides whether it should).
+bool topk_prefilter_fits(const clsa_params& p, const float* scores, int64_t score_stride, const DeviceInfo& dev) {
+  if (p.max_seq_len <= kCandCap) return false;               // short rows fit the general kernel's shared memory
+  {
+    // The candidate list must hold what the sampled pivot lets through on the longest row: the pivot sits at rank
+    // r of the sample (the kernel's formula), so about n r / kSample scores pass it, give or take n sqrt(r) / kSample;
+    // a launch whose rows would mostly overflow the list is better served by the general kernel from the start
+    // (k = 4096 of 131072: 5960 +- 440 expected against 6144 slots).
+    const double n = (double)p.max_seq_len, k = (double)(p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len);
+    const double expect = (double)kSample * k / n * 1.10;
+    const double r = expect + 3.5 * sqrt(expect) + 4.0;
+    if (n * (r + 2.5 * sqrt(r)) / (double)kSample > (double)kCandCap) return false;
+  }
+  if (score_stride % 4 != 0 || reinterpret_cast<uintptr_t>(scores) % 16 != 0) return false;
   const int bitmap_words = ((p.max_seq_len + 31) / 32 + 3) & ~3;
   const size_t smem = sizeof(FShared) + (size_t)bitmap_words * sizeof(uint32_t);
   const size_t half_sm = ((size_t)dev.max_smem_optin + 1024) / 2 - 1024;  // two blocks per SM
-  if (smem > half_sm) return cudaSuccess;                          // rows too long for the bitmaps
+  return smem <= half_sm;                                    // longer rows do not fit the bitmaps
+}
+
+// Launches the one-sweep kernel (the shape must fit, see above). The caller follows up with the general kernel
+// restricted to rows whose count is -1.
+cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx,
+                                  int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
+  (void)dev;
+  const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
+  const int bitmap_words = ((p.max_seq_len + 31) / 32 + 3) & ~3;
+  const size_t smem = sizeof(FShared) + (size_t)bitmap_words * sizeof(uint32_t);
   cudaError_t err = cudaFuncSetAttribute(topk_prefilter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  topk_prefilter_kernel<<<(unsigned)rows, kThreads, smem, stream>>>(scores, score_stride, p.seq_len, (int)p.q_per_seq,
-                                                                    (int)p.causal, (int)p.top_k, (int)p.max_seq_len,
-                                                                    bitmap_words, idx, count, status);
-  *launched = 1;
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)rows, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, topk_prefilter_kernel, scores, score_stride, p.seq_len, (int)p.q_per_seq, (int)p.causal,
+                            (int)p.top_k, (int)p.max_seq_len, bitmap_words, idx, count, status);
 }
 
 }  // namespace clsa

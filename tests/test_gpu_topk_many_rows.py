@@ -138,13 +138,17 @@ def test_many_rows_misaligned_rows_and_non_finite_scores_keep_the_contract():
                                    g2.count[:, finite_rows], sub)
 
 
-def test_many_sequences_one_query_each():
-    """The same route when the rows are 640 sequences of different lengths (a large decode batch), not the queries
-    of one chunk: selection only, on random scores, against the oracle's sort."""
-    B, k, n_max = ROWS, 800, 16000
-    rng = np.random.default_rng(99)
+@pytest.mark.parametrize("B,k,n_max", [(ROWS, 800, 16000), (40, 2048, 131072), (64, 2048, 100000), (150, 512, 40000),
+                                       (34, 4096, 131072), (48, 3000, 131072)],
+                         ids=["640x16000", "40x131072", "64x100000", "150x40000", "34x131072-k4096", "48x131072-k3000"])
+def test_many_sequences_one_query_each(B, k, n_max):
+    """The same route when the rows are sequences of different lengths (a decode batch), not the queries of one
+    chunk: 640 rows, and batches just large enough that their clusters would not all be resident at once (the
+    one-sweep kernel takes those too, unless k is so large that its candidate list would overflow: k = 4096 of
+    131072 stays with the cluster kernel). Selection only, on random scores, against the oracle's sort."""
+    rng = np.random.default_rng(99 + B)
     lens = rng.integers(500, n_max + 1, B).astype(np.int32)
-    lens[:3] = (n_max, 799, 6145)                      # longest, shorter than k, just above the candidate list's capacity
+    lens[:3] = (n_max, k - 1, 6145)                    # longest, shorter than k, just above the candidate list's capacity
     dev = torch.device("cuda:0")
     stride = (n_max + 63) // 64 * 64
     sc_host = (rng.standard_normal((B, 1, stride)) * 11.3).astype(np.float32)
