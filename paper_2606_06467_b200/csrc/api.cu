@@ -54,7 +54,7 @@ clsa_status check_shape(const clsa_params* p) {
   if (p->num_q_heads % p->num_kv_heads != 0) return CLSA_ERR_INVALID_ARG;
   if (p->causal != 0 && p->causal != 1) return CLSA_ERR_INVALID_ARG;
   if (p->sweep != 0 && p->sweep != 1) return CLSA_ERR_INVALID_ARG;
-  if (p->attn_plan != 0 && p->attn_plan != 1) return CLSA_ERR_INVALID_ARG;
+  if (p->attn_plan < 0 || p->attn_plan > 2) return CLSA_ERR_INVALID_ARG;
   if (p->max_seq_len < p->q_per_seq) return CLSA_ERR_INVALID_ARG;
   if (!isfinite(p->sm_scale) || !(p->sm_scale > 0.f)) return CLSA_ERR_INVALID_ARG;  // the kernels take maxima before scaling
   if ((int64_t)p->num_seqs * p->q_per_seq > (int64_t)1 << 30) return CLSA_ERR_INVALID_ARG;
@@ -111,9 +111,11 @@ clsa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? CLSA_OK : CLSA_
 // them in L2 (measured at the headline: 286 us per step against 320 us with alternating directions).
 cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, void* const* out_layers, const int32_t* idx,
                           const int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t s) {
+  const int fine_tail = chain_fine_tail(p, dev);  // the last layers use smaller blocks so that the chain ends flush
   for (int l = 0; l < p.num_layers; ++l) {
     const cudaError_t err = launch_sparse_attn(p, q_layers[l], idx, count, out_layers[l], nullptr, status, p.sweep & 1,
-                                               l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0, 1, dev, s);
+                                               l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0,
+                                               l >= p.num_layers - fine_tail ? 2 : 1, dev, s);
     if (err != cudaSuccess) return err;
   }
   return cudaSuccess;

@@ -34,8 +34,13 @@ struct AttnPlan {
   int head_groups;      // ceil(Hkv / HC): grid.y
   size_t smem_bytes;
 };
-// throughput != 0: a few large blocks (the launch shares the GPU with its neighbours on the stream)
+// throughput: 0 = a launch on its own (whole-GPU shape); 1 = a few large blocks (the launch shares the GPU with its
+// neighbours on the stream); 2 = the same with half the KV heads per block, where that is possible (twice the
+// blocks: used for the last layers of a chain, see chain_fine_tail)
 AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int throughput);
+// How many of the last layers of an L-layer chain should use the finer shape (throughput = 2) so that the chain's
+// blocks fill the SMs evenly to the end.
+int chain_fine_tail(const clsa_params& p, const DeviceInfo& dev);
 
 struct TopkPlan {
   int cluster;      // blocks per (sequence, query) row, a thread-block cluster

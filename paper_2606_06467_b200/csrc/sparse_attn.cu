@@ -27,6 +27,9 @@
 // `reverse` flips the order in which a warp walks its range (a locality hint for callers that issue
 // dependent layers one by one; the chained layers of a step all walk the same way).
 #include <cooperative_groups.h>
+#include <vector>
+#include <functional>
+#include <algorithm>
 
 #include <mutex>
 
@@ -572,6 +575,7 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
     // (measured: 32 blocks per layer beat 16, 64 and 128 at every batch size tried).
     hc = hc_max;
     while (hc > 1 && rows * ((hkv + hc - 1) / hc) < 32) hc /= 2;
+    if (throughput == 2 && hc > 1) hc /= 2;
   } else {
     // Heads per block: as few as it takes for all blocks to be resident at once (more blocks, and the
     // split over tokens then stays inside a block); as many as possible once there are more rows than SMs.
@@ -594,7 +598,7 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   plan.rows_per_block = 1;
   {
     const int per_block = plan.warps / hc;  // (row, range) slots of a block
-    const int64_t want_blocks = throughput ? 32 : 2 * (int64_t)dev.sm_count;
+    const int64_t want_blocks = throughput ? (throughput == 2 ? 64 : 32) : 2 * (int64_t)dev.sm_count;
     for (int rb = per_block; rb > 1; --rb) {
       if (per_block % rb != 0) continue;
       if ((rows + rb - 1) / rb * plan.head_groups >= want_blocks) { plan.rows_per_block = rb; break; }
@@ -615,6 +619,73 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   }
   plan.cluster = c;
   return plan;
+}
+
+// The layers of a chain are launched back to back and none waits for its predecessor, so their blocks fill the
+// SMs like a list schedule: a block starts when an SM frees up, and a layer's blocks are placed only once the layer
+// before it has started all of its own. With equal blocks the last round is usually part empty (16 layers of 32
+// blocks on 148 SMs: 3.46 rounds, the fourth with 68 blocks). Blocks of half the size in the last few layers fill
+// that round at a finer grain. How many layers: the schedule is simulated for every choice with a block's duration
+// modelled as a fixed part (launch gap, ramp, merge: 9.5 us measured) plus its bytes at the per-SM gather rate
+// (118 GB/s measured), and the best choice is taken if it gains at least 2 %. Cached per shape.
+int chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
+  const int L = p.num_layers;
+  if (L < 2 || L > 256) return 0;
+  if (p.block_table != nullptr) return 0;  // paged caches: measured, the finer blocks cost more than the fuller last round returns
+  const AttnPlan base = make_attn_plan(p, dev, 1), fine = make_attn_plan(p, dev, 2);
+  if (base.cluster != 1 || fine.cluster != 1 || fine.heads_per_block == base.heads_per_block ||
+      fine.rows_per_block != base.rows_per_block)
+    return 0;
+  const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
+  const int64_t nb_base = (rows + base.rows_per_block - 1) / base.rows_per_block * base.head_groups;
+  const int64_t nb_fine = (rows + fine.rows_per_block - 1) / fine.rows_per_block * fine.head_groups;
+  if (nb_base > 4096 || nb_fine > 8192) return 0;  // far more blocks than SMs: the last round is a small part of the whole
+  struct Key { int L, sms, k, hb, hf; int64_t nb, nf; int tail; };
+  static std::mutex mu;
+  static Key seen[16];
+  static int used = 0;
+  std::lock_guard<std::mutex> lock(mu);
+  for (int i = 0; i < used; ++i)
+    if (seen[i].L == L && seen[i].sms == dev.sm_count && seen[i].k == p.top_k && seen[i].hb == base.heads_per_block &&
+        seen[i].hf == fine.heads_per_block && seen[i].nb == nb_base && seen[i].nf == nb_fine)
+      return seen[i].tail;
+  const double k_eff = (double)(p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len);
+  auto duration = [&](const AttnPlan& pl) {  // microseconds
+    const double bytes = (double)pl.heads_per_block * pl.rows_per_block * k_eff * 512.0;
+    return 9.5 + bytes / 118e3;
+  };
+  const double d_base = duration(base), d_fine = duration(fine);
+  std::vector<double> heap((size_t)dev.sm_count);
+  auto makespan = [&](int tail) {
+    std::fill(heap.begin(), heap.end(), 0.0);  // all equal: a valid min-heap (std::greater)
+    double end = 0.0, gate = 0.0;
+    for (int l = 0; l < L; ++l) {
+      const bool f = l >= L - tail;
+      const int64_t nb = f ? nb_fine : nb_base;
+      const double d = f ? d_fine : d_base;
+      double last_start = gate;
+      for (int64_t j = 0; j < nb; ++j) {
+        std::pop_heap(heap.begin(), heap.end(), std::greater<double>());
+        const double t = std::max(heap.back(), gate);
+        heap.back() = t + d;
+        std::push_heap(heap.begin(), heap.end(), std::greater<double>());
+        end = std::max(end, t + d);
+        last_start = std::max(last_start, t);
+      }
+      gate = last_start;
+    }
+    return end;
+  };
+  const double plain = makespan(0);
+  double best = plain;
+  int best_tail = 0;
+  for (int tail = 1; tail <= L; ++tail) {
+    const double m = makespan(tail);
+    if (m < best - 1e-9) { best = m; best_tail = tail; }
+  }
+  if (best > 0.98 * plain) best_tail = 0;
+  if (used < 16) seen[used++] = Key{L, dev.sm_count, p.top_k, base.heads_per_block, fine.heads_per_block, nb_base, nb_fine, best_tail};
+  return best_tail;
 }
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,

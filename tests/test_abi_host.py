@@ -67,7 +67,7 @@ def test_bad_arguments_are_refused_on_the_host(clsa):
     for kw, want in (
         (dict(num_seqs=0), clsa.CLSA_ERR_INVALID_ARG), (dict(top_k=0), clsa.CLSA_ERR_INVALID_ARG),
         (dict(num_q_heads=30), clsa.CLSA_ERR_INVALID_ARG), (dict(causal=2), clsa.CLSA_ERR_INVALID_ARG),
-        (dict(sweep=3), clsa.CLSA_ERR_INVALID_ARG), (dict(attn_plan=2), clsa.CLSA_ERR_INVALID_ARG), (dict(max_seq_len=0), clsa.CLSA_ERR_INVALID_ARG),
+        (dict(sweep=3), clsa.CLSA_ERR_INVALID_ARG), (dict(attn_plan=3), clsa.CLSA_ERR_INVALID_ARG), (dict(max_seq_len=0), clsa.CLSA_ERR_INVALID_ARG),
         (dict(sm_scale=float("nan")), clsa.CLSA_ERR_INVALID_ARG), (dict(sm_scale=0.0), clsa.CLSA_ERR_INVALID_ARG), (dict(num_layers=0), clsa.CLSA_ERR_INVALID_ARG),
         (dict(head_dim=64), clsa.CLSA_ERR_UNSUPPORTED), (dict(idx_dim=96), clsa.CLSA_ERR_UNSUPPORTED),
         (dict(num_q_heads=34, num_kv_heads=2), clsa.CLSA_ERR_UNSUPPORTED),

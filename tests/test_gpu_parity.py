@@ -49,21 +49,29 @@ def _run_all(w, layers=None, check_lse=True):
         out1, lse1 = g.sparse_attn(l, sweep=0, plan=1)
         check_attention(prob, w, l, out1, lse1 if check_lse else None, idx_np, cnt_np)
         assert (out.float() - out1.float()).abs().max().item() <= 2e-2
-        singles.append(out1)
+        # ... and its finer variant, which a chain may use for its last layers
+        out2, lse2 = g.sparse_attn(l, sweep=0, plan=2)
+        check_attention(prob, w, l, out2, lse2 if check_lse else None, idx_np, cnt_np)
+        singles.append((out1, out2))
     # the chain: same index for all layers, byte-identical to the separate calls in the chain's launch shape
     g.idx.fill_(-7); g.count.fill_(-7)
     outs = g.decode_step()
     torch.cuda.synchronize()
     np.testing.assert_array_equal(g.idx.cpu().numpy(), idx_np)
     np.testing.assert_array_equal(g.count.cpu().numpy(), cnt_np)
+    def same_as_a_single(o, l):   # bit for bit one of the two side-by-side shapes, the finer one only in a tail
+        return [torch.equal(o.view(torch.int16), x.view(torch.int16)) for x in singles[l]]
+
+    fine = [not same_as_a_single(outs[l], l)[0] for l in range(g.L)]
     for l in range(g.L):
-        assert torch.equal(outs[l].view(torch.int16), singles[l].view(torch.int16)), f"layer {l}: chain != separate call"
+        assert any(same_as_a_single(outs[l], l)), f"layer {l}: chain != separate call"
+    assert fine == sorted(fine), f"the finer shape is used for the last layers only: {fine}"
     # the attention half of the chain on its own, fed the index that is already there
     layer_outs = [g.new_out() for _ in range(g.L)]
     clsa.clsa_sparse_attn_layers(g.params, [g.t["q_layers"][l] for l in range(g.L)], g.idx, g.count, layer_outs, g.ws)
     torch.cuda.synchronize()
     for l in range(g.L):
-        assert torch.equal(layer_outs[l].view(torch.int16), singles[l].view(torch.int16)), f"layer {l}: layers call"
+        assert torch.equal(layer_outs[l].view(torch.int16), outs[l].view(torch.int16)), f"layer {l}: layers call"
     np.testing.assert_array_equal(g.idx.cpu().numpy(), idx_np)  # the shared index is read, never written
     assert g.status() == 0
     return g, prob
