@@ -66,6 +66,7 @@ def _run_all(w, layers=None, check_lse=True):
     for l in range(g.L):
         assert any(same_as_a_single(outs[l], l)), f"layer {l}: chain != separate call"
     assert fine == sorted(fine), f"the finer shape is used for the last layers only: {fine}"
+    g.fine_layers = sum(fine)
     # the attention half of the chain on its own, fed the index that is already there
     layer_outs = [g.new_out() for _ in range(g.L)]
     clsa.clsa_sparse_attn_layers(g.params, [g.t["q_layers"][l] for l in range(g.L)], g.idx, g.count, layer_outs, g.ws)
@@ -100,6 +101,16 @@ def test_ragged_with_duplicates_and_short_sequences():
     dup = dup[local[local[dup]] == local[dup]]   # keep copies whose source position still holds its own base row
     assert dup.size > 10
     np.testing.assert_array_equal(gs[b, 0, dup].view(np.uint32), gs[b, 0, local[dup]].view(np.uint32))
+
+
+def test_chain_with_finer_last_layers():
+    """The headline's launch geometry at a context the oracle handles in seconds: 16 layers of 32 blocks do not fill
+    148 SMs evenly, so the chain gives its last layers the finer shape; every layer still equals the separate call of
+    its shape bit for bit, and the oracle within tolerance."""
+    w = Workload(MID.replace(num_seqs=16, ctx=4096, top_k=2048, num_layers=16, seed=31))
+    g, _ = _run_all(w, check_lse=False)
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert 1 <= g.fine_layers <= 8, g.fine_layers
 
 
 def test_planted_tokens_are_selected():
