@@ -67,6 +67,8 @@ typedef enum {
 #define CLSA_DEV_BAD_SEQLEN 2u  /* seq_len[b] < q_per_seq or > max_seq_len: that sequence was skipped */
 #define CLSA_DEV_BAD_COUNT 4u   /* count[b,t] < 0 or > top_k: clamped */
 #define CLSA_DEV_TIMEOUT 8u     /* a bounded wait inside a kernel ran out; the kernel returned early, results are invalid */
+#define CLSA_DEV_BAD_WORKSPACE 16u /* the workspace header was not zero before its first use (the score kernel found its
+                                      scheduling counters out of range): results are invalid */
 
 typedef void* clsa_stream; /* a cudaStream_t */
 
@@ -116,7 +118,8 @@ typedef struct {
 /* Bytes of workspace that any of the calls below may need for these params (the maximum over the
  * four; clsa_decode_step additionally keeps the fp32 score matrix there). Reads only the scalar
  * fields. *bytes is HOST memory. The workspace must be 256-byte aligned; its first 256 bytes hold
- * the device status word and must be zero before the first call (cudaMemset or clsa_clear_status).
+ * the device status word and the score kernel's scheduling counters (which every launch leaves at
+ * zero) and must be zero before the first call (cudaMemset or clsa_clear_status).
  * Calls that overlap on the GPU must not share a workspace. */
 CLSA_API clsa_status clsa_workspace_bytes(const clsa_params* p, size_t* bytes);
 

@@ -15,7 +15,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libclsa.so")
 
 CLSA_OK, CLSA_ERR_INVALID_ARG, CLSA_ERR_UNSUPPORTED, CLSA_ERR_WORKSPACE, CLSA_ERR_CUDA = range(5)
-CLSA_DEV_BAD_INDEX, CLSA_DEV_BAD_SEQLEN, CLSA_DEV_BAD_COUNT, CLSA_DEV_TIMEOUT = 1, 2, 4, 8
+CLSA_DEV_BAD_INDEX, CLSA_DEV_BAD_SEQLEN, CLSA_DEV_BAD_COUNT, CLSA_DEV_TIMEOUT, CLSA_DEV_BAD_WORKSPACE = 1, 2, 4, 8, 16
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

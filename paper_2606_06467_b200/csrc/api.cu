@@ -155,7 +155,8 @@ clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, float* sc
   if (p->q_per_seq > 1)
     return from_cuda(launch_index_scores_gemm(*p, q_idx, scores, score_stride, static_cast<uint32_t*>(workspace), dev,
                                               static_cast<cudaStream_t>(stream)));
-  return from_cuda(launch_index_scores_decode(*p, q_idx, scores, score_stride, static_cast<uint32_t*>(workspace), dev,
+  return from_cuda(launch_index_scores_decode(*p, q_idx, scores, score_stride, static_cast<uint32_t*>(workspace),
+                                              static_cast<uint32_t*>(workspace) + kSchedWord, dev,
                                               static_cast<cudaStream_t>(stream)));
 }
 
@@ -212,7 +213,7 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
   auto status = reinterpret_cast<uint32_t*>(base);
   auto scores = reinterpret_cast<float*>(base + w.scores_off);
   auto s = static_cast<cudaStream_t>(stream);
-  cudaError_t err = launch_index_scores_decode(*p, q_idx, scores, w.score_stride, status, dev, s);
+  cudaError_t err = launch_index_scores_decode(*p, q_idx, scores, w.score_stride, status, status + kSchedWord, dev, s);
   if (err != cudaSuccess) return CLSA_ERR_CUDA;
   err = launch_topk(*p, scores, w.score_stride, idx, count, status, dev, s);
   if (err != cudaSuccess) return CLSA_ERR_CUDA;
@@ -314,7 +315,11 @@ clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, con
   uint32_t* status = dev_status != nullptr ? dev_status : reinterpret_cast<uint32_t*>(base);
   if (dev_status == nullptr && cudaMemsetAsync(base, 0, kStatusBytes, s) != cudaSuccess) return CLSA_ERR_CUDA;
   auto scores = reinterpret_cast<float*>(base + kStatusBytes);
-  if (launch_index_scores_decode(*p, q_idx, scores, stride, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
+  // the score kernel's scheduling counters always live in the scratch array's header (zero when the library is
+  // loaded, and left at zero by every launch), also when the status word is the caller's
+  if (launch_index_scores_decode(*p, q_idx, scores, stride, status, reinterpret_cast<uint32_t*>(base) + kSchedWord, dev, s) !=
+      cudaSuccess)
+    return CLSA_ERR_CUDA;
   if (launch_topk(*p, scores, stride, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
   if (launch_layers(*p, q_layers, out_layers, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
   return CLSA_OK;

@@ -18,7 +18,8 @@ struct DeviceInfo {
 // Cached per device (queried once). Returns false if the CUDA runtime reports an error.
 bool device_info(DeviceInfo* out);
 
-constexpr size_t kStatusBytes = 256;   // status word + padding at the start of the workspace
+constexpr size_t kStatusBytes = 256;   // status word, scheduling counters and padding at the start of the workspace
+constexpr int kSchedWord = 16;         // 32-bit word of that header where the score kernel's two ticket counters sit (zero between launches)
 constexpr int kAttnWarpsNarrow = 12;    // warps per attention block (groups of up to 8 query heads per KV head), each an autonomous worker
 constexpr int kAttnWarpsWide = 8;      // the same for groups of 9..16 query heads (more registers per thread)
 constexpr int kAttnStageTokens = 16;   // tokens per pipeline stage (one PV MMA k-step)
@@ -61,8 +62,10 @@ WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& de
 // ---------------------------------------------------------------------------------------------
 // Kernel launchers (each returns the cudaError_t of its launches)
 // ---------------------------------------------------------------------------------------------
+// sched: two 32-bit counters, zero between launches, for the kernel's on-demand tile schedule (in a workspace they
+// sit kSchedWord words behind the status word)
 cudaError_t launch_index_scores_decode(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
-                                       uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+                                       uint32_t* status, uint32_t* sched, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
                                      uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,

@@ -314,3 +314,37 @@ def test_outputs_may_live_in_pinned_host_memory():
         assert g.status() == 0
         for l in range(g.L):
             assert torch.equal(host[l].view(torch.int16), dev_outs[l].cpu().view(torch.int16)), l
+
+
+def test_uncleared_workspace_header_is_flagged():
+    """The score kernel hands out part of its tiles through two counters in the workspace header, which every launch
+    leaves at zero. A header that was never cleared makes it skip tiles; it notices (a ticket beyond the last
+    possible one) and sets CLSA_DEV_BAD_WORKSPACE instead of returning wrong scores silently. After
+    clsa_clear_status the same workspace works."""
+    B, n = 5, 131072                                   # enough tiles for the on-demand part of the schedule
+    dev = torch.device("cuda:0")
+    gen = torch.Generator(device=dev).manual_seed(3)
+    kidx = torch.randn((B * n, 128), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    q = torch.randn((B, 1, 128), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    kv = torch.zeros((8, 8, 128), dtype=torch.bfloat16, device=dev)
+    seq_start = torch.arange(B, dtype=torch.int64, device=dev) * n   # the params hold raw pointers: keep these alive
+    seq_len = torch.full((B,), n, dtype=torch.int32, device=dev)
+    p = clsa.make_params(num_seqs=B, q_per_seq=1, num_q_heads=32, num_kv_heads=8, head_dim=128, idx_dim=128, top_k=64,
+                         num_layers=1, max_seq_len=n, sm_scale=0.1, seq_start=seq_start, seq_len=seq_len, k_cache=kv,
+                         v_cache=kv, idx_k_cache=kidx)
+    good_ws = torch.zeros(clsa.clsa_workspace_bytes(p), dtype=torch.uint8, device=dev)
+    want = torch.full((B, 1, n), float("nan"), dtype=torch.float32, device=dev)
+    clsa.clsa_index_scores(p, q, want, n, good_ws)
+    assert clsa.clsa_device_status(good_ws) == 0
+    ref = torch.einsum("bd,bnd->bn", q[:, 0].float(), kidx.view(B, n, 128).float())
+    assert (want[:, 0] - ref).abs().max().item() < 1e-3 * ref.abs().max().item()
+    assert good_ws[:256].count_nonzero().item() == 0                 # the counters are back at zero
+    bad_ws = torch.zeros_like(good_ws)
+    bad_ws[:256].view(torch.int32)[16] = 1 << 30                     # as if the header had never been cleared
+    got = torch.full_like(want, float("nan"))
+    clsa.clsa_index_scores(p, q, got, n, bad_ws)
+    assert clsa.clsa_device_status(bad_ws) & clsa.CLSA_DEV_BAD_WORKSPACE
+    clsa.clsa_clear_status(bad_ws)
+    clsa.clsa_index_scores(p, q, got, n, bad_ws)
+    assert clsa.clsa_device_status(bad_ws) == 0
+    assert torch.equal(got, want)
