@@ -348,3 +348,64 @@ def test_uncleared_workspace_header_is_flagged():
     clsa.clsa_index_scores(p, q, got, n, bad_ws)
     assert clsa.clsa_device_status(bad_ws) == 0
     assert torch.equal(got, want)
+
+
+@pytest.mark.parametrize("d_idx,paged", [(128, False), (64, False), (128, True), (64, True)])
+def test_score_kernel_on_demand_tiles_cover_every_row_once(d_idx, paged):
+    """Launches large enough for the on-demand part of the score kernel's schedule (ragged lengths, both indexer
+    widths, contiguous and paged caches): every visible position gets its score, nothing beyond it is written, a
+    second launch on the same workspace gives the same bits (the counters went back to zero), and the values match
+    a plain fp32 product."""
+    B, n_max = 24, 131072
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(11 + d_idx)
+    lens = rng.integers(1000, n_max + 1, B).astype(np.int32)
+    lens[:2] = (n_max, 1)
+    gen = torch.Generator(device=dev).manual_seed(5)
+    bs = 64
+    if paged:
+        blocks_per_seq = (n_max + bs - 1) // bs
+        nblocks = int(sum((int(x) + bs - 1) // bs for x in lens))
+        perm = torch.from_numpy(rng.permutation(nblocks).astype(np.int32))
+        table = torch.zeros((B, blocks_per_seq), dtype=torch.int32)
+        at = 0
+        for b in range(B):
+            nb = (int(lens[b]) + bs - 1) // bs
+            table[b, :nb] = perm[at: at + nb]
+            at += nb
+        rows = nblocks * bs
+        seq_start = torch.zeros(B, dtype=torch.int64, device=dev)
+        table_d = table.to(dev)
+    else:
+        starts = np.concatenate([[0], np.cumsum((lens.astype(np.int64) + 63) // 64 * 64)[:-1]])
+        rows = int(starts[-1] + lens[-1])
+        seq_start = torch.from_numpy(starts).to(dev)
+        table_d = None
+    kidx = torch.randn((rows, d_idx), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    q = torch.randn((B, 1, d_idx), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    kv = torch.zeros((8, 8, 128), dtype=torch.bfloat16, device=dev)
+    seq_len = torch.from_numpy(lens).to(dev)
+    p = clsa.make_params(num_seqs=B, q_per_seq=1, num_q_heads=32, num_kv_heads=8, head_dim=128, idx_dim=d_idx, top_k=64,
+                         num_layers=1, max_seq_len=n_max, sm_scale=0.1, seq_start=seq_start, seq_len=seq_len, k_cache=kv,
+                         v_cache=kv, idx_k_cache=kidx, block_table=table_d, block_size=bs if paged else 0)
+    ws = torch.zeros(clsa.clsa_workspace_bytes(p), dtype=torch.uint8, device=dev)
+    outs = []
+    for _ in range(2):
+        s = torch.full((B, 1, n_max), float("nan"), dtype=torch.float32, device=dev)
+        clsa.clsa_index_scores(p, q, s, n_max, ws)
+        outs.append(s)
+    assert clsa.clsa_device_status(ws) == 0
+    assert ws[:256].count_nonzero().item() == 0
+    assert torch.equal(outs[0].nan_to_num(nan=-7.0), outs[1].nan_to_num(nan=-7.0))
+    got = outs[0][:, 0]
+    for b in range(B):
+        n = int(lens[b])
+        if paged:
+            pos = torch.arange(n, device=dev)
+            r = table_d[b, pos // bs].long() * bs + pos % bs
+        else:
+            r = int(seq_start[b]) + torch.arange(n, device=dev)
+        ref = kidx[r].float() @ q[b, 0].float()
+        assert not torch.isnan(got[b, :n]).any(), b
+        assert torch.isnan(got[b, n:]).all(), b
+        assert (got[b, :n] - ref).abs().max().item() <= 1e-3 * max(1.0, ref.abs().max().item()), b
