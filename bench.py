@@ -620,6 +620,15 @@ def run_ours(args):
         roofline["achieved_in_step"] = gathered_per_layer / (in_step_us * 1e-6) / 1e9
         roofline["frac_in_step"] = roofline["achieved_in_step"] / peak
     roofline["traffic"] = profiled_traffic(c.name, "sparse_attn_kernel")
+    if breakdown is not None and T == 1:
+        # the step's other streaming kernel, as one event-timed public call (launch latency included)
+        key_bytes = int(w.seq_len.astype("int64").sum()) * c.idx_dim * 2
+        idx_gbs = key_bytes / (breakdown["index_scores"] * 1e-6) / 1e9
+        roofline["others"] = [{"kernel": "index_scores_decode_kernel (one event-timed call)", "bound": "hbm",
+                               "algorithmic_bytes_per_launch": key_bytes, "achieved": idx_gbs, "frac": idx_gbs / peak,
+                               "traffic": profiled_traffic(c.name, "index_scores_decode_kernel")},
+                              {"kernel": "topk_radix_kernel", "bound": "latency",
+                               "us": breakdown["topk"], "note": "cluster barriers and dependent sweeps, not bytes"}]
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
