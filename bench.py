@@ -442,13 +442,10 @@ def run_ours(args):
         out_list = outs if out_list is None else out_list
         if T == 1:
             clsa.clsa_decode_step(p, q_idx_t, q_list, out_list, idx, cnt, ws, stream=None)
-        else:  # a prefill chunk is not chained by the library: the three calls, in order
+        else:  # a prefill chunk: the scores (a GEMM here), the top-k, and the layers as one call
             clsa.clsa_index_scores(p, q_idx_t, chunk_scores, stride, ws, stream=None)
             clsa.clsa_topk(p, chunk_scores, stride, idx, cnt, ws, stream=None)
-            for l in range(L):
-                p.sweep = l & 1
-                clsa.clsa_sparse_attn(p, q_list[l], idx, cnt, out_list[l], None, ws, stream=None)
-            p.sweep = 0
+            clsa.clsa_sparse_attn_layers(p, q_list, idx, cnt, out_list, ws, stream=None)
 
     def step():
         run_step(t["q_idx"], q_layers)
