@@ -63,6 +63,18 @@ index_scores_decode_kernel(const uint16_t* __restrict__ kidx, int64_t tok_stride
         const int r = row0 + u * RPI + sub;
         kw[u] = r < n ? __ldcs(reinterpret_cast<const uint4*>(base + (int64_t)u * RPI * tok_stride)) : make_uint4(0, 0, 0, 0);
       }
+    } else if ((1 << block_shift) >= ROWS_PER_WARP) {
+      // paged cache whose blocks hold at least a warp's run of rows (which starts on a multiple of its length): the
+      // run lies in one block, so one lookup gives a base pointer and the loads are the strided ones of the contiguous
+      // layout (a lookup and a 64-bit product per load cost registers, and with them loads in flight)
+      const int32_t* table = block_table + (int64_t)b * max_blocks;
+      const int64_t blk = __ldg(table + (row0 >> block_shift));  // row0 < n: this block exists
+      const uint16_t* base = kidx + ((blk << block_shift) + ((row0 + sub) & ((1 << block_shift) - 1))) * tok_stride + col;
+#pragma unroll
+      for (int u = 0; u < kLoads; ++u) {
+        const int r = row0 + u * RPI + sub;
+        kw[u] = r < n ? __ldcs(reinterpret_cast<const uint4*>(base + (int64_t)u * RPI * tok_stride)) : make_uint4(0, 0, 0, 0);
+      }
     } else {
       // paged cache: position r lives in block table[b][r >> shift] at offset r & (block_size - 1)
       const int32_t* table = block_table + (int64_t)b * max_blocks;

@@ -350,10 +350,10 @@ def test_uncleared_workspace_header_is_flagged():
     assert torch.equal(got, want)
 
 
-@pytest.mark.parametrize("d_idx,paged", [(128, False), (64, False), (128, True), (64, True)])
+@pytest.mark.parametrize("d_idx,paged", [(128, 0), (64, 0), (128, 16), (64, 16), (64, 64)])
 def test_score_kernel_on_demand_tiles_cover_every_row_once(d_idx, paged):
     """Launches large enough for the on-demand part of the score kernel's schedule (ragged lengths, both indexer
-    widths, contiguous and paged caches): every visible position gets its score, nothing beyond it is written, a
+    widths, contiguous and paged caches -- blocks shorter and longer than a warp's run of rows): every visible position gets its score, nothing beyond it is written, a
     second launch on the same workspace gives the same bits (the counters went back to zero), and the values match
     a plain fp32 product."""
     B, n_max = 24, 131072
@@ -362,7 +362,7 @@ def test_score_kernel_on_demand_tiles_cover_every_row_once(d_idx, paged):
     lens = rng.integers(1000, n_max + 1, B).astype(np.int32)
     lens[:2] = (n_max, 1)
     gen = torch.Generator(device=dev).manual_seed(5)
-    bs = 64
+    bs = paged if paged else 64
     if paged:
         blocks_per_seq = (n_max + bs - 1) // bs
         nblocks = int(sum((int(x) + bs - 1) // bs for x in lens))
