@@ -91,9 +91,10 @@ typedef struct {
                            next kernel). 1: a few large blocks per launch (about 32), for launches that run side by
                            side with their neighbours on the stream, as the L layers of clsa_decode_step and
                            clsa_sparse_attn_layers do (whatever this field says). 2: as 1 with half the KV heads per
-                           block where that is possible (twice the blocks); the chained calls use it for their last few
-                           layers so that the chain's blocks keep every SM busy to the end. Results of the shapes
-                           agree to rounding (different split of the selected set), not bit for bit. */
+                           block where that is possible (twice the blocks); the chained calls use it for a tail of
+                           their work -- the last query rows of one layer and every layer behind it -- so that the
+                           chain's blocks keep every SM busy to the end. Results of the shapes agree to rounding
+                           (different split of the selected set), not bit for bit. */
   const int64_t* seq_start; /* [B] first cache row of each sequence */
   const int32_t* seq_len;   /* [B] valid tokens n_b >= T, including the T query tokens */
   const void* k_cache;      /* bf16 [rows][Hkv][D]; element (r,g,d) at r*kv_token_stride + g*kv_head_stride + d */
@@ -159,8 +160,8 @@ CLSA_API clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const
  *   q_layers   HOST array of L device pointers, each bf16 [B][T][Hq][D]
  *   out_layers HOST array of L device pointers, each bf16 [B][T][Hq][D]
  * Equivalent, bit for bit, to clsa_index_scores, clsa_topk and L calls of clsa_sparse_attn made one
- * after another with attn_plan = 1, or 2 for some number of the last layers (and the same p->sweep for every
- * layer). The layers do not wait for one
+ * after another with attn_plan = 1, or, for a tail of the (layer, query row) order, 2 (and the same p->sweep for
+ * every layer): each row of each layer's output is that of one of the two shapes. The layers do not wait for one
  * another (each reads only the index, the caches and its own queries), so several of them are in flight at once.
  * T > 1 is not chained here. */
 CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
@@ -172,7 +173,7 @@ CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, c
  * arrive on another stream while the routing runs, making `stream` wait on that upload just before this call.
  *   q_layers / out_layers  HOST arrays of L device pointers, each bf16 [B][T][Hq][D], 16-byte aligned
  *   idx, count             as written by clsa_topk (read only)
- * Bit for bit the L calls of clsa_sparse_attn with attn_plan = 1 (2 for some of the last layers, see attn_plan), the same p->sweep and lse = NULL, launched
+ * Bit for bit the L calls of clsa_sparse_attn with attn_plan = 1 (2 for a tail of the work, see attn_plan), the same p->sweep and lse = NULL, launched
  * so that a layer does not wait for its predecessor (which is why the calls are offered as one). */
 CLSA_API clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* const* q_layers, const int32_t* idx,
                                              const int32_t* count, void* const* out_layers, void* workspace,

@@ -111,11 +111,12 @@ clsa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? CLSA_OK : CLSA_
 // them in L2 (measured at the headline: 286 us per step against 320 us with alternating directions).
 cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, void* const* out_layers, const int32_t* idx,
                           const int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t s) {
-  const int fine_tail = chain_fine_tail(p, dev);  // the last layers use smaller blocks so that the chain ends flush
+  const ChainTail tail = chain_fine_tail(p, dev);  // the last layers use smaller blocks so that the chain ends flush
   for (int l = 0; l < p.num_layers; ++l) {
+    const bool fine = l >= p.num_layers - tail.layers;
+    const int fine_rows = l == p.num_layers - tail.layers - 1 ? tail.rows : 0;  // the layer where the finer shape begins
     const cudaError_t err = launch_sparse_attn(p, q_layers[l], idx, count, out_layers[l], nullptr, status, p.sweep & 1,
-                                               l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0,
-                                               l >= p.num_layers - fine_tail ? 2 : 1, dev, s);
+                                               l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0, fine ? 2 : 1, fine_rows, dev, s);
     if (err != cudaSuccess) return err;
   }
   return cudaSuccess;
@@ -186,7 +187,7 @@ clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t*
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
   return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, 1, 0,
-                                      p->attn_plan, dev,
+                                      p->attn_plan, 0, dev,
                                       static_cast<cudaStream_t>(stream)));
 }
 

@@ -39,9 +39,13 @@ struct AttnPlan {
 // neighbours on the stream); 2 = the same with half the KV heads per block, where that is possible (twice the
 // blocks: used for the last layers of a chain, see chain_fine_tail)
 AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int throughput);
-// How many of the last layers of an L-layer chain should use the finer shape (throughput = 2) so that the chain's
-// blocks fill the SMs evenly to the end.
-int chain_fine_tail(const clsa_params& p, const DeviceInfo& dev);
+// Which part of an L-layer chain should use the finer shape (throughput = 2) so that the chain's blocks fill the SMs
+// evenly to the end: the last `layers` layers entirely, and the last `rows` query rows of the layer before them.
+struct ChainTail {
+  int layers;
+  int rows;
+};
+ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev);
 
 struct TopkPlan {
   int cluster;      // blocks per (sequence, query) row, a thread-block cluster
@@ -75,7 +79,7 @@ cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int
                                   int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
-                               int throughput_plan, const DeviceInfo& dev, cudaStream_t stream);
+                               int throughput_plan, int fine_rows, const DeviceInfo& dev, cudaStream_t stream);
 
 cudaError_t launch_project_append(const clsa_params& p, int d_model, const void* h, const void* w_q_idx,
                                   const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,

@@ -69,6 +69,9 @@ struct AttnArgs {
   int off32;          // every row offset of the caches fits 32 bits when counted in 16-byte units
   int64_t rows_max;   // extent of the cache row space (off32 only): rows at or beyond it are refused like bad indices
   int keep;           // 1: the rows are fetched with the L2 evict_last priority (launches behind this one read them again)
+  int coarse_blocks;  // -1: one block size, 2-D grid. >= 0: a 1-D grid of two block sizes (no cluster, one row per block):
+                      // the first coarse_blocks blocks take heads_per_block KV heads each, row by row; the blocks behind
+                      // them take half as many (twice the token ranges) and cover the remaining rows
   float scale_log2;
 };
 
@@ -132,20 +135,38 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
 // WARPS = warps per block: 12 for NT = 1 (about 165 registers per thread), 8 for NT = 2.
 // MULTI: a block serves several query rows (rows_per_block > 1); the single-row instances keep the row uniform
 // over the block.
-template <int NT, bool PAGED, int WARPS, bool MULTI>
+// MIXED = the launch has two block sizes (AttnArgs::coarse_blocks); a variant of its own so that launches of one
+// size keep their block shape in kernel parameters, not registers.
+template <int NT, bool PAGED, int WARPS, bool MULTI, bool MIXED = false>
 __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   cg::cluster_group cluster = cg::this_cluster();
   const int C = (int)cluster.num_blocks();
   const int crank = (int)cluster.block_rank();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int HC = a.heads_per_block, S = a.subs, G = a.group;
+  int HC_ = a.heads_per_block, S_ = a.subs;
+  unsigned bx = blockIdx.x, by = blockIdx.y;
+  if (MIXED) {
+    const int hgc = (a.num_kv_heads + HC_ - 1) / HC_;  // coarse blocks per row
+    if ((int)blockIdx.x < a.coarse_blocks) {
+      bx = blockIdx.x / hgc;
+      by = blockIdx.x % hgc;
+    } else {
+      const int j = (int)blockIdx.x - a.coarse_blocks;
+      HC_ >>= 1;
+      S_ <<= 1;
+      const int hgf = (a.num_kv_heads + HC_ - 1) / HC_;  // fine blocks per row
+      bx = a.coarse_blocks / hgc + j / hgf;
+      by = j % hgf;
+    }
+  }
+  const int HC = HC_, S = S_, G = a.group;
   const int g_local = warp % HC;
   const int RB = MULTI ? a.rows_per_block : 1;
   const int row_local = MULTI ? (warp / HC) / S : 0;  // which of the block's rows
   const int sub = (warp / HC) - row_local * S;       // which of that row's token ranges
-  const int64_t r_true = (int64_t)(blockIdx.x / C) * RB + row_local;
-  const int g = blockIdx.y * HC + g_local;          // KV head of this warp
+  const int64_t r_true = (int64_t)(bx / C) * RB + row_local;
+  const int g = by * HC + g_local;                  // KV head of this warp
   const bool active = sub < S && row_local < RB && r_true < a.num_rows && g < a.num_kv_heads;
   const int64_t r = (!MULTI || r_true < a.num_rows) ? r_true : a.num_rows - 1;  // query row (clamped past the last row)
   const int nsplit = C * S;                         // token ranges of the row
@@ -196,7 +217,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
     }
   }
   if (cnt < 0 || cnt > a.top_k) {
-    if (lane == 0 && sub == 0 && g_local == 0 && crank == 0 && blockIdx.y == 0 && active) flag_status(a.status, CLSA_DEV_BAD_COUNT);
+    if (lane == 0 && sub == 0 && g_local == 0 && crank == 0 && by == 0 && active) flag_status(a.status, CLSA_DEV_BAD_COUNT);
     cnt = cnt < 0 ? 0 : a.top_k;
   }
   const int t_lo = min(cnt, slot_lo), t_hi = active ? min(cnt, slot_hi) : t_lo;
@@ -447,13 +468,13 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
   if (C == 1) __syncthreads(); else cluster.sync();
 
   // Output jobs (KV head of this block's group, query head of the group) dealt over the cluster's warps.
-  const int heads_here = min(HC, a.num_kv_heads - (int)blockIdx.y * HC);
+  const int heads_here = min(HC, a.num_kv_heads - (int)by * HC);
   const int jobs_per_row = heads_here * G;
   const int njobs = RB * jobs_per_row;
   const uint32_t smem_base = smem_u32(smem);
   for (int job = crank + C * warp; job < njobs; job += C * WARPS) {
     const int rl = MULTI ? job / jobs_per_row : 0;  // which of the block's rows
-    const int64_t r_job = (int64_t)(blockIdx.x / C) * RB + rl;
+    const int64_t r_job = (int64_t)(bx / C) * RB + rl;
     if (MULTI && r_job >= a.num_rows) continue;
     const int jrow = job - rl * jobs_per_row;
     const int jg = jrow / G, hh = jrow - jg * G;   // local KV head, query head within the group
@@ -507,7 +528,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
       }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
-    const int64_t item = r_job * a.num_q_heads + (int64_t)(blockIdx.y * HC + jg) * G + hh;
+    const int64_t item = r_job * a.num_q_heads + (int64_t)(by * HC + jg) * G + hh;
     uint2 packed;
     packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
     packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
@@ -628,42 +649,39 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
 // that round at a finer grain. How many layers: the schedule is simulated for every choice with a block's duration
 // modelled as a fixed part (launch gap, ramp, merge: 9.5 us measured) plus its bytes at the per-SM gather rate
 // (118 GB/s measured), and the best choice is taken if it gains at least 2 %. Cached per shape.
-int chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
+ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
+  ChainTail none = {0, 0};
   const int L = p.num_layers;
-  if (L < 2 || L > 256) return 0;
-  if (p.block_table != nullptr) return 0;  // paged caches: measured, the finer blocks cost more than the fuller last round returns
+  if (L < 2 || L > 256) return none;
+  if (p.block_table != nullptr) return none;  // paged caches: measured, the finer blocks cost more than the fuller last round returns
   const AttnPlan base = make_attn_plan(p, dev, 1), fine = make_attn_plan(p, dev, 2);
   if (base.cluster != 1 || fine.cluster != 1 || fine.heads_per_block == base.heads_per_block ||
-      fine.rows_per_block != base.rows_per_block)
-    return 0;
+      base.rows_per_block != 1 || fine.rows_per_block != 1)
+    return none;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
-  const int64_t nb_base = (rows + base.rows_per_block - 1) / base.rows_per_block * base.head_groups;
-  const int64_t nb_fine = (rows + fine.rows_per_block - 1) / fine.rows_per_block * fine.head_groups;
-  if (nb_base > 4096 || nb_fine > 8192) return 0;  // far more blocks than SMs: the last round is a small part of the whole
-  struct Key { int L, sms, k, hb, hf; int64_t nb, nf; int tail; };
+  const int64_t nb_base = rows * base.head_groups, nb_fine = rows * fine.head_groups;
+  if (nb_base > 4096 || nb_fine > 8192) return none;  // far more blocks than SMs: the last round is a small part of the whole
+  struct Key { int L, sms, k, hb, hf; int64_t rows; ChainTail tail; };
   static std::mutex mu;
   static Key seen[16];
   static int used = 0;
   std::lock_guard<std::mutex> lock(mu);
   for (int i = 0; i < used; ++i)
     if (seen[i].L == L && seen[i].sms == dev.sm_count && seen[i].k == p.top_k && seen[i].hb == base.heads_per_block &&
-        seen[i].hf == fine.heads_per_block && seen[i].nb == nb_base && seen[i].nf == nb_fine)
+        seen[i].hf == fine.heads_per_block && seen[i].rows == rows)
       return seen[i].tail;
   const double k_eff = (double)(p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len);
   auto duration = [&](const AttnPlan& pl) {  // microseconds
-    const double bytes = (double)pl.heads_per_block * pl.rows_per_block * k_eff * 512.0;
+    const double bytes = (double)pl.heads_per_block * k_eff * 512.0;
     return 9.5 + bytes / 118e3;
   };
   const double d_base = duration(base), d_fine = duration(fine);
   std::vector<double> heap((size_t)dev.sm_count);
-  auto makespan = [&](int tail) {
+  // layers [0, L - tail - 1) coarse; layer L - tail - 1 coarse except its last `part` rows; the last `tail` layers fine
+  auto makespan = [&](int tail, int64_t part) {
     std::fill(heap.begin(), heap.end(), 0.0);  // all equal: a valid min-heap (std::greater)
     double end = 0.0, gate = 0.0;
-    for (int l = 0; l < L; ++l) {
-      const bool f = l >= L - tail;
-      const int64_t nb = f ? nb_fine : nb_base;
-      const double d = f ? d_fine : d_base;
-      double last_start = gate;
+    auto place = [&](int64_t nb, double d, double& last_start) {
       for (int64_t j = 0; j < nb; ++j) {
         std::pop_heap(heap.begin(), heap.end(), std::greater<double>());
         const double t = std::max(heap.back(), gate);
@@ -672,25 +690,36 @@ int chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
         end = std::max(end, t + d);
         last_start = std::max(last_start, t);
       }
+    };
+    for (int l = 0; l < L; ++l) {
+      double last_start = gate;
+      if (l >= L - tail) place(nb_fine, d_fine, last_start);
+      else if (l == L - tail - 1 && part > 0) {
+        place((rows - part) * base.head_groups, d_base, last_start);
+        place(part * fine.head_groups, d_fine, last_start);
+      } else place(nb_base, d_base, last_start);
       gate = last_start;
     }
     return end;
   };
-  const double plain = makespan(0);
+  const double plain = makespan(0, 0);
   double best = plain;
-  int best_tail = 0;
-  for (int tail = 1; tail <= L; ++tail) {
-    const double m = makespan(tail);
-    if (m < best - 1e-9) { best = m; best_tail = tail; }
-  }
-  if (best > 0.98 * plain) best_tail = 0;
-  if (used < 16) seen[used++] = Key{L, dev.sm_count, p.top_k, base.heads_per_block, fine.heads_per_block, nb_base, nb_fine, best_tail};
+  ChainTail best_tail = none;
+  const int64_t step = rows >= 8 ? rows / 8 : 1;  // partial layers in eighths of the rows
+  for (int tail = 0; tail < L; ++tail)
+    for (int64_t part = 0; part < rows; part += step) {
+      if (tail == 0 && part == 0) continue;
+      const double m = makespan(tail, part);
+      if (m < best - 1e-9) { best = m; best_tail = ChainTail{tail, (int)part}; }
+    }
+  if (best > 0.98 * plain) best_tail = none;
+  if (used < 16) seen[used++] = Key{L, dev.sm_count, p.top_k, base.heads_per_block, fine.heads_per_block, rows, best_tail};
   return best_tail;
 }
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
-                               int throughput_plan, const DeviceInfo& dev, cudaStream_t stream) {
+                               int throughput_plan, int fine_rows, const DeviceInfo& dev, cudaStream_t stream) {
   const AttnPlan plan = make_attn_plan(p, dev, throughput_plan);
   AttnArgs a;
   a.q = static_cast<const uint16_t*>(q);
@@ -724,6 +753,7 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   // fetches all of them with evict_last, so that scores, indices and outputs passing through L2 do not push them
   // out before the layers behind it arrive; a launch on its own leaves the replacement policy alone.
   a.keep = keep_for_next ? 1 : 0;
+  a.coarse_blocks = -1;
   a.scale_log2 = p.sm_scale * kLog2e;
   // With the extent of the row space known (num_cache_rows) and below 2^32 16-byte units, row offsets are 32-bit.
   a.rows_max = p.num_cache_rows;
@@ -737,11 +767,26 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   else if (plan.warps == kAttnWarpsNarrow) kernel = CLSA_ATTN_PICK(1, kAttnWarpsNarrow);
   else kernel = CLSA_ATTN_PICK(1, kAttnWarpsWide);
 #undef CLSA_ATTN_PICK
+  const bool can_mix = a.group <= 8 && !multi && !pg;  // the shapes a chain's partly finer layer can have
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((rows + plan.rows_per_block - 1) / plan.rows_per_block * plan.cluster), (unsigned)plan.head_groups, 1);
+  // Two block sizes in one launch (the layer of a chain where the finer shape begins, see chain_fine_tail): the
+  // last fine_rows rows get blocks of half the KV heads. Only where the plan allows it; otherwise one size.
+  if (can_mix && throughput_plan == 1 && fine_rows > 0 && fine_rows < rows && plan.cluster == 1 &&
+      plan.rows_per_block == 1 && plan.heads_per_block > 1) {
+    kernel = plan.warps == kAttnWarpsNarrow ? sparse_attn_kernel<1, false, kAttnWarpsNarrow, false, true>
+                                            : sparse_attn_kernel<1, false, kAttnWarpsWide, false, true>;
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
+    if (err != cudaSuccess) return err;
+    const int hc_fine = plan.heads_per_block / 2;
+    const int64_t coarse = (rows - fine_rows) * plan.head_groups;
+    const int64_t fine = (int64_t)fine_rows * ((p.num_kv_heads + hc_fine - 1) / hc_fine);
+    a.coarse_blocks = (int)coarse;
+    cfg.gridDim = dim3((unsigned)(coarse + fine), 1, 1);
+  }
   cfg.blockDim = dim3((unsigned)plan.warps * 32, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
