@@ -111,7 +111,7 @@ clsa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? CLSA_OK : CLSA_
 // them in L2 (measured at the headline: 286 us per step against 320 us with alternating directions).
 cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, void* const* out_layers, const int32_t* idx,
                           const int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t s) {
-  const ChainTail tail = chain_fine_tail(p, dev);  // the last layers use smaller blocks so that the chain ends flush
+  const ChainTail tail = chain_fine_tail(p, dev);  // the end of the chain uses smaller blocks so that it ends flush
   for (int l = 0; l < p.num_layers; ++l) {
     const bool fine = l >= p.num_layers - tail.layers;
     const int fine_rows = l == p.num_layers - tail.layers - 1 ? tail.rows : 0;  // the layer where the finer shape begins

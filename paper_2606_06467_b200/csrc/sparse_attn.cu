@@ -645,10 +645,11 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
 // The layers of a chain are launched back to back and none waits for its predecessor, so their blocks fill the
 // SMs like a list schedule: a block starts when an SM frees up, and a layer's blocks are placed only once the layer
 // before it has started all of its own. With equal blocks the last round is usually part empty (16 layers of 32
-// blocks on 148 SMs: 3.46 rounds, the fourth with 68 blocks). Blocks of half the size in the last few layers fill
-// that round at a finer grain. How many layers: the schedule is simulated for every choice with a block's duration
-// modelled as a fixed part (launch gap, ramp, merge: 9.5 us measured) plus its bytes at the per-SM gather rate
-// (118 GB/s measured), and the best choice is taken if it gains at least 2 %. Cached per shape.
+// blocks on 148 SMs: 3.46 rounds, the fourth with 68 blocks). Blocks of half the size at the end of the chain --
+// the last query rows of one layer and every layer behind it -- fill that round at a finer grain. Where the finer
+// shape begins: the schedule is simulated for every choice (whole layers, and eighths of the rows of the layer before
+// them) with a block's duration modelled as a fixed part (launch gap, ramp, merge: 9.5 us measured) plus its bytes at
+// the per-SM gather rate (118 GB/s measured), and the best choice is taken if it gains at least 2 %. Cached per shape.
 ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
   ChainTail none = {0, 0};
   const int L = p.num_layers;
