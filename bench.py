@@ -295,9 +295,7 @@ def compare_baselines(clsa, torch, w, t, p, ws, idx, cnt, q_layers, outs, flush,
         for l in range(L):
             clsa.clsa_index_scores(p, t["q_idx"], scores, stride, ws, stream=stream)
             clsa.clsa_topk(p, scores, stride, idx, cnt, ws, stream=stream)
-            p.sweep = l & 1
-            clsa.clsa_sparse_attn(p, q_layers[l], idx, cnt, outs[l], None, ws, stream=stream)
-        p.sweep = 0
+            clsa.clsa_sparse_attn_hinted(p, q_layers[l], idx, cnt, outs[l], None, clsa.make_hints(reverse=l & 1), ws, stream=stream)
 
     unamortised_ms = timed(per_layer_routing)
     # dense: every position selected
@@ -308,11 +306,11 @@ def compare_baselines(clsa, torch, w, t, p, ws, idx, cnt, q_layers, outs, flush,
     all_idx = torch.arange(n, dtype=torch.int32, device=idx.device).repeat(B, 1).reshape(B, 1, n)
     all_idx = torch.where(all_idx < t["seq_len"].reshape(B, 1, 1), all_idx, torch.full_like(all_idx, -1))
     all_cnt = t["seq_len"].reshape(B, 1).to(torch.int32).contiguous()
+    ws_dense = torch.zeros(clsa.clsa_workspace_bytes(pd), dtype=torch.uint8, device=idx.device)
 
     def dense_layers():
         for l in range(L):
-            pd.sweep = l & 1
-            clsa.clsa_sparse_attn(pd, q_layers[l], all_idx, all_cnt, outs[l], None, ws, stream=stream)
+            clsa.clsa_sparse_attn_hinted(pd, q_layers[l], all_idx, all_cnt, outs[l], None, clsa.make_hints(reverse=l & 1), ws_dense, stream=stream)
 
     dense_ms = timed(dense_layers, reps=2)
     return {
@@ -329,7 +327,7 @@ def compare_baselines(clsa, torch, w, t, p, ws, idx, cnt, q_layers, outs, flush,
 
 
 # --------------------------------------------------------------------------------------- CUDA arm
-def time_projection(clsa, torch, w, p, ws, dev):
+def time_projection(clsa, torch, w, t, p, ws, dev):
     """clsa_project_append alone: the weights of Eq. 2 (and of the shared K/V rows) streamed once against the
     B*T newest hidden states. One launch lasts a few microseconds, below what a pair of events resolves, so 8
     launches are captured in a CUDA graph, once back to back (weights stay in L2: warm) and once each behind an
@@ -340,7 +338,8 @@ def time_projection(clsa, torch, w, p, ws, dev):
     scrub = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     def call():
-        clsa.clsa_project_append(p, c.d_model, proj["h"], proj["w_q_idx"], proj["w_k_idx"], proj["w_k"], proj["w_v"], q, ws)
+        clsa.clsa_project_append(p, c.d_model, proj["h"], proj["w_q_idx"], proj["w_k_idx"], proj["w_k"], proj["w_v"], q,
+                                 t["idx_k_cache"], t["k_cache"], t["v_cache"], ws)
 
     def flush():
         scrub.fill_(1)
@@ -581,10 +580,9 @@ def run_ours(args):
             clsa.clsa_topk(p, scores, stride, idx, cnt, ws, stream=stream)
             marks[2].record(stream)
             for l in range(L):           # L public calls back to back, no event between them
-                p.sweep = l & 1
-                clsa.clsa_sparse_attn(p, q_layers[l], idx, cnt, outs[l], None, ws, stream=stream)
+                clsa.clsa_sparse_attn_hinted(p, q_layers[l], idx, cnt, outs[l], None,
+                                             clsa.make_hints(reverse=l & 1, keep_rows=l + 1 < L, only_q_pending=l > 0), ws, stream=stream)
             marks[3].record(stream)
-            p.sweep = 0
             torch.cuda.synchronize()
             if i >= 2:
                 acc["index_scores"] += marks[0].elapsed_time(marks[1])
@@ -650,7 +648,7 @@ def run_ours(args):
 
     projection = None
     if args.project and rank == 0 and world == 1:   # last: it overwrites the newest rows of the caches
-        projection = time_projection(clsa, torch, w, p, ws, dev)
+        projection = time_projection(clsa, torch, w, t, p, ws, dev)
 
     if rank == 0:
         line = {

@@ -83,18 +83,9 @@ typedef struct {
   int32_t num_layers;   /* L >= 1; read by clsa_decode_step and clsa_workspace_bytes only */
   int32_t causal;       /* 0 or 1, see "Visibility" */
   int32_t max_seq_len;  /* host-known upper bound of seq_len[], used for grid sizing (no device read-back) */
-  float sm_scale;       /* softmax scale of Eq. 4's Attn, > 0; 1/sqrt(head_dim) in the benchmarks */
-  int32_t sweep;        /* 0 or 1: direction in which clsa_sparse_attn walks the selected set; a cache-locality
-                           hint only (results agree to rounding). clsa_decode_step walks every layer in this direction */
-  int32_t attn_plan;    /* launch shape of clsa_sparse_attn. 0: the whole GPU on this one launch (shortest time for a
-                           launch that has to finish before anything else can run -- a layer whose output feeds the
-                           next kernel). 1: a few large blocks per launch (about 32), for launches that run side by
-                           side with their neighbours on the stream, as the L layers of clsa_decode_step and
-                           clsa_sparse_attn_layers do (whatever this field says). 2: as 1 with half the KV heads per
-                           block where that is possible (twice the blocks); the chained calls use it for a tail of
-                           their work -- the last query rows of one layer and every layer behind it -- so that the
-                           chain's blocks keep every SM busy to the end. Results of the shapes agree to rounding
-                           (different split of the selected set), not bit for bit. */
+  float sm_scale;       /* softmax scale of Eq. 4's Attn; finite and > 0 (the kernels take running maxima over the raw
+                           dot products, which is only valid for a positive scale; other values are refused with
+                           CLSA_ERR_INVALID_ARG); 1/sqrt(head_dim) in the benchmarks */
   const int64_t* seq_start; /* [B] first cache row of each sequence */
   const int32_t* seq_len;   /* [B] valid tokens n_b >= T, including the T query tokens */
   const void* k_cache;      /* bf16 [rows][Hkv][D]; element (r,g,d) at r*kv_token_stride + g*kv_head_stride + d */
@@ -116,11 +107,13 @@ typedef struct {
   int32_t max_blocks_per_seq; /* >= ceil(max_seq_len / block_size) (paged only) */
 } clsa_params;
 
-/* Bytes of workspace that any of the calls below may need for these params (the maximum over the
- * four; clsa_decode_step additionally keeps the fp32 score matrix there). Reads only the scalar
- * fields. *bytes is HOST memory. The workspace must be 256-byte aligned; its first 256 bytes hold
- * the device status word and the score kernel's scheduling counters (which every launch leaves at
- * zero) and must be zero before the first call (cudaMemset or clsa_clear_status).
+/* Bytes of workspace that any of the calls below may need for these params (the maximum over them:
+ * the status header, the scratch through which a standalone decode clsa_sparse_attn merges the
+ * partial results of its blocks -- arrival counters and partial slots -- and the fp32 score matrix
+ * that clsa_decode_step keeps there). Reads only the scalar fields. *bytes is HOST memory. The workspace must be 256-byte aligned
+ * and ALL of it zero before the first call (cudaMemset): its first 256 bytes hold the device status
+ * word and the score kernel's scheduling counters, the attention scratch begins with arrival counters;
+ * every launch leaves all of these counters at zero again, and clsa_clear_status zeroes the status word.
  * Calls that overlap on the GPU must not share a workspace. */
 CLSA_API clsa_status clsa_workspace_bytes(const clsa_params* p, size_t* bytes);
 
@@ -151,19 +144,52 @@ CLSA_API clsa_status clsa_topk(const clsa_params* p, const float* scores, int64_
  *   q   bf16 [B][T][Hq][D]           this layer's queries, 16-byte aligned
  *   out bf16 [B][T][Hq][D]           round-to-nearest-even from fp32 accumulators
  *   lse fp32 [B][T][Hq] or NULL      log-sum-exp of the scaled logits (natural log)
- * A (b,t) with count 0 yields zeros and lse = -inf. */
+ * A (b,t) with count 0 yields zeros and lse = -inf. A sequence with seq_len < T or > max_seq_len is treated as
+ * count 0 and flags CLSA_DEV_BAD_SEQLEN (its index entries are never used as addresses).
+ * The launch assumes nothing about what runs before it on the stream and waits for it; it has the whole GPU to
+ * itself (the shape for a layer whose output feeds the next kernel). Needs the whole workspace of
+ * clsa_workspace_bytes when T == 1 (such launches merge the partial results of their blocks through it). */
 CLSA_API clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t* idx, const int32_t* count,
                              void* out, float* lse, void* workspace, size_t workspace_bytes, clsa_stream stream);
+
+/* What a caller knows about the launches around one clsa_sparse_attn call. Hints select the launch shape and the
+ * order of memory accesses; they never change what is computed (results of different hints agree to rounding: the
+ * selected set is split differently), and all-zero hints are always valid. */
+typedef struct {
+  int32_t reverse;        /* 0 or 1: walk the selected set from its end. A decoder that issues its layers one by one
+                             alternates this from layer to layer, so that a layer starts on the rows its predecessor
+                             fetched last (still in L2). */
+  int32_t shared_gpu;     /* 0: the launch has the GPU to itself (the work is cut at token granularity over all SMs).
+                             1: it runs side by side with its neighbours on the stream (launches that do not wait for
+                             one another, as the L layers of clsa_decode_step): a few large blocks, about 32 per launch.
+                             2: as 1 with half the KV heads per block where that is possible (twice the blocks); the
+                             chained calls use it for a tail of their work so that the chain's blocks keep every SM
+                             busy to the end (see clsa_chain_plan). */
+  int32_t keep_rows;      /* 1: another launch that reads the same selected rows follows (the next layer): fetch them
+                             with the L2 evict_last priority so that other traffic does not push them out in between. */
+  int32_t only_q_pending; /* 1: idx, count, seq_len, the block table and the caches were all complete before the kernel
+                             in front of this call on the stream was launched; only q may still be in the making
+                             (every layer of a decoder after the first). The row copies then start before the launch
+                             waits for that kernel. Setting it when the index is still being written reads a stale
+                             index. */
+} clsa_attn_hints;
+
+/* clsa_sparse_attn with hints (NULL = all zero = clsa_sparse_attn). */
+CLSA_API clsa_status clsa_sparse_attn_hinted(const clsa_params* p, const void* q, const int32_t* idx, const int32_t* count,
+                                    void* out, float* lse, const clsa_attn_hints* hints, void* workspace,
+                                    size_t workspace_bytes, clsa_stream stream);
 
 /* One step (Sec. 2.1: the routing index is computed once and shared by the layers): index scores, TopK, then L
  * sparse-attention launches on `stream`, all fed the same idx/count, which are returned.
  *   q_layers   HOST array of L device pointers, each bf16 [B][T][Hq][D]
  *   out_layers HOST array of L device pointers, each bf16 [B][T][Hq][D]
- * Equivalent, bit for bit, to clsa_index_scores, clsa_topk and L calls of clsa_sparse_attn made one
- * after another with attn_plan = 1, or, for a tail of the (layer, query row) order, 2 (and the same p->sweep for
- * every layer): each row of each layer's output is that of one of the two shapes. The layers do not wait for one
- * another (each reads only the index, the caches and its own queries), so several of them are in flight at once.
- * T > 1 is not chained here. */
+ * Equivalent, bit for bit, to clsa_index_scores, clsa_topk and L calls of clsa_sparse_attn_hinted made one after
+ * another with hints {reverse 0, shared_gpu 1 or -- for the tail of the (layer, query row) order that clsa_chain_plan
+ * reports -- 2, keep_rows 1 except for the last layer}: each row of each layer's output is that of one of the two
+ * shapes. The layers do not wait for one another (each reads only the index, the caches and its own queries, all of which the caller
+ * hands over up front), so several of them are in flight at once and share the selected rows through L2. A decoder
+ * whose layer l+1 queries depend on layer l's output cannot use this call: it issues clsa_index_scores, clsa_topk
+ * and one clsa_sparse_attn_hinted per layer instead. T > 1 is not chained here. */
 CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
                              void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
                              size_t workspace_bytes, clsa_stream stream);
@@ -173,8 +199,8 @@ CLSA_API clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, c
  * arrive on another stream while the routing runs, making `stream` wait on that upload just before this call.
  *   q_layers / out_layers  HOST arrays of L device pointers, each bf16 [B][T][Hq][D], 16-byte aligned
  *   idx, count             as written by clsa_topk (read only)
- * Bit for bit the L calls of clsa_sparse_attn with attn_plan = 1 (2 for a tail of the work, see attn_plan), the same p->sweep and lse = NULL, launched
- * so that a layer does not wait for its predecessor (which is why the calls are offered as one). */
+ * Bit for bit the L calls of clsa_sparse_attn_hinted with the hints given under clsa_decode_step and lse = NULL,
+ * launched so that a layer does not wait for its predecessor (which is why the calls are offered as one). */
 CLSA_API clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* const* q_layers, const int32_t* idx,
                                              const int32_t* count, void* const* out_layers, void* workspace,
                                              size_t workspace_bytes, clsa_stream stream);
@@ -190,13 +216,16 @@ CLSA_API clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* c
  *   w_q_idx, w_k_idx  bf16 [d_idx][d_model]: one OUTPUT feature per row (y[o] = sum_j h[j] * w[o][j]), 16-byte aligned
  *   w_k, w_v bf16 [Hkv*D][d_model], feature g*D + d is element d of KV head g; both NULL = indexer branch only
  *   q_idx_out bf16 [B][T][d_idx], 16-byte aligned
- * THIS CALL WRITES the caches named by p (idx_k_cache, and k_cache/v_cache when w_k is given) although clsa_params
- * declares them const: exactly the rows above, nothing else. seq_len must already count the new tokens. Calls that
+ *   idx_k_cache_out          the K_idx cache, writable: same address, layout and paging as p->idx_k_cache describes
+ *   k_cache_out, v_cache_out the K and V caches, writable (both NULL together with w_k and w_v)
+ * The call writes exactly the cache rows above through these three pointers and nothing else; p's own (const) cache
+ * pointers are not written through and need not be set. seq_len must already count the new tokens. Calls that
  * follow on the same stream (clsa_index_scores, clsa_decode_step) see the appended rows. A sequence with
  * seq_len < T or > max_seq_len is skipped and flags CLSA_DEV_BAD_SEQLEN. Built for decoding (B*T up to a few
  * dozen rows, where the op is a stream of the weights); larger B*T works but re-reads the weights per 64 rows. */
 CLSA_API clsa_status clsa_project_append(const clsa_params* p, int32_t d_model, const void* h, const void* w_q_idx,
                                          const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,
+                                         void* idx_k_cache_out, void* k_cache_out, void* v_cache_out,
                                          void* workspace, size_t workspace_bytes, clsa_stream stream);
 
 /* The same step as clsa_decode_step for callers that cannot allocate device memory. (The paper has
@@ -204,25 +233,47 @@ CLSA_API clsa_status clsa_project_append(const clsa_params* p, int32_t d_model, 
  * workspace: code that runs inside a region where cudaMalloc is forbidden or would synchronise the
  * device (a latency-critical serving loop, a plug-in that is handed tensors but no allocator, a
  * process whose memory pool is already fully reserved). For them the scratch that clsa_decode_step
- * keeps in the caller's workspace -- the status word and the fp32 score matrix -- lives in a
- * device array built into the library: 8 MiB + 256 bytes per GPU that loads the library, held until
+ * keeps in the caller's workspace -- the status header and the fp32 score matrix (the chained
+ * attention launches need none of the scratch that a standalone clsa_sparse_attn does) -- lives in a
+ * device array built into the library: 16 MiB + 256 bytes per GPU that loads the library, held until
  * the process exits. This entry point calls no cudaMalloc, cudaFree or any other allocating routine.
- *   Limit: num_seqs * round_up(max_seq_len, 64) <= 2 097 152 scores (for example 16 sequences of
- *     131 072 tokens); larger shapes return CLSA_ERR_WORKSPACE and launch nothing. T must be 1.
+ *   Limit: clsa_workspace_bytes(p) <= 16 MiB + 256 bytes (for example 16 sequences of 131 072 tokens
+ *     with 32/8 heads: 8 MiB of scores behind 4.3 MiB of attention scratch that this entry point
+ *     leaves unused); larger shapes return CLSA_ERR_WORKSPACE and launch nothing. T must be 1.
  *   dev_status: DEVICE pointer to one uint32 owned by the caller that receives the CLSA_DEV_* bits
- *     (the caller zeroes it), or NULL to drop them into the built-in array's own word, which the
- *     call then clears first.
+ *     (the caller zeroes it), or NULL to drop them into the built-in array's own word.
  *   First call on a device: looks up the array's device address (once per device, with that device
  *     current). Make this first call outside any stream capture.
  *   Sharing: every call on a GPU uses the same array, which still holds the previous call's
- *     scores. Nothing needs to be cleared between calls except the status word, which the call does
- *     itself; but two calls whose GPU work overlaps (different streams, or different threads) race
- *     on the scores and give wrong indices. Serialise them, or use clsa_decode_step with one
- *     workspace per stream.
- * All other arguments, results and error behaviour are those of clsa_decode_step. */
+ *     contents. Every call begins by zeroing the array's header (status word and scheduling
+ *     counters) on `stream`, so a call that was cut short (or two calls that raced) cannot poison
+ *     later ones; the scores need no clearing (every entry that is read is written first). Two calls whose GPU work overlaps
+ *     (different streams, or different threads) race on the array and give wrong results for those
+ *     calls. Serialise them, or use clsa_decode_step with one workspace per stream.
+ * All other arguments, results and error behaviour are those of clsa_decode_step, with which the
+ * results agree bit for bit. */
 CLSA_API clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, const void* const* q_layers,
                                              void* const* out_layers, int32_t* idx, int32_t* count,
                                              uint32_t* dev_status, clsa_stream stream);
+
+/* Measurement aid (the paper has no counterpart): the memory accesses of one decode clsa_sparse_attn launch -- the
+ * same split of the selected set over the SMs, the same 16-byte asynchronous copies of K and V rows into the same
+ * shared-memory ring -- with the arithmetic, the queries and the outputs left out. Timing it on rows that are, or
+ * are not, resident in L2 gives the rate the memory system delivers to this access pattern, the ceiling that the
+ * attention kernel is measured against. T must be 1. hints as for clsa_sparse_attn_hinted (NULL = all zero;
+ * shared_gpu and only_q_pending are ignored: the probe is the shape of a launch that has the GPU to itself). Writes only into the workspace (which must be the whole clsa_workspace_bytes). */
+CLSA_API clsa_status clsa_gather_probe(const clsa_params* p, const int32_t* idx, const int32_t* count,
+                                       const clsa_attn_hints* hints, void* workspace, size_t workspace_bytes,
+                                       clsa_stream stream);
+
+/* Host only, no CUDA call: which part of an L-layer chain (clsa_decode_step, clsa_sparse_attn_layers) uses the finer
+ * launch shape (shared_gpu = 2) on a device with `sm_count` SMs and a peak SM clock of `clock_khz`: the last
+ * *fine_layers layers entirely and the last *fine_rows query rows of the layer before them (both 0: one shape
+ * throughout; always so for T > 1, for paged caches and for devices the block model was not measured on). The choice
+ * comes from a model of how the chain's blocks fill the SMs; it costs a few microseconds the first time a shape is
+ * seen and is remembered afterwards. Outputs are HOST pointers. */
+CLSA_API clsa_status clsa_chain_plan(const clsa_params* p, int32_t sm_count, int32_t clock_khz, int32_t* fine_layers,
+                                     int32_t* fine_rows);
 
 /* Zero the status word (asynchronous, on `stream`). */
 CLSA_API clsa_status clsa_clear_status(void* workspace, size_t workspace_bytes, clsa_stream stream);

@@ -32,8 +32,7 @@ class clsa_params(ctypes.Structure):
         ("num_seqs", ctypes.c_int32), ("q_per_seq", ctypes.c_int32), ("num_q_heads", ctypes.c_int32),
         ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("idx_dim", ctypes.c_int32),
         ("top_k", ctypes.c_int32), ("num_layers", ctypes.c_int32), ("causal", ctypes.c_int32),
-        ("max_seq_len", ctypes.c_int32), ("sm_scale", ctypes.c_float), ("sweep", ctypes.c_int32),
-        ("attn_plan", ctypes.c_int32),
+        ("max_seq_len", ctypes.c_int32), ("sm_scale", ctypes.c_float),
         ("seq_start", ctypes.c_void_p), ("seq_len", ctypes.c_void_p),
         ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
         ("kv_token_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64),
@@ -42,30 +41,41 @@ class clsa_params(ctypes.Structure):
     ]
 
 
+class clsa_attn_hints(ctypes.Structure):
+    """Mirror of `clsa_attn_hints` in include/clsa.h."""
+
+    _fields_ = [("reverse", ctypes.c_int32), ("shared_gpu", ctypes.c_int32), ("keep_rows", ctypes.c_int32),
+                ("only_q_pending", ctypes.c_int32)]
+
+
 _P = ctypes.POINTER(clsa_params)
+_H = ctypes.POINTER(clsa_attn_hints)
 _vp, _i64, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
 _lib.clsa_workspace_bytes.argtypes = [_P, ctypes.POINTER(_sz)]
 _lib.clsa_index_scores.argtypes = [_P, _vp, _vp, _i64, _vp, _sz, _vp]
 _lib.clsa_topk.argtypes = [_P, _vp, _i64, _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_sparse_attn.argtypes = [_P, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.clsa_sparse_attn_hinted.argtypes = [_P, _vp, _vp, _vp, _vp, _vp, _H, _vp, _sz, _vp]
+_lib.clsa_gather_probe.argtypes = [_P, _vp, _vp, _H, _vp, _sz, _vp]
 _lib.clsa_decode_step.argtypes = [_P, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_decode_step_static.argtypes = [_P, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _vp, _vp, _vp]
 _lib.clsa_sparse_attn_layers.argtypes = [_P, ctypes.POINTER(_vp), _vp, _vp, ctypes.POINTER(_vp), _vp, _sz, _vp]
-_lib.clsa_project_append.argtypes = [_P, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.clsa_project_append.argtypes = [_P, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.clsa_chain_plan.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
 _lib.clsa_clear_status.argtypes = [_vp, _sz, _vp]
 _lib.clsa_device_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32), _vp]
 _lib.clsa_status_string.argtypes = [ctypes.c_int]
 _lib.clsa_status_string.restype = ctypes.c_char_p
 _lib.clsa_version.restype = ctypes.c_int
-for _name in ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_decode_step",
-              "clsa_decode_step_static", "clsa_sparse_attn_layers", "clsa_project_append", "clsa_clear_status",
-              "clsa_device_status"):
+for _name in ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_sparse_attn_hinted",
+              "clsa_gather_probe", "clsa_decode_step", "clsa_decode_step_static", "clsa_sparse_attn_layers",
+              "clsa_project_append", "clsa_chain_plan", "clsa_clear_status", "clsa_device_status"):
     getattr(_lib, _name).restype = ctypes.c_int
 
-EXPORTS = ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_decode_step",
-           "clsa_decode_step_static", "clsa_sparse_attn_layers", "clsa_project_append", "clsa_clear_status",
-           "clsa_device_status",
-           "clsa_status_string", "clsa_version")
+EXPORTS = ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_sparse_attn_hinted",
+           "clsa_gather_probe", "clsa_decode_step", "clsa_decode_step_static", "clsa_sparse_attn_layers",
+           "clsa_project_append", "clsa_chain_plan", "clsa_clear_status", "clsa_device_status", "clsa_status_string",
+           "clsa_version")
 
 
 class ClsaError(RuntimeError):
@@ -105,7 +115,7 @@ def _nbytes(ws, ws_bytes):
 
 
 def make_params(*, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim=128, idx_dim, top_k, num_layers=1,
-                causal=0, max_seq_len, sm_scale, sweep=0, attn_plan=0, seq_start=None, seq_len=None, k_cache=None, v_cache=None,
+                causal=0, max_seq_len, sm_scale, seq_start=None, seq_len=None, k_cache=None, v_cache=None,
                 kv_token_stride=None, kv_head_stride=None, idx_k_cache=None, idx_token_stride=None,
                 num_cache_rows=None, block_table=None, block_size=0, max_blocks_per_seq=None) -> clsa_params:
     """Fill a clsa_params. Tensor arguments contribute their device address (and, for the caches, their strides
@@ -113,7 +123,7 @@ def make_params(*, num_seqs, q_per_seq=1, num_q_heads, num_kv_heads, head_dim=12
     p = clsa_params()
     p.num_seqs, p.q_per_seq, p.num_q_heads, p.num_kv_heads = num_seqs, q_per_seq, num_q_heads, num_kv_heads
     p.head_dim, p.idx_dim, p.top_k, p.num_layers, p.causal = head_dim, idx_dim, top_k, num_layers, causal
-    p.max_seq_len, p.sm_scale, p.sweep, p.attn_plan = max_seq_len, sm_scale, sweep, attn_plan
+    p.max_seq_len, p.sm_scale = max_seq_len, sm_scale
     p.seq_start, p.seq_len = _ptr(seq_start), _ptr(seq_len)
     p.k_cache, p.v_cache, p.idx_k_cache = _ptr(k_cache), _ptr(v_cache), _ptr(idx_k_cache)
     if kv_token_stride is None and k_cache is not None and not isinstance(k_cache, int):
@@ -156,6 +166,23 @@ def clsa_sparse_attn(p, q, idx, count, out, lse, workspace, workspace_bytes=None
            "clsa_sparse_attn")
 
 
+def make_hints(reverse=0, shared_gpu=0, keep_rows=0, only_q_pending=0) -> clsa_attn_hints:
+    return clsa_attn_hints(int(reverse), int(shared_gpu), int(keep_rows), int(only_q_pending))
+
+
+def clsa_sparse_attn_hinted(p, q, idx, count, out, lse, hints, workspace, workspace_bytes=None, stream=None) -> None:
+    """clsa_sparse_attn with a clsa_attn_hints (or None): launch shape and access order, never the result."""
+    _check(_lib.clsa_sparse_attn_hinted(ctypes.byref(p), _ptr(q), _ptr(idx), _ptr(count), _ptr(out), _ptr(lse),
+                                        None if hints is None else ctypes.byref(hints), _ptr(workspace),
+                                        _nbytes(workspace, workspace_bytes), _stream(stream)), "clsa_sparse_attn_hinted")
+
+
+def clsa_gather_probe(p, idx, count, hints, workspace, workspace_bytes=None, stream=None) -> None:
+    """Measurement aid: the memory accesses of one decode attention launch without its arithmetic."""
+    _check(_lib.clsa_gather_probe(ctypes.byref(p), _ptr(idx), _ptr(count), None if hints is None else ctypes.byref(hints),
+                                  _ptr(workspace), _nbytes(workspace, workspace_bytes), _stream(stream)), "clsa_gather_probe")
+
+
 def clsa_decode_step(p, q_idx, q_layers, out_layers, idx, count, workspace, workspace_bytes=None, stream=None) -> None:
     """q_layers / out_layers: sequences of L tensors (or addresses), one per cross-decoder layer."""
     L = p.num_layers
@@ -168,9 +195,9 @@ def clsa_decode_step(p, q_idx, q_layers, out_layers, idx, count, workspace, work
 
 
 def clsa_decode_step_static(p, q_idx, q_layers, out_layers, idx, count, dev_status=None, stream=None) -> None:
-    """clsa_decode_step for callers that cannot allocate: its scratch (status word and fp32 scores) is a fixed
-    8 MiB array inside the library, shared by every call on the GPU, so no workspace is passed. Shapes with more
-    than 2 Mi score slots raise ClsaError(CLSA_ERR_WORKSPACE). Calls must not overlap on the GPU; make the first
+    """clsa_decode_step for callers that cannot allocate: its scratch (a whole workspace) is a fixed 16 MiB array
+    inside the library, shared by every call on the GPU, so no workspace is passed. Shapes whose workspace would be
+    larger raise ClsaError(CLSA_ERR_WORKSPACE). Calls must not overlap on the GPU; make the first
     call on a device outside stream capture. `dev_status`: optional caller-owned uint32 device tensor."""
     L = p.num_layers
     if len(q_layers) != L or len(out_layers) != L:
@@ -192,13 +219,22 @@ def clsa_sparse_attn_layers(p, q_layers, idx, count, out_layers, workspace, work
                                         _nbytes(workspace, workspace_bytes), _stream(stream)), "clsa_sparse_attn_layers")
 
 
-def clsa_project_append(p, d_model, h, w_q_idx, w_k_idx, w_k, w_v, q_idx_out, workspace, workspace_bytes=None,
-                        stream=None) -> None:
+def clsa_project_append(p, d_model, h, w_q_idx, w_k_idx, w_k, w_v, q_idx_out, idx_k_cache_out, k_cache_out,
+                        v_cache_out, workspace, workspace_bytes=None, stream=None) -> None:
     """Eq. 2 for the T newest tokens of every sequence and the append of their K_idx (and, with w_k/w_v, K and V)
-    rows to the caches named by `p`, which this call WRITES. Weights are [n_out][d_model]."""
+    rows through the writable cache pointers `idx_k_cache_out`, `k_cache_out`, `v_cache_out` (the caches that `p`
+    describes). Weights are [n_out][d_model]."""
     _check(_lib.clsa_project_append(ctypes.byref(p), int(d_model), _ptr(h), _ptr(w_q_idx), _ptr(w_k_idx), _ptr(w_k),
-                                    _ptr(w_v), _ptr(q_idx_out), _ptr(workspace), _nbytes(workspace, workspace_bytes),
+                                    _ptr(w_v), _ptr(q_idx_out), _ptr(idx_k_cache_out), _ptr(k_cache_out),
+                                    _ptr(v_cache_out), _ptr(workspace), _nbytes(workspace, workspace_bytes),
                                     _stream(stream)), "clsa_project_append")
+
+
+def clsa_chain_plan(p, sm_count, clock_khz):
+    """(fine_layers, fine_rows): the tail of an L-layer chain that uses the finer launch shape. Host only."""
+    a, b = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(_lib.clsa_chain_plan(ctypes.byref(p), int(sm_count), int(clock_khz), ctypes.byref(a), ctypes.byref(b)), "clsa_chain_plan")
+    return int(a.value), int(b.value)
 
 
 def clsa_clear_status(workspace, workspace_bytes=None, stream=None) -> None:

@@ -19,7 +19,8 @@ bool device_info(DeviceInfo* out) {
     DeviceInfo d;
     if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&d.l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess) {
+        cudaDeviceGetAttribute(&d.l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.clock_khz, cudaDevAttrClockRate, dev) != cudaSuccess) {
       cudaGetLastError();
       return false;
     }
@@ -30,11 +31,20 @@ bool device_info(DeviceInfo* out) {
   return true;
 }
 
+// header | scratch of the decode attention launches | fp32 score matrix of clsa_decode_step
 WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& dev) {
-  (void)dev;
   WorkspaceLayout w;
   auto align = [](size_t x) { return (x + 255) / 256 * 256; };
-  w.scores_off = kStatusBytes;
+  w.attn_off = kStatusBytes;
+  w.attn_bytes = w.attn_counter_bytes = 0;
+  w.attn_part_off = w.attn_off;
+  if (p.q_per_seq == 1) {
+    const SkPlan alone = make_sk_plan(p, dev);
+    w.attn_counter_bytes = sk_counter_bytes(p, alone);
+    w.attn_part_off = w.attn_off + w.attn_counter_bytes;
+    w.attn_bytes = w.attn_counter_bytes + sk_partial_bytes(p, alone);
+  }
+  w.scores_off = w.attn_off + w.attn_bytes;
   w.score_stride = ((int64_t)p.max_seq_len + 63) / 64 * 64;
   w.scores_bytes = align((size_t)p.num_seqs * p.q_per_seq * w.score_stride * sizeof(float));
   w.total = w.scores_off + w.scores_bytes;
@@ -53,10 +63,11 @@ clsa_status check_shape(const clsa_params* p) {
     return CLSA_ERR_INVALID_ARG;
   if (p->num_q_heads % p->num_kv_heads != 0) return CLSA_ERR_INVALID_ARG;
   if (p->causal != 0 && p->causal != 1) return CLSA_ERR_INVALID_ARG;
-  if (p->sweep != 0 && p->sweep != 1) return CLSA_ERR_INVALID_ARG;
-  if (p->attn_plan < 0 || p->attn_plan > 2) return CLSA_ERR_INVALID_ARG;
   if (p->max_seq_len < p->q_per_seq) return CLSA_ERR_INVALID_ARG;
   if (!isfinite(p->sm_scale) || !(p->sm_scale > 0.f)) return CLSA_ERR_INVALID_ARG;  // the kernels take maxima before scaling
+  if (p->num_layers > 4096) return CLSA_ERR_INVALID_ARG;
+  // the decode attention kernel numbers its 16-token stages with 32 bits
+  if ((double)p->num_seqs * p->q_per_seq * p->num_kv_heads * ((p->top_k + 15) / 16) >= 2147483648.0) return CLSA_ERR_UNSUPPORTED;
   if ((int64_t)p->num_seqs * p->q_per_seq > (int64_t)1 << 30) return CLSA_ERR_INVALID_ARG;
   if (p->head_dim != 128) return CLSA_ERR_UNSUPPORTED;
   if (p->idx_dim != 64 && p->idx_dim != 128) return CLSA_ERR_UNSUPPORTED;
@@ -96,6 +107,12 @@ clsa_status check_workspace(const void* ws, size_t ws_bytes, size_t need) {
   return CLSA_OK;
 }
 
+// Below this occupancy of the whole-unit shape a launch with the GPU to itself takes the token-granular kernel
+// (measured on a B200, per layer at k = 2048, 32/8 heads: 1 sequence 10.9 against 12.5 us, 20 sequences 26.1 against
+// 30.4; where the whole-unit shape fills 65 % or more of its rounds it is as fast or faster, its merge staying inside
+// a block).
+constexpr double kTokenGranularBelow = 0.6;
+
 #define CLSA_TRY(expr)                     \
   do {                                     \
     const clsa_status st__ = (expr);       \
@@ -104,19 +121,50 @@ clsa_status check_workspace(const void* ws, size_t ws_bytes, size_t need) {
 
 clsa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? CLSA_OK : CLSA_ERR_CUDA; }
 
+clsa_status check_hints(const clsa_attn_hints* h) {
+  if (h == nullptr) return CLSA_OK;
+  for (int32_t v : {h->reverse, h->keep_rows, h->only_q_pending})
+    if (v != 0 && v != 1) return CLSA_ERR_INVALID_ARG;
+  if (h->shared_gpu < 0 || h->shared_gpu > 2) return CLSA_ERR_INVALID_ARG;
+  return CLSA_OK;
+}
+
+// One attention launch. A decode launch (one query per sequence) that has the GPU to itself goes to the
+// token-granular kernel and merges its split partials through the workspace; launches that share the GPU with their
+// neighbours (chained layers) and chunk launches (T > 1, far more query rows than SMs) go to the kernel that gives
+// whole (row, KV head) units to blocks.
+cudaError_t launch_attention(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
+                             float* lse, uint32_t* status, unsigned char* ws_base, const WorkspaceLayout& w,
+                             const clsa_attn_hints& h, int wait_prior, int fine_rows, const DeviceInfo& dev, cudaStream_t s) {
+  // With the GPU to itself, a decode launch whose (row, KV head) units would leave many SMs idle in the last round of
+  // whole-unit blocks (20 rows x 8 heads: 160 units on 148 SMs) cuts its work at token granularity instead.
+  if (p.q_per_seq == 1 && h.shared_gpu == 0 && attn_alone_occupancy(p, dev) < kTokenGranularBelow) {
+    const SkPlan plan = make_sk_plan(p, dev);
+    auto arrive = reinterpret_cast<uint32_t*>(ws_base + w.attn_off);
+    auto part = reinterpret_cast<float*>(ws_base + w.attn_part_off);
+    return launch_sparse_attn_sk(p, plan, q, idx, count, out, lse, status, arrive, part, h.reverse, wait_prior,
+                                 h.only_q_pending, h.keep_rows, s);
+  }
+  return launch_sparse_attn(p, q, idx, count, out, lse, status, h.reverse, wait_prior, h.only_q_pending, h.keep_rows,
+                            h.shared_gpu, fine_rows, dev, s);
+}
+
 // The L attention launches that share one index. Layer 0 follows whatever produced the index and must wait for it;
 // every later layer reads only what was complete before its predecessor started (the index, the caches, the caller's
 // queries), so it does not wait, and several layers are in flight at once. All of them walk the selected set in the
-// same direction (p.sweep): a layer then trails its predecessor by a few microseconds over the same rows and finds
-// them in L2 (measured at the headline: 286 us per step against 320 us with alternating directions).
+// same direction: a layer then trails its predecessor by a few microseconds over the same rows and finds them in L2.
+// The end of the chain uses smaller blocks so that it ends flush (chain_fine_tail).
 cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, void* const* out_layers, const int32_t* idx,
-                          const int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t s) {
-  const ChainTail tail = chain_fine_tail(p, dev);  // the end of the chain uses smaller blocks so that it ends flush
+                          const int32_t* count, uint32_t* status, unsigned char* ws_base, const DeviceInfo& dev,
+                          cudaStream_t s) {
+  const WorkspaceLayout w = make_workspace_layout(p, dev);
+  const ChainTail tail = chain_fine_tail(p, dev);
   for (int l = 0; l < p.num_layers; ++l) {
     const bool fine = l >= p.num_layers - tail.layers;
     const int fine_rows = l == p.num_layers - tail.layers - 1 ? tail.rows : 0;  // the layer where the finer shape begins
-    const cudaError_t err = launch_sparse_attn(p, q_layers[l], idx, count, out_layers[l], nullptr, status, p.sweep & 1,
-                                               l == 0 ? 1 : 0, l + 1 < p.num_layers ? 1 : 0, fine ? 2 : 1, fine_rows, dev, s);
+    const clsa_attn_hints h = {0, fine ? 2 : 1, l + 1 < p.num_layers ? 1 : 0, 0};
+    const cudaError_t err = launch_attention(p, q_layers[l], idx, count, out_layers[l], nullptr, status, ws_base, w, h,
+                                             l == 0 ? 1 : 0, fine_rows, dev, s);
     if (err != cudaSuccess) return err;
   }
   return cudaSuccess;
@@ -175,25 +223,57 @@ clsa_status clsa_topk(const clsa_params* p, const float* scores, int64_t score_s
                                static_cast<cudaStream_t>(stream)));
 }
 
-clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t* idx, const int32_t* count, void* out,
-                             float* lse, void* workspace, size_t workspace_bytes, clsa_stream stream) {
+clsa_status clsa_sparse_attn_hinted(const clsa_params* p, const void* q, const int32_t* idx, const int32_t* count,
+                                    void* out, float* lse, const clsa_attn_hints* hints, void* workspace,
+                                    size_t workspace_bytes, clsa_stream stream) {
   CLSA_TRY(check_shape(p));
   CLSA_TRY(check_seq(p));
   CLSA_TRY(check_kv_cache(p));
+  CLSA_TRY(check_hints(hints));
   if (q == nullptr || idx == nullptr || count == nullptr || out == nullptr) return CLSA_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(out, 16) || !aligned(idx, 4) || !aligned(count, 4) || !aligned(lse, 4))
     return CLSA_ERR_INVALID_ARG;
-  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
+  if (workspace == nullptr || !aligned(workspace, 256)) return CLSA_ERR_WORKSPACE;
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
-  return from_cuda(launch_sparse_attn(*p, q, idx, count, out, lse, static_cast<uint32_t*>(workspace), p->sweep & 1, 1, 0,
-                                      p->attn_plan, 0, dev,
-                                      static_cast<cudaStream_t>(stream)));
+  const WorkspaceLayout w = make_workspace_layout(*p, dev);
+  const clsa_attn_hints h = hints != nullptr ? *hints : clsa_attn_hints{0, 0, 0, 0};
+  // a decode launch with the GPU to itself merges its split partials through the scratch behind the header
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, p->q_per_seq == 1 && h.shared_gpu == 0 ? w.scores_off : kStatusBytes));
+  auto base = static_cast<unsigned char*>(workspace);
+  return from_cuda(launch_attention(*p, q, idx, count, out, lse, reinterpret_cast<uint32_t*>(base), base, w, h, 1, 0, dev,
+                                    static_cast<cudaStream_t>(stream)));
 }
 
-clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
-                             void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
-                             size_t workspace_bytes, clsa_stream stream) {
+clsa_status clsa_sparse_attn(const clsa_params* p, const void* q, const int32_t* idx, const int32_t* count, void* out,
+                             float* lse, void* workspace, size_t workspace_bytes, clsa_stream stream) {
+  return clsa_sparse_attn_hinted(p, q, idx, count, out, lse, nullptr, workspace, workspace_bytes, stream);
+}
+
+clsa_status clsa_gather_probe(const clsa_params* p, const int32_t* idx, const int32_t* count, const clsa_attn_hints* hints,
+                              void* workspace, size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  CLSA_TRY(check_kv_cache(p));
+  CLSA_TRY(check_hints(hints));
+  if (idx == nullptr || count == nullptr || !aligned(idx, 4) || !aligned(count, 4)) return CLSA_ERR_INVALID_ARG;
+  if (p->q_per_seq != 1) return CLSA_ERR_UNSUPPORTED;
+  if (workspace == nullptr || !aligned(workspace, 256)) return CLSA_ERR_WORKSPACE;
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  const WorkspaceLayout w = make_workspace_layout(*p, dev);
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, w.scores_off));
+  const clsa_attn_hints h = hints != nullptr ? *hints : clsa_attn_hints{0, 0, 0, 0};
+  auto base = static_cast<unsigned char*>(workspace);
+  const SkPlan plan = make_sk_plan(*p, dev);
+  return from_cuda(launch_gather_probe(*p, plan, idx, count, reinterpret_cast<uint32_t*>(base),
+                                       reinterpret_cast<float*>(base + w.attn_part_off), h.reverse, h.keep_rows,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+// Argument checks shared by the two whole-step entry points.
+static clsa_status check_step_args(const clsa_params* p, const void* q_idx, const void* const* q_layers,
+                                   void* const* out_layers, const int32_t* idx, const int32_t* count) {
   CLSA_TRY(check_shape(p));
   CLSA_TRY(check_seq(p));
   CLSA_TRY(check_idx_cache(p));
@@ -205,21 +285,33 @@ clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void
     if (q_layers[l] == nullptr || out_layers[l] == nullptr || !aligned(q_layers[l], 16) || !aligned(out_layers[l], 16))
       return CLSA_ERR_INVALID_ARG;
   if (p->q_per_seq != 1) return CLSA_ERR_UNSUPPORTED;
+  return CLSA_OK;
+}
+
+// index scores -> top-k -> L attention launches, all on `s`, scratch carved from `base` by `w`
+static clsa_status run_step(const clsa_params* p, const void* q_idx, const void* const* q_layers, void* const* out_layers,
+                            int32_t* idx, int32_t* count, unsigned char* base, uint32_t* status, const WorkspaceLayout& w,
+                            const DeviceInfo& dev, cudaStream_t s) {
+  auto scores = reinterpret_cast<float*>(base + w.scores_off);
+  auto sched = reinterpret_cast<uint32_t*>(base) + kSchedWord;
+  if (launch_index_scores_decode(*p, q_idx, scores, w.score_stride, status, sched, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
+  if (launch_topk(*p, scores, w.score_stride, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
+  if (launch_layers(*p, q_layers, out_layers, idx, count, status, base, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
+  return CLSA_OK;
+}
+
+clsa_status clsa_decode_step(const clsa_params* p, const void* q_idx, const void* const* q_layers,
+                             void* const* out_layers, int32_t* idx, int32_t* count, void* workspace,
+                             size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_step_args(p, q_idx, q_layers, out_layers, idx, count));
   if (workspace == nullptr || !aligned(workspace, 256)) return CLSA_ERR_WORKSPACE;
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
   const WorkspaceLayout w = make_workspace_layout(*p, dev);
   CLSA_TRY(check_workspace(workspace, workspace_bytes, w.total));
   auto base = static_cast<unsigned char*>(workspace);
-  auto status = reinterpret_cast<uint32_t*>(base);
-  auto scores = reinterpret_cast<float*>(base + w.scores_off);
-  auto s = static_cast<cudaStream_t>(stream);
-  cudaError_t err = launch_index_scores_decode(*p, q_idx, scores, w.score_stride, status, status + kSchedWord, dev, s);
-  if (err != cudaSuccess) return CLSA_ERR_CUDA;
-  err = launch_topk(*p, scores, w.score_stride, idx, count, status, dev, s);
-  if (err != cudaSuccess) return CLSA_ERR_CUDA;
-  if (launch_layers(*p, q_layers, out_layers, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
-  return CLSA_OK;
+  return run_step(p, q_idx, q_layers, out_layers, idx, count, base, reinterpret_cast<uint32_t*>(base), w, dev,
+                  static_cast<cudaStream_t>(stream));
 }
 
 clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* const* q_layers, const int32_t* idx,
@@ -233,40 +325,47 @@ clsa_status clsa_sparse_attn_layers(const clsa_params* p, const void* const* q_l
   for (int l = 0; l < p->num_layers; ++l)
     if (q_layers[l] == nullptr || out_layers[l] == nullptr || !aligned(q_layers[l], 16) || !aligned(out_layers[l], 16))
       return CLSA_ERR_INVALID_ARG;
-  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
+  if (workspace == nullptr || !aligned(workspace, 256)) return CLSA_ERR_WORKSPACE;
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
-  return from_cuda(launch_layers(*p, q_layers, out_layers, idx, count, static_cast<uint32_t*>(workspace), dev,
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
+  auto base = static_cast<unsigned char*>(workspace);
+  return from_cuda(launch_layers(*p, q_layers, out_layers, idx, count, reinterpret_cast<uint32_t*>(base), base, dev,
                                  static_cast<cudaStream_t>(stream)));
 }
 
 clsa_status clsa_project_append(const clsa_params* p, int32_t d_model, const void* h, const void* w_q_idx,
                                 const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,
-                                void* workspace, size_t workspace_bytes, clsa_stream stream) {
+                                void* idx_k_cache_out, void* k_cache_out, void* v_cache_out, void* workspace,
+                                size_t workspace_bytes, clsa_stream stream) {
   CLSA_TRY(check_shape(p));
   CLSA_TRY(check_seq(p));
-  CLSA_TRY(check_idx_cache(p));
-  if (h == nullptr || w_q_idx == nullptr || w_k_idx == nullptr || q_idx_out == nullptr) return CLSA_ERR_INVALID_ARG;
+  if (p->idx_token_stride < p->idx_dim || p->idx_token_stride % 8 != 0) return CLSA_ERR_INVALID_ARG;
+  if (h == nullptr || w_q_idx == nullptr || w_k_idx == nullptr || q_idx_out == nullptr || idx_k_cache_out == nullptr)
+    return CLSA_ERR_INVALID_ARG;
   if ((w_k == nullptr) != (w_v == nullptr)) return CLSA_ERR_INVALID_ARG;
+  if ((w_k != nullptr) != (k_cache_out != nullptr) || (w_v != nullptr) != (v_cache_out != nullptr)) return CLSA_ERR_INVALID_ARG;
   if (!aligned(h, 16) || !aligned(w_q_idx, 16) || !aligned(w_k_idx, 16) || !aligned(w_k, 16) || !aligned(w_v, 16) ||
-      !aligned(q_idx_out, 16))
+      !aligned(q_idx_out, 16) || !aligned(idx_k_cache_out, 16) || !aligned(k_cache_out, 16) || !aligned(v_cache_out, 16))
     return CLSA_ERR_INVALID_ARG;
   if (d_model < 32) return CLSA_ERR_INVALID_ARG;
   if (d_model % 32 != 0) return CLSA_ERR_UNSUPPORTED;
-  if (w_k != nullptr) CLSA_TRY(check_kv_cache(p));
+  if (w_k != nullptr) {
+    if (p->kv_head_stride < p->head_dim || p->kv_head_stride % 8 != 0) return CLSA_ERR_INVALID_ARG;
+    if (p->kv_token_stride < p->head_dim || p->kv_token_stride % 8 != 0) return CLSA_ERR_INVALID_ARG;
+  }
   CLSA_TRY(check_workspace(workspace, workspace_bytes, kStatusBytes));
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
-  return from_cuda(launch_project_append(*p, d_model, h, w_q_idx, w_k_idx, w_k, w_v, q_idx_out,
-                                         static_cast<uint32_t*>(workspace), dev, static_cast<cudaStream_t>(stream)));
+  return from_cuda(launch_project_append(*p, d_model, h, w_q_idx, w_k_idx, w_k, w_v, q_idx_out, idx_k_cache_out, k_cache_out,
+                                         v_cache_out, static_cast<uint32_t*>(workspace), dev, static_cast<cudaStream_t>(stream)));
 }
 
 // ---- entry point that allocates nothing -----------------------------------------------------------
-// Scratch of clsa_decode_step_static: the status word followed by the fp32 score matrix, in a
-// file-scope device array that every GPU loading this library keeps until the process exits.
+// Scratch of clsa_decode_step_static: a whole workspace (status header, attention merge scratch, fp32 score
+// matrix) in a file-scope device array that every GPU loading this library keeps until the process exits.
 namespace {
-constexpr size_t kStaticScoreSlots = (size_t)2 << 20;  // 2 Mi fp32 scores = 8 MiB
-constexpr size_t kStaticScratchBytes = kStatusBytes + kStaticScoreSlots * sizeof(float);
+constexpr size_t kStaticScratchBytes = kStatusBytes + ((size_t)16 << 20);
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 // In host code `g_static_scratch` is only a handle for the runtime, not a device address: the real
@@ -293,36 +392,32 @@ cudaError_t static_scratch_address(unsigned char** out) {
 clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, const void* const* q_layers,
                                     void* const* out_layers, int32_t* idx, int32_t* count, uint32_t* dev_status,
                                     clsa_stream stream) {
-  CLSA_TRY(check_shape(p));
-  CLSA_TRY(check_seq(p));
-  CLSA_TRY(check_idx_cache(p));
-  CLSA_TRY(check_kv_cache(p));
-  if (q_idx == nullptr || q_layers == nullptr || out_layers == nullptr || idx == nullptr || count == nullptr)
-    return CLSA_ERR_INVALID_ARG;
-  if (!aligned(q_idx, 16) || !aligned(idx, 4) || !aligned(count, 4) || !aligned(dev_status, 4)) return CLSA_ERR_INVALID_ARG;
-  for (int l = 0; l < p->num_layers; ++l)
-    if (q_layers[l] == nullptr || out_layers[l] == nullptr || !aligned(q_layers[l], 16) || !aligned(out_layers[l], 16))
-      return CLSA_ERR_INVALID_ARG;
-  if (p->q_per_seq != 1) return CLSA_ERR_UNSUPPORTED;
-  const int64_t stride = ((int64_t)p->max_seq_len + 63) / 64 * 64;
-  if ((uint64_t)p->num_seqs * (uint64_t)stride > kStaticScoreSlots) return CLSA_ERR_WORKSPACE;  // beyond the fixed scratch
+  CLSA_TRY(check_step_args(p, q_idx, q_layers, out_layers, idx, count));
+  if (!aligned(dev_status, 4)) return CLSA_ERR_INVALID_ARG;
   DeviceInfo dev;
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  const WorkspaceLayout w = make_workspace_layout(*p, dev);
+  if (w.total > kStaticScratchBytes) return CLSA_ERR_WORKSPACE;  // beyond the fixed scratch
   unsigned char* base = nullptr;
   if (static_scratch_address(&base) != cudaSuccess) return CLSA_ERR_CUDA;
   auto s = static_cast<cudaStream_t>(stream);
-  // The array keeps whatever the previous call left: the status word must start at zero. The score
-  // matrix needs no clearing (every entry that is read is written first).
+  // The array keeps whatever the previous call left. What must start at zero is cleared on every call, whoever owns
+  // the status word: the header (status word, the score kernel's ticket counters) -- a call that was cut short, or
+  // two calls that raced, cannot poison later ones. The scores need no clearing (every entry that is read is written
+  // first).
+  if (cudaMemsetAsync(base, 0, kStatusBytes, s) != cudaSuccess) return CLSA_ERR_CUDA;
   uint32_t* status = dev_status != nullptr ? dev_status : reinterpret_cast<uint32_t*>(base);
-  if (dev_status == nullptr && cudaMemsetAsync(base, 0, kStatusBytes, s) != cudaSuccess) return CLSA_ERR_CUDA;
-  auto scores = reinterpret_cast<float*>(base + kStatusBytes);
-  // the score kernel's scheduling counters always live in the scratch array's header (zero when the library is
-  // loaded, and left at zero by every launch), also when the status word is the caller's
-  if (launch_index_scores_decode(*p, q_idx, scores, stride, status, reinterpret_cast<uint32_t*>(base) + kSchedWord, dev, s) !=
-      cudaSuccess)
-    return CLSA_ERR_CUDA;
-  if (launch_topk(*p, scores, stride, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
-  if (launch_layers(*p, q_layers, out_layers, idx, count, status, dev, s) != cudaSuccess) return CLSA_ERR_CUDA;
+  return run_step(p, q_idx, q_layers, out_layers, idx, count, base, status, w, dev, s);
+}
+
+clsa_status clsa_chain_plan(const clsa_params* p, int32_t sm_count, int32_t clock_khz, int32_t* fine_layers,
+                            int32_t* fine_rows) {
+  if (fine_layers == nullptr || fine_rows == nullptr || sm_count < 1 || clock_khz < 1) return CLSA_ERR_INVALID_ARG;
+  CLSA_TRY(check_shape(p));
+  DeviceInfo dev = {sm_count, 227 * 1024, 0, clock_khz};
+  const ChainTail t = p->q_per_seq == 1 ? chain_fine_tail(*p, dev) : ChainTail{0, 0};
+  *fine_layers = t.layers;
+  *fine_rows = t.rows;
   return CLSA_OK;
 }
 
@@ -350,6 +445,6 @@ const char* clsa_status_string(clsa_status s) {
   return "unknown status";
 }
 
-int clsa_version(void) { return 100; }
+int clsa_version(void) { return 200; }
 
 }  // extern "C"

@@ -14,6 +14,7 @@ struct DeviceInfo {
   int sm_count;
   int max_smem_optin;  // bytes of dynamic shared memory a block may opt in to
   int l2_bytes;
+  int clock_khz;       // peak SM clock
 };
 // Cached per device (queried once). Returns false if the CUDA runtime reports an error.
 bool device_info(DeviceInfo* out);
@@ -47,6 +48,22 @@ struct ChainTail {
 };
 ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev);
 
+// Launch shape of the token-granular decode attention kernel (sparse_attn_sk.cu).
+struct SkPlan {
+  int warps;             // warps per block, each an autonomous worker
+  int blocks;            // grid size: one block per SM (fewer for small launches)
+  int workers;           // W: warps that get a span of the stage list (<= blocks * wpb, <= total_stages)
+  int wpb;               // workers per block (<= warps)
+  int aligned;           // 1: every unit has workers of its own (no span crosses a unit boundary); 0: flat split
+  int unit_stages;       // NS = ceil(k / 16): 16-token stages per (query row, KV head) unit
+  int64_t units;         // rows * Hkv
+  int64_t total_stages;  // units * NS
+  size_t smem_bytes;
+};
+SkPlan make_sk_plan(const clsa_params& p, const DeviceInfo& dev);
+size_t sk_counter_bytes(const clsa_params& p, const SkPlan& plan);  // arrival counters of one launch
+size_t sk_partial_bytes(const clsa_params& p, const SkPlan& plan);  // partial slots of one launch
+
 struct TopkPlan {
   int cluster;      // blocks per (sequence, query) row, a thread-block cluster
   int slice_cap;    // score slots each block keeps in shared memory (0 = re-read global memory each pass)
@@ -57,6 +74,11 @@ struct TopkPlan {
 TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev, bool one_sweep_fits);
 
 struct WorkspaceLayout {
+  // Scratch of a decode attention launch that has the GPU to itself (q_per_seq == 1; empty otherwise): arrival
+  // counters, then partial slots.
+  size_t attn_off, attn_bytes;
+  size_t attn_counter_bytes;
+  size_t attn_part_off;             // start of the partial slots
   size_t scores_off, scores_bytes;  // fp32 score matrix of clsa_decode_step
   int64_t score_stride;
   size_t total;
@@ -78,11 +100,27 @@ bool topk_prefilter_fits(const clsa_params& p, const float* scores, int64_t scor
 cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx,
                                   int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
-                               float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
-                               int throughput_plan, int fine_rows, const DeviceInfo& dev, cudaStream_t stream);
+                               float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
+                               int keep_for_next, int throughput_plan, int fine_rows, const DeviceInfo& dev,
+                               cudaStream_t stream);
+// Share of its rounds of one-block-per-SM that the whole-unit kernel's launch-on-its-own shape fills (0..1).
+double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev);
 
+// Decode attention with token-granular work items (q_per_seq == 1). arrive: sk_counter_bytes(plan) of counters that
+// are zero (every launch leaves them so); part: sk_partial_bytes(p, plan) of partial slots. Launches in flight
+// together need counters and slots of their own.
+cudaError_t launch_sparse_attn_sk(const clsa_params& p, const SkPlan& plan, const void* q, const int32_t* idx,
+                                  const int32_t* count, void* out, float* lse, uint32_t* status, uint32_t* arrive,
+                                  float* part, int reverse, int wait_prior, int only_q_pending, int keep_rows,
+                                  cudaStream_t stream);
+// The same gather without the arithmetic (measurement aid); part as above (used as a sink).
+cudaError_t launch_gather_probe(const clsa_params& p, const SkPlan& plan, const int32_t* idx, const int32_t* count,
+                                uint32_t* status, float* part, int reverse, int keep_rows, cudaStream_t stream);
+
+// idx_k_out / k_out / v_out: the caches of p, writable (k_out and v_out may be null together with w_k and w_v)
 cudaError_t launch_project_append(const clsa_params& p, int d_model, const void* h, const void* w_q_idx,
                                   const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,
+                                  void* idx_k_out, void* k_out, void* v_out,
                                   uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------

@@ -176,6 +176,7 @@ __global__ void __launch_bounds__(kWarps * 32) project_append_kernel(const ProjA
 
 cudaError_t launch_project_append(const clsa_params& p, int d_model, const void* h, const void* w_q_idx,
                                   const void* w_k_idx, const void* w_k, const void* w_v, void* q_idx_out,
+                                  void* idx_k_out, void* k_out, void* v_out,
                                   uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
   (void)dev;
   ProjArgs a;
@@ -190,9 +191,9 @@ cudaError_t launch_project_append(const clsa_params& p, int d_model, const void*
   a.seg_end[2] = 2 * p.idx_dim + kv;
   a.seg_end[3] = 2 * p.idx_dim + 2 * kv;
   a.q_idx_out = static_cast<uint16_t*>(q_idx_out);
-  a.idx_k_cache = static_cast<uint16_t*>(const_cast<void*>(p.idx_k_cache));
-  a.k_cache = static_cast<uint16_t*>(const_cast<void*>(p.k_cache));
-  a.v_cache = static_cast<uint16_t*>(const_cast<void*>(p.v_cache));
+  a.idx_k_cache = static_cast<uint16_t*>(idx_k_out);
+  a.k_cache = static_cast<uint16_t*>(k_out);
+  a.v_cache = static_cast<uint16_t*>(v_out);
   a.idx_token_stride = p.idx_token_stride;
   a.kv_token_stride = p.kv_token_stride;
   a.kv_head_stride = p.kv_head_stride;

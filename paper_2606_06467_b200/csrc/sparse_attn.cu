@@ -1,4 +1,7 @@
-// GQA sparse attention over the selected rows only (Eq. 4), one launch per cross-decoder layer.
+// GQA sparse attention over the selected rows only (Eq. 4), one launch per cross-decoder layer: the kernel for
+// launches that share the GPU with their neighbours on the stream (the chained layers of a decode step) and for
+// launches with many query rows (prefill chunks). A decode launch that has the GPU to itself uses the token-granular
+// kernel in sparse_attn_sk.cu, which shares this file's staging ring and arithmetic.
 //
 // The kernel is bound by the gather of K/V rows from HBM (4 flops per byte per KV head), so its
 // shape is chosen for memory behaviour; the small matrix products ride on warp-level bf16 MMAs
@@ -27,26 +30,16 @@
 // `reverse` flips the order in which a warp walks its range (a locality hint for callers that issue
 // dependent layers one by one; the chained layers of a step all walk the same way).
 #include <cooperative_groups.h>
-#include <vector>
-#include <functional>
-#include <algorithm>
-
 #include <mutex>
 
-#include "common.cuh"
+#include "attn_common.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace clsa {
 namespace {
 
-static_assert(kAttnStages == 2, "the position pipeline in the kernel is written for a 2-deep ring");
-constexpr int kStageBytes = kAttnStageTokens * 256 * 2;  // 16 K rows + 16 V rows of 256 bytes
-constexpr int kWarpRingBytes = kAttnStages * kStageBytes;
-constexpr int kPartialStride = 132;                      // floats per head of a partial: 128 outputs, max, sum, pad
 constexpr int kMergeBatch = 8;
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 
 struct AttnArgs {
   const uint16_t* q;
@@ -66,70 +59,16 @@ struct AttnArgs {
   int heads_per_block, subs, rows_per_block, reverse;
   int64_t num_rows;
   int wait_prior;  // 1: inputs may come from the kernel launched just before this one (wait for it first)
+  int early;       // 1 (with wait_prior): only q is pending; index, counts and caches may be read before the wait
   int off32;          // every row offset of the caches fits 32 bits when counted in 16-byte units
   int64_t rows_max;   // extent of the cache row space (off32 only): rows at or beyond it are refused like bad indices
   int keep;           // 1: the rows are fetched with the L2 evict_last priority (launches behind this one read them again)
   int coarse_blocks;  // -1: one block size, 2-D grid. >= 0: a 1-D grid of two block sizes (no cluster, one row per block):
                       // the first coarse_blocks blocks take heads_per_block KV heads each, row by row; the blocks behind
                       // them take half as many (twice the token ranges) and cover the remaining rows
+  int max_seq_len;    // sequences longer than this (or shorter than q_per_seq) are skipped and flagged
   float scale_log2;
 };
-
-// 16-byte asynchronous copy global -> shared with an L2 eviction-priority hint.
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid, uint64_t policy) {
-  const int bytes = valid ? 16 : 0;  // 0 source bytes: the 16 destination bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;\n"
-               ::"r"(dst), "l"(src), "r"(bytes), "l"(policy) : "memory");
-}
-// The same without the source-size operand (the whole 16 bytes are copied).
-__device__ __forceinline__ void cp_async16_full(uint32_t dst, const void* src, uint64_t policy) {
-  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "l"(policy) : "memory");
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_last() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// 2^x by the hardware approximation (2 ulp; -inf gives +0).
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
-  uint32_t y;
-  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
-  return y;
-}
 
 // NT = number of 8-head tiles that hold the query heads of one KV head (1 for groups up to 8, 2 up to 16).
 // WARPS = warps per block: 12 for NT = 1 (about 165 registers per thread), 8 for NT = 2.
@@ -188,8 +127,18 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
   // kernel of the stream be scheduled (as SMs free up). The order matters: a kernel launched behind
   // this one may skip its own wait on the grounds that everything it reads was complete before this
   // grid started reading -- which holds only if this grid has waited before it releases anybody.
-  if (a.wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // A launch whose only pending input is q (a.early) waits later: behind the first stage of row copies, in front of
+  // the first read of q and of every global write.
+  bool waited = !(a.wait_prior && a.early);
+  if (a.wait_prior && !a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (waited) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  auto wait_now = [&]() {
+    if (!waited) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+      waited = true;
+    }
+  };
 
   // The row's k slots are cut into nsplit ranges of `per` slots (a multiple of the stage size); the
   // split does not depend on the row's count, so the first positions can be fetched together with it.
@@ -202,7 +151,12 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
   constexpr bool paged = PAGED;
   const int64_t s0 = paged ? 0 : a.seq_start[b];  // paged: positions are translated to cache rows when they are fetched
   const int32_t* table = paged ? a.block_table + (int64_t)b * a.max_blocks : nullptr;
-  const int n = a.seq_len[b];
+  // A sequence whose length lies outside its declared bounds is never read: with n = 0 no position passes the range
+  // check, every stage is masked, and the row comes out as zeros with lse = -inf. (A select, not a branch: the length
+  // is first needed when the first copies are issued, and the flag is raised behind the main loop.)
+  const int n_raw = a.seq_len[b];
+  const bool n_ok = n_raw >= a.q_per_seq && n_raw <= a.max_seq_len;
+  const int n = n_ok ? n_raw : 0;
   // Positions are fetched two pipeline steps before they are used and (paged caches) their block numbers one
   // step before, so that no load is consumed in the step that issued it. The first three steps' positions are
   // fetched here, speculatively for a range that lies entirely below the row's count (entries past the count
@@ -237,7 +191,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
   if (t_lo < t_hi) {
     // Q^T fragments (B operand, 128 x 8 per head tile): head = rowq, two consecutive d per register.
     uint32_t qb[NT][8][2];
-    {
+    auto load_q = [&]() {
       const uint16_t* qbase = a.q + (r * a.num_q_heads + h0) * 128;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
@@ -250,7 +204,8 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
           qb[nt][ks][1] = hv ? *reinterpret_cast<const uint32_t*>(qbase + head * 128 + d + 8) : 0u;
         }
       }
-    }
+    };
+    if (waited) load_q();
 
     const int nstages = (t_hi - t_lo + kAttnStageTokens - 1) / kAttnStageTokens;
     const uint16_t* kbase = a.kc + g * a.head_stride + (lane & 15) * 8;
@@ -293,7 +248,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
         const int my_idx = paged ? (blk << a.block_shift) + (raw & ((1 << a.block_shift) - 1)) : raw;
         const bool in_range = raw >= 0 && raw < n && (!a.off32 || (uint64_t)(s0 + my_idx) < (uint64_t)a.rows_max);
         const uint32_t okmask = __ballot_sync(0xffffffffu, in_range) & 0xffffu;
-        const bool bad = lane < kAttnStageTokens && !in_range && (stage_t0(i) + lane) < t_hi;
+        const bool bad = lane < kAttnStageTokens && !in_range && n_ok && (stage_t0(i) + lane) < t_hi;
         if (bad) flag_status(a.status, CLSA_DEV_BAD_INDEX);
         if (lane == 0) stage_mask[buf] = okmask;
         if (a.off32) {
@@ -342,6 +297,10 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
       const int b0 = load_blk(r0);
       blkA = load_blk(rawA);
       issue(0, r0, b0);
+    }
+    if (!waited) {  // only q was pending: the first stage of copies is in flight, now wait for q's producer
+      wait_now();
+      load_q();
     }
 #pragma unroll 1
     for (int i = 0; i < nstages; ++i) {
@@ -444,6 +403,9 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { lA[nt] = lacc[nt][0]; lB[nt] = lacc[nt][1]; }
   }
+
+  wait_now();  // a warp without tokens has not waited yet; what follows writes global memory
+  if (!n_ok && lane == 0 && sub == 0 && g_local == 0 && crank == 0 && by == 0 && active) flag_status(a.status, CLSA_DEV_BAD_SEQLEN);
 
   // ---- split-K merge through (distributed) shared memory --------------------------------------------
   // Each warp parks its partial in its own (now idle) staging ring: [G][kPartialStride] floats, row = head.
@@ -647,14 +609,121 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
 // before it has started all of its own. With equal blocks the last round is usually part empty (16 layers of 32
 // blocks on 148 SMs: 3.46 rounds, the fourth with 68 blocks). Blocks of half the size at the end of the chain --
 // the last query rows of one layer and every layer behind it -- fill that round at a finer grain. Where the finer
-// shape begins: the schedule is simulated for every choice (whole layers, and eighths of the rows of the layer before
-// them) with a block's duration modelled as a fixed part (launch gap, ramp, merge: 9.5 us measured) plus its bytes at
-// the per-SM gather rate (118 GB/s measured), and the best choice is taken if it gains at least 2 %. Cached per shape.
+// shape begins: the schedule is simulated for a short list of choices (up to kTailMaxLayers whole layers, and eighths
+// of the rows of the layer before them) with a block's duration modelled as a fixed part (launch gap, ramp, merge)
+// plus its bytes at the per-SM gather rate, and the best choice is taken if it gains at least 2 %.
+//
+// Host cost. Blocks of one launch are equal, so the SMs' free times take few distinct values: the schedule is kept
+// as a short sorted list of (time, number of SMs) groups and a launch of nb blocks is placed group by group, not
+// block by block; the coarse layers that every candidate shares are placed once. A shape that has not been seen
+// costs a few microseconds; results are memoised (LRU, keyed on every input of the model), and the lock guards only
+// the memo, not the simulation.
+namespace {
+
+constexpr int kTailMaxLayers = 3;       // whole layers the finer shape may take (the last round is at most that deep)
+constexpr double kBlockFixedUs = 9.5;   // launch gap + pipeline ramp + merge of one block, measured on a B200
+constexpr double kPortBytesPerClock = 64.0 * 0.94;  // L2 -> SM port, and the share of it the gather reaches
+
+// SM free times as sorted groups (ascending time).
+struct SmGroups {
+  static constexpr int kMax = 24;
+  double t[kMax];
+  int c[kMax];
+  int n;
+  void init(int sms) { n = 1; t[0] = 0.0; c[0] = sms; }
+  // Places nb blocks of duration d, none before `gate`; returns the start time of the last one placed.
+  double place(int64_t nb, double d, double gate, double& end) {
+    double last_start = gate;
+    while (nb > 0) {
+      const double start = t[0] > gate ? t[0] : gate;
+      const int take = (int64_t)c[0] <= nb ? c[0] : (int)nb;
+      nb -= take;
+      last_start = start;
+      const double fin = start + d;
+      if (fin > end) end = fin;
+      // remove `take` SMs from the first group, add them at time fin
+      if (take == c[0]) { for (int i = 1; i < n; ++i) { t[i - 1] = t[i]; c[i - 1] = c[i]; } --n; }
+      else c[0] -= take;
+      int pos = n;
+      while (pos > 0 && t[pos - 1] > fin) --pos;
+      if (pos > 0 && t[pos - 1] == fin) { c[pos - 1] += take; continue; }
+      if (n == kMax) {  // cannot happen with two block sizes; merge into the last group rather than overflow
+        c[n - 1] += take;
+        if (fin > t[n - 1]) t[n - 1] = fin;
+        continue;
+      }
+      for (int i = n; i > pos; --i) { t[i] = t[i - 1]; c[i] = c[i - 1]; }
+      t[pos] = fin; c[pos] = take; ++n;
+    }
+    return last_start;
+  }
+};
+
+struct TailKey {
+  int L, sms, clock_khz, k_eff, hb, hf, hkv;
+  int64_t rows;
+  bool operator==(const TailKey& o) const {
+    return L == o.L && sms == o.sms && clock_khz == o.clock_khz && k_eff == o.k_eff && hb == o.hb && hf == o.hf &&
+           hkv == o.hkv && rows == o.rows;
+  }
+};
+
+ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fine, int hg_base, int hg_fine) {
+  const ChainTail none = {0, 0};
+  const double rate = kPortBytesPerClock * (double)key.clock_khz * 1e3 / 1e6;  // bytes per microsecond per SM
+  auto duration = [&](int heads_per_block) { return kBlockFixedUs + (double)heads_per_block * key.k_eff * 512.0 / rate; };
+  const double d_base = duration(key.hb), d_fine = duration(key.hf);
+  const int L = key.L;
+  const int max_tail = L - 1 < kTailMaxLayers ? L - 1 : kTailMaxLayers;
+  // state after the coarse layers that every candidate shares: layers [0, L - max_tail - 1)
+  SmGroups g;
+  g.init(key.sms);
+  double end = 0.0, gate = 0.0;
+  const int shared = L - max_tail - 1;
+  // snapshots[i]: state after `shared + i` coarse layers
+  SmGroups snap[kTailMaxLayers + 2];
+  double snap_gate[kTailMaxLayers + 2], snap_end[kTailMaxLayers + 2];
+  for (int l = 0; l < shared; ++l) gate = g.place(nb_base, d_base, gate, end);
+  for (int i = 0; i <= max_tail + 1; ++i) {
+    snap[i] = g; snap_gate[i] = gate; snap_end[i] = end;
+    if (i <= max_tail) gate = g.place(nb_base, d_base, gate, end);
+  }
+  const double plain = snap_end[max_tail + 1];  // all L layers coarse
+  double best = plain;
+  ChainTail best_tail = none;
+  const int64_t rows = key.rows;
+  const int64_t step = rows >= 8 ? rows / 8 : 1;  // partial layers in eighths of the rows
+  for (int tail = 0; tail <= max_tail; ++tail)
+    for (int64_t part = 0; part < rows; part += step) {
+      if (tail == 0 && part == 0) continue;
+      // layers [0, L - tail - 1) coarse; layer L - tail - 1 coarse except its last `part` rows; the last `tail` fine
+      const int coarse_layers = L - tail - 1;
+      SmGroups h = snap[coarse_layers - shared];
+      double gt = snap_gate[coarse_layers - shared], en = snap_end[coarse_layers - shared];
+      if (part > 0) {
+        const double g0 = gt;
+        const double s1 = h.place((rows - part) * hg_base, d_base, g0, en);
+        const double s2 = h.place(part * hg_fine, d_fine, g0, en);
+        gt = s1 > s2 ? s1 : s2;
+      } else {
+        gt = h.place(nb_base, d_base, gt, en);
+      }
+      for (int l = 0; l < tail; ++l) gt = h.place(nb_fine, d_fine, gt, en);
+      if (en < best - 1e-9) { best = en; best_tail = ChainTail{tail, (int)part}; }
+    }
+  if (best > 0.98 * plain) best_tail = none;
+  return best_tail;
+}
+
+}  // namespace
+
 ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
-  ChainTail none = {0, 0};
+  const ChainTail none = {0, 0};
   const int L = p.num_layers;
-  if (L < 2 || L > 256) return none;
-  if (p.block_table != nullptr) return none;  // paged caches: measured, the finer blocks cost more than the fuller last round returns
+  if (L < 2) return none;
+  if (p.block_table != nullptr) return none;  // paged caches: the finer blocks cost more than the fuller last round returns
+  // The block model above was measured on a B200 (148 SMs); on anything else the chain keeps one block size.
+  if (dev.sm_count != 148 || dev.clock_khz <= 0) return none;
   const AttnPlan base = make_attn_plan(p, dev, 1), fine = make_attn_plan(p, dev, 2);
   if (base.cluster != 1 || fine.cluster != 1 || fine.heads_per_block == base.heads_per_block ||
       base.rows_per_block != 1 || fine.rows_per_block != 1)
@@ -662,65 +731,42 @@ ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   const int64_t nb_base = rows * base.head_groups, nb_fine = rows * fine.head_groups;
   if (nb_base > 4096 || nb_fine > 8192) return none;  // far more blocks than SMs: the last round is a small part of the whole
-  struct Key { int L, sms, k, hb, hf; int64_t rows; ChainTail tail; };
+  const TailKey key = {L, dev.sm_count, dev.clock_khz, p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len,
+                       base.heads_per_block, fine.heads_per_block, p.num_kv_heads, rows};
+  struct Entry { TailKey key; ChainTail tail; uint64_t used; };
+  constexpr int kMemo = 64;
   static std::mutex mu;
-  static Key seen[16];
-  static int used = 0;
-  std::lock_guard<std::mutex> lock(mu);
-  for (int i = 0; i < used; ++i)
-    if (seen[i].L == L && seen[i].sms == dev.sm_count && seen[i].k == p.top_k && seen[i].hb == base.heads_per_block &&
-        seen[i].hf == fine.heads_per_block && seen[i].rows == rows)
-      return seen[i].tail;
-  const double k_eff = (double)(p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len);
-  auto duration = [&](const AttnPlan& pl) {  // microseconds
-    const double bytes = (double)pl.heads_per_block * k_eff * 512.0;
-    return 9.5 + bytes / 118e3;
-  };
-  const double d_base = duration(base), d_fine = duration(fine);
-  std::vector<double> heap((size_t)dev.sm_count);
-  // layers [0, L - tail - 1) coarse; layer L - tail - 1 coarse except its last `part` rows; the last `tail` layers fine
-  auto makespan = [&](int tail, int64_t part) {
-    std::fill(heap.begin(), heap.end(), 0.0);  // all equal: a valid min-heap (std::greater)
-    double end = 0.0, gate = 0.0;
-    auto place = [&](int64_t nb, double d, double& last_start) {
-      for (int64_t j = 0; j < nb; ++j) {
-        std::pop_heap(heap.begin(), heap.end(), std::greater<double>());
-        const double t = std::max(heap.back(), gate);
-        heap.back() = t + d;
-        std::push_heap(heap.begin(), heap.end(), std::greater<double>());
-        end = std::max(end, t + d);
-        last_start = std::max(last_start, t);
-      }
-    };
-    for (int l = 0; l < L; ++l) {
-      double last_start = gate;
-      if (l >= L - tail) place(nb_fine, d_fine, last_start);
-      else if (l == L - tail - 1 && part > 0) {
-        place((rows - part) * base.head_groups, d_base, last_start);
-        place(part * fine.head_groups, d_fine, last_start);
-      } else place(nb_base, d_base, last_start);
-      gate = last_start;
-    }
-    return end;
-  };
-  const double plain = makespan(0, 0);
-  double best = plain;
-  ChainTail best_tail = none;
-  const int64_t step = rows >= 8 ? rows / 8 : 1;  // partial layers in eighths of the rows
-  for (int tail = 0; tail < L; ++tail)
-    for (int64_t part = 0; part < rows; part += step) {
-      if (tail == 0 && part == 0) continue;
-      const double m = makespan(tail, part);
-      if (m < best - 1e-9) { best = m; best_tail = ChainTail{tail, (int)part}; }
-    }
-  if (best > 0.98 * plain) best_tail = none;
-  if (used < 16) seen[used++] = Key{L, dev.sm_count, p.top_k, base.heads_per_block, fine.heads_per_block, rows, best_tail};
-  return best_tail;
+  static Entry memo[kMemo];
+  static int filled = 0;
+  static uint64_t tick = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < filled; ++i)
+      if (memo[i].key == key) { memo[i].used = ++tick; return memo[i].tail; }
+  }
+  const ChainTail tail = simulate_fine_tail(key, nb_base, nb_fine, base.head_groups, fine.head_groups);  // outside the lock
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    int slot = 0;
+    if (filled < kMemo) slot = filled++;
+    else for (int i = 1; i < kMemo; ++i) if (memo[i].used < memo[slot].used) slot = i;  // least recently used
+    memo[slot] = Entry{key, tail, ++tick};
+  }
+  return tail;
+}
+
+double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev) {
+  const AttnPlan plan = make_attn_plan(p, dev, 0);
+  const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
+  const int64_t blocks = (rows + plan.rows_per_block - 1) / plan.rows_per_block * plan.cluster * plan.head_groups;
+  const int64_t rounds = (blocks + dev.sm_count - 1) / dev.sm_count;
+  return (double)blocks / (double)(rounds * dev.sm_count);
 }
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
-                               float* lse, uint32_t* status, int reverse, int wait_prior, int keep_for_next,
-                               int throughput_plan, int fine_rows, const DeviceInfo& dev, cudaStream_t stream) {
+                               float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
+                               int keep_for_next, int throughput_plan, int fine_rows, const DeviceInfo& dev,
+                               cudaStream_t stream) {
   const AttnPlan plan = make_attn_plan(p, dev, throughput_plan);
   AttnArgs a;
   a.q = static_cast<const uint16_t*>(q);
@@ -750,11 +796,13 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.num_rows = (int64_t)p.num_seqs * p.q_per_seq;
   a.reverse = reverse;
   a.wait_prior = wait_prior;
+  a.early = (wait_prior && only_q_pending) ? 1 : 0;
   // L2 priority of the gathered rows. A launch with a successor that will read the same rows (the chained layers)
   // fetches all of them with evict_last, so that scores, indices and outputs passing through L2 do not push them
   // out before the layers behind it arrive; a launch on its own leaves the replacement policy alone.
   a.keep = keep_for_next ? 1 : 0;
   a.coarse_blocks = -1;
+  a.max_seq_len = p.max_seq_len;
   a.scale_log2 = p.sm_scale * kLog2e;
   // With the extent of the row space known (num_cache_rows) and below 2^32 16-byte units, row offsets are 32-bit.
   a.rows_max = p.num_cache_rows;

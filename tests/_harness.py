@@ -69,14 +69,17 @@ class GpuProblem:
         clsa.clsa_topk(self.params, scores, scores.shape[-1], self.idx, self.count, self.ws)
         return self.idx, self.count
 
-    def sparse_attn(self, layer, idx=None, count=None, lse=True, sweep=0, plan=0):
+    def sparse_attn(self, layer, idx=None, count=None, lse=True, reverse=0, shared_gpu=0, keep_rows=0, only_q_pending=0):
+        """One layer through clsa_sparse_attn (all hints zero) or clsa_sparse_attn_hinted."""
         c = self.cfg
         out = self.new_out()
         l = torch.full((c.num_seqs, c.q_per_seq, c.num_q_heads), float("nan"), dtype=torch.float32, device=self.dev) if lse else None
-        self.params.sweep, self.params.attn_plan = sweep, plan
-        clsa.clsa_sparse_attn(self.params, self.t["q_layers"][layer], self.idx if idx is None else idx,
-                              self.count if count is None else count, out, l, self.ws)
-        self.params.sweep, self.params.attn_plan = 0, 0
+        args = (self.params, self.t["q_layers"][layer], self.idx if idx is None else idx,
+                self.count if count is None else count, out, l)
+        if reverse or shared_gpu or keep_rows or only_q_pending:
+            clsa.clsa_sparse_attn_hinted(*args, clsa.make_hints(reverse, shared_gpu, keep_rows, only_q_pending), self.ws)
+        else:
+            clsa.clsa_sparse_attn(*args, self.ws)
         return out, l
 
     def decode_step(self):

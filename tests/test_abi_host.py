@@ -30,11 +30,11 @@ def _declared_functions():
 
 def test_every_declared_symbol_is_exported(clsa):
     names = _declared_functions()
-    assert len(names) == 12 and set(names) == set(clsa.EXPORTS)
+    assert len(names) == 15 and set(names) == set(clsa.EXPORTS)
     lib = ctypes.CDLL(clsa.LIB_PATH)
     for n in names:
         assert hasattr(lib, n), n
-    assert clsa.clsa_version() == 100
+    assert clsa.clsa_version() == 200
     assert clsa.clsa_status_string(0) == "ok" and "unsupported" in clsa.clsa_status_string(2)
 
 
@@ -67,7 +67,7 @@ def test_bad_arguments_are_refused_on_the_host(clsa):
     for kw, want in (
         (dict(num_seqs=0), clsa.CLSA_ERR_INVALID_ARG), (dict(top_k=0), clsa.CLSA_ERR_INVALID_ARG),
         (dict(num_q_heads=30), clsa.CLSA_ERR_INVALID_ARG), (dict(causal=2), clsa.CLSA_ERR_INVALID_ARG),
-        (dict(sweep=3), clsa.CLSA_ERR_INVALID_ARG), (dict(attn_plan=3), clsa.CLSA_ERR_INVALID_ARG), (dict(max_seq_len=0), clsa.CLSA_ERR_INVALID_ARG),
+        (dict(max_seq_len=0), clsa.CLSA_ERR_INVALID_ARG), (dict(sm_scale=-1.0), clsa.CLSA_ERR_INVALID_ARG),
         (dict(sm_scale=float("nan")), clsa.CLSA_ERR_INVALID_ARG), (dict(sm_scale=0.0), clsa.CLSA_ERR_INVALID_ARG), (dict(num_layers=0), clsa.CLSA_ERR_INVALID_ARG),
         (dict(head_dim=64), clsa.CLSA_ERR_UNSUPPORTED), (dict(idx_dim=96), clsa.CLSA_ERR_UNSUPPORTED),
         (dict(num_q_heads=34, num_kv_heads=2), clsa.CLSA_ERR_UNSUPPORTED),
@@ -94,6 +94,16 @@ def test_bad_arguments_are_refused_on_the_host(clsa):
     assert raw.clsa_sparse_attn(P(_good(clsa, k_cache=0x10004)), 0x50000, 0x60000, 0x70000, 0x80000, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
     assert raw.clsa_sparse_attn(P(_good(clsa, kv_head_stride=64)), 0x50000, 0x60000, 0x70000, 0x80000, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
     assert raw.clsa_sparse_attn(P(good), 0x50000, 0x60000, 0x70000, 0x80000, None, None, wsb, st) == clsa.CLSA_ERR_WORKSPACE
+    # decode launches need their merge scratch, whose size depends on the device: without one the call stops at the device query
+    too_small = (clsa.CLSA_ERR_WORKSPACE, clsa.CLSA_ERR_CUDA)
+    assert raw.clsa_sparse_attn(P(good), 0x50000, 0x60000, 0x70000, 0x80000, None, ws, 256, st) in too_small
+    for bad in (clsa.make_hints(reverse=2), clsa.make_hints(shared_gpu=-1), clsa.make_hints(shared_gpu=3), clsa.make_hints(keep_rows=7), clsa.make_hints(only_q_pending=2)):
+        assert raw.clsa_sparse_attn_hinted(P(good), 0x50000, 0x60000, 0x70000, 0x80000, None, P(bad), ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+        assert raw.clsa_gather_probe(P(good), 0x60000, 0x70000, P(bad), ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_sparse_attn_hinted(P(good), None, 0x60000, 0x70000, 0x80000, None, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_gather_probe(P(good), None, 0x70000, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_gather_probe(P(good), 0x60000, 0x70000, None, ws, 256, st) in too_small
+    assert raw.clsa_gather_probe(P(_good(clsa, q_per_seq=4, max_seq_len=1024)), 0x60000, 0x70000, None, ws, wsb, st) == clsa.CLSA_ERR_UNSUPPORTED
     # decode step
     L = good.num_layers
     qs = (ctypes.c_void_p * L)(0x50000, 0x51000)
@@ -105,15 +115,63 @@ def test_bad_arguments_are_refused_on_the_host(clsa):
     assert raw.clsa_sparse_attn_layers(P(good), qs, 0x60000, 0x70000, qs, None, wsb, st) == clsa.CLSA_ERR_WORKSPACE
     # projections + append
     h, wq, wk, wkk, wv, qo = 0x90000, 0xA0000, 0xB0000, 0xC0000, 0xD0000, 0xE0000
-    assert raw.clsa_project_append(P(good), 2560, None, wq, wk, wkk, wv, qo, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
-    assert raw.clsa_project_append(P(good), 2560, h, wq, wk, wkk, None, qo, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG  # K without V
-    assert raw.clsa_project_append(P(good), 2560, h, wq + 8, wk, None, None, qo, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
-    assert raw.clsa_project_append(P(good), 0, h, wq, wk, None, None, qo, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
-    assert raw.clsa_project_append(P(good), 2568, h, wq, wk, None, None, qo, ws, wsb, st) == clsa.CLSA_ERR_UNSUPPORTED
-    assert raw.clsa_project_append(P(_good(clsa, k_cache=None)), 2560, h, wq, wk, wkk, wv, qo, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
-    assert raw.clsa_project_append(P(good), 2560, h, wq, wk, None, None, qo, None, wsb, st) == clsa.CLSA_ERR_WORKSPACE
+    ko, kk, vv = 0x30000, 0x10000, 0x20000   # the writable cache pointers
+    assert raw.clsa_project_append(P(good), 2560, None, wq, wk, wkk, wv, qo, ko, kk, vv, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_project_append(P(good), 2560, h, wq, wk, wkk, None, qo, ko, kk, vv, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG  # K without V
+    assert raw.clsa_project_append(P(good), 2560, h, wq + 8, wk, None, None, qo, ko, None, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_project_append(P(good), 0, h, wq, wk, None, None, qo, ko, None, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_project_append(P(good), 2568, h, wq, wk, None, None, qo, ko, None, None, ws, wsb, st) == clsa.CLSA_ERR_UNSUPPORTED
+    assert raw.clsa_project_append(P(good), 2560, h, wq, wk, wkk, wv, qo, ko, None, vv, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG  # weights without a cache to write
+    assert raw.clsa_project_append(P(good), 2560, h, wq, wk, None, None, qo, ko, kk, vv, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG  # a cache without weights
+    assert raw.clsa_project_append(P(good), 2560, h, wq, wk, None, None, qo, None, None, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw.clsa_project_append(P(good), 2560, h, wq, wk, None, None, qo, ko, None, None, None, wsb, st) == clsa.CLSA_ERR_WORKSPACE
     assert raw.clsa_clear_status(None, 0, st) == clsa.CLSA_ERR_WORKSPACE
     assert raw.clsa_device_status(None, None, st) == clsa.CLSA_ERR_INVALID_ARG
+
+
+def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
+    """clsa_chain_plan (the host-side model behind the chained layers' launch shapes) needs no GPU. A shape that has
+    not been seen must cost microseconds, not milliseconds -- a server whose batch size keeps changing pays it on the
+    step that first sees a shape -- and shapes are remembered beyond a handful; two models that differ only in the
+    number of KV heads must not share an entry."""
+    import time
+
+    def plan(**kw):
+        return clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, **kw), 148, 1965000)
+
+    assert plan(num_seqs=16) in ((2, 2), (2, 4), (3, 0), (2, 6), (2, 8))      # the headline: a short finer tail
+    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16), 132, 1755000) == (0, 0)  # a device the model was not measured on
+    shapes = [dict(num_seqs=b, top_k=k) for b in range(1, 51) for k in (1024, 2048)]
+    t0 = time.perf_counter()
+    first = [clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, num_layers=16, **sh), 148, 1965000) for sh in shapes]
+    cold = (time.perf_counter() - t0) / len(shapes)
+    t0 = time.perf_counter()
+    again = [clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, num_layers=16, **sh), 148, 1965000) for sh in shapes[-60:]]
+    warm = (time.perf_counter() - t0) / 60
+    assert again == first[-60:]
+    assert cold < 100e-6, f"{cold * 1e6:.1f} us per unseen shape (ctypes call included)"
+    assert warm < 30e-6, f"{warm * 1e6:.1f} us per remembered shape"
+    # The memo may never hand one model's answer to another (models that share heads per block and rows but differ in
+    # the number of KV heads have different block counts): whatever was asked before, the answer is the same. Two
+    # fresh processes ask the same 72 models in opposite orders and must agree on every one.
+    code = (
+        "import sys, json; sys.path.insert(0, %r); import paper_2606_06467_b200 as c\n"
+        "cfgs = [(b, hq, hkv, k) for b in (4, 8, 12, 16, 20, 32) for hq, hkv in ((32, 8), (64, 16), (16, 4), (20, 4)) for k in (1024, 2048, 4096)]\n"
+        "cfgs = cfgs[::-1] if sys.argv[1] == 'r' else cfgs\n"
+        "out = {}\n"
+        "for b, hq, hkv, k in cfgs:\n"
+        "    p = c.make_params(num_seqs=b, num_q_heads=hq, num_kv_heads=hkv, idx_dim=128, top_k=k, num_layers=16, max_seq_len=131072, sm_scale=0.1)\n"
+        "    out[str((b, hq, hkv, k))] = c.clsa_chain_plan(p, 148, 1965000)\n"
+        "print(json.dumps(out, sort_keys=True))\n" % ROOT)
+    fwd = subprocess.check_output([sys.executable, "-c", code, "f"])
+    rev = subprocess.check_output([sys.executable, "-c", code, "r"])
+    assert fwd == rev and len(fwd) > 500
+    # paged caches, prefill chunks and single layers keep one shape
+    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16, block_table=0x5000, block_size=16, max_blocks_per_seq=8192), 148, 1965000) == (0, 0)
+    assert plan(num_seqs=16, q_per_seq=4) == (0, 0) and clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=1, num_seqs=16), 148, 1965000) == (0, 0)
+    n = ctypes.c_int32(0)
+    assert clsa.raw().clsa_chain_plan(ctypes.byref(_good(clsa)), 0, 1965000, ctypes.byref(n), ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
+    assert clsa.raw().clsa_chain_plan(ctypes.byref(_good(clsa)), 148, 1965000, None, ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
 
 
 def test_binding_raises_with_the_status(clsa):

@@ -79,7 +79,7 @@ def test_full_size_prefill_chunk():
     T, n, k = cfg.q_per_seq, cfg.ctx, cfg.top_k
     gs = g.index_scores()
     gi, gc = g.topk(gs)
-    outs = [g.sparse_attn(l, sweep=l, lse=False)[0] for l in range(2)]
+    outs = [g.sparse_attn(l, reverse=l, lse=False)[0] for l in range(2)]
     torch.cuda.synchronize()
     assert g.status() == 0
     # every row: count, range, order, finiteness

@@ -17,10 +17,14 @@ entry._load_build_module().build()
 
 import oracle
 import paper_2606_06467_b200 as clsa
-from _harness import GpuProblem, check_attention, check_scores, check_topk_band, check_topk_exact_on_gpu_scores
+from _harness import SCORE_RTOL, GpuProblem, check_attention, check_scores, check_topk_band, check_topk_exact_on_gpu_scores
 from workloads import HEADLINE, MID, RAGGED, TINY, Workload
 
 pytestmark = pytest.mark.gpu
+
+
+def _bf16_bits(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
 def _full_oracle(w):
@@ -42,36 +46,37 @@ def _run_all(w, layers=None, check_lse=True):
     idx_np, cnt_np = gi.cpu().numpy().copy(), gc.cpu().numpy().copy()
     singles = []
     for l in range(g.L):
-        # the shape for a launch on its own (the whole GPU on one layer) ...
-        out, lse = g.sparse_attn(l, sweep=l & 1)
+        # a launch on its own (the whole GPU on one layer), walking forwards or backwards ...
+        out, lse = g.sparse_attn(l, reverse=l & 1)
         check_attention(prob, w, l, out, lse if check_lse else None, idx_np, cnt_np)
-        # ... and the shape the chain uses (a few large blocks per layer, one direction): the same result to rounding
-        out1, lse1 = g.sparse_attn(l, sweep=0, plan=1)
+        # ... the same when only q is pending (row copies start before the launch waits for its predecessor) ...
+        out_e, lse_e = g.sparse_attn(l, reverse=l & 1, only_q_pending=1, keep_rows=1)
+        assert torch.equal(out.view(torch.int16), out_e.view(torch.int16)), "hints that do not change the split change nothing"
+        # ... and the shapes the chain uses (a few large blocks per layer, one direction): the same result to rounding
+        keep = 1 if l + 1 < g.L else 0
+        out1, lse1 = g.sparse_attn(l, shared_gpu=1, keep_rows=keep)
         check_attention(prob, w, l, out1, lse1 if check_lse else None, idx_np, cnt_np)
         assert (out.float() - out1.float()).abs().max().item() <= 2e-2
         # ... and its finer variant, which a chain may use for its last layers
-        out2, lse2 = g.sparse_attn(l, sweep=0, plan=2)
+        out2, lse2 = g.sparse_attn(l, shared_gpu=2, keep_rows=keep)
         check_attention(prob, w, l, out2, lse2 if check_lse else None, idx_np, cnt_np)
         singles.append((out1, out2))
-    # the chain: same index for all layers, byte-identical to the separate calls in the chain's launch shape
+    # the chain: same index for all layers, byte-identical to the separate calls in the chain's launch shapes
     g.idx.fill_(-7); g.count.fill_(-7)
     outs = g.decode_step()
     torch.cuda.synchronize()
     np.testing.assert_array_equal(g.idx.cpu().numpy(), idx_np)
     np.testing.assert_array_equal(g.count.cpu().numpy(), cnt_np)
-    def shape_of_rows(o, l):
-        """Per query row: 1 or 2 = the side-by-side shape whose separate call gives these bits, 0 if both do (a
-        row whose selected set fits one token range comes out the same however it is split)."""
-        rows = o.shape[0] * o.shape[1]
-        a, b1, b2 = (x.reshape(rows, -1).view(torch.int16) for x in (o, singles[l][0], singles[l][1]))
-        eq1, eq2 = (a == b1).all(dim=1), (a == b2).all(dim=1)
-        assert bool((eq1 | eq2).all()), f"layer {l}: chain != separate call"
-        return torch.where(eq1 & eq2, 0, torch.where(eq1, 1, 2)).cpu().tolist()
-
-    # the finer shape only in a tail of the (layer, row) order: some last rows of one layer, then whole layers
-    shapes = [x for l in range(g.L) for x in shape_of_rows(outs[l], l) if x != 0]
-    assert shapes == sorted(shapes), f"the finer shape is used for a tail only: {shapes}"
-    g.fine_layers = sum(1 for l in range(g.L) if 2 in shape_of_rows(outs[l], l))
+    props = torch.cuda.get_device_properties(0)
+    fine_layers, fine_rows = clsa.clsa_chain_plan(g.params, props.multi_processor_count, props.clock_rate)
+    rows = w.cfg.num_seqs * w.cfg.q_per_seq
+    for l in range(g.L):
+        # which shape each query row of this layer takes, as clsa_chain_plan reports it
+        n_fine = rows if l >= g.L - fine_layers else (fine_rows if l == g.L - fine_layers - 1 else 0)
+        a, b1, b2 = (x.reshape(rows, -1).view(torch.int16) for x in (outs[l], singles[l][0], singles[l][1]))
+        assert torch.equal(a[: rows - n_fine], b1[: rows - n_fine]), f"layer {l}: chain != separate call (shape 1)"
+        assert torch.equal(a[rows - n_fine:], b2[rows - n_fine:]), f"layer {l}: chain != separate call (shape 2)"
+    g.fine_layers = fine_layers
     # the attention half of the chain on its own, fed the index that is already there
     layer_outs = [g.new_out() for _ in range(g.L)]
     clsa.clsa_sparse_attn_layers(g.params, [g.t["q_layers"][l] for l in range(g.L)], g.idx, g.count, layer_outs, g.ws)
@@ -111,11 +116,34 @@ def test_ragged_with_duplicates_and_short_sequences():
 def test_chain_with_finer_last_layers():
     """The headline's launch geometry at a context the oracle handles in seconds: 16 layers of 32 blocks do not fill
     148 SMs evenly, so the chain gives its last layers the finer shape; every layer still equals the separate call of
-    its shape bit for bit, and the oracle within tolerance."""
+    its shape bit for bit, and the oracle within tolerance. The launches with the GPU to themselves cut 128 (row, KV
+    head) units over 148 blocks: spans that end inside a unit, partials merged across blocks."""
     w = Workload(MID.replace(num_seqs=16, ctx=4096, top_k=2048, num_layers=16, seed=31))
     g, _ = _run_all(w, check_lse=False)
     if torch.cuda.get_device_properties(0).multi_processor_count == 148:
-        assert 1 <= g.fine_layers <= 8, g.fine_layers
+        assert 1 <= g.fine_layers <= 3, g.fine_layers
+
+
+@pytest.mark.parametrize("B,k,heads", [(20, 512, (32, 8)), (5, 1000, (20, 4)), (37, 96, (32, 8)), (3, 4096, (8, 1)), (1, 333, (32, 8)),
+                                       (87, 200, (32, 8)), (21, 2048, (32, 8))])
+def test_standalone_attention_at_awkward_batch_sizes(B, k, heads):
+    """A launch that has the GPU to itself cuts its work at token granularity when whole (row, KV head) units would
+    fill the SMs poorly: unit counts that do not divide the SM count (20 and 21 rows: every unit's workers sit in two
+    or three blocks, partials merged across blocks), more units than the workers' even shares allow (87 rows: flat
+    split, spans across unit boundaries, whole units written by one warp), a group of 5 query heads, a single KV
+    head, one sequence; 37 rows fill two rounds exactly and stay with the whole-unit kernel. Every case against the
+    oracle, both walking directions, with and without the early row copies."""
+    w = Workload(MID.replace(num_seqs=B, ctx=max(2 * k, 3000) + 11, top_k=k, num_layers=2, num_q_heads=heads[0],
+                             num_kv_heads=heads[1], seed=500 + B))
+    g = GpuProblem(w)
+    prob = _full_oracle(w)
+    gi, gc = g.topk(g.index_scores())
+    idx_np, cnt_np = gi.cpu().numpy().copy(), gc.cpu().numpy().copy()
+    for l in range(2):
+        out, lse = g.sparse_attn(l, reverse=l, keep_rows=1 - l, only_q_pending=l)
+        check_attention(prob, w, l, out, lse, idx_np, cnt_np)
+    assert g.status() == 0
+    assert g.ws[256: 256 + B * heads[0] * 4].count_nonzero().item() == 0, "the arrival counters are back at zero"
 
 
 def test_planted_tokens_are_selected():
@@ -204,7 +232,7 @@ def test_attention_accepts_any_order_and_flags_bad_indices():
     out_p, lse_p = g.sparse_attn(0, idx=torch.from_numpy(perm).to(g.dev))
     check_attention(prob, w, 0, out_p, lse_p, perm, cnt_np)
     # both sweep directions agree with the oracle
-    out_r, lse_r = g.sparse_attn(0, sweep=1)
+    out_r, lse_r = g.sparse_attn(0, reverse=1)
     check_attention(prob, w, 0, out_r, lse_r, idx_np, cnt_np)
     # empty selection for sequence 1 -> zeros and -inf; sequence 0 untouched
     cnt0 = cnt_np.copy(); cnt0[1, 0] = 0
@@ -257,6 +285,41 @@ def test_sequence_longer_than_max_seq_len_is_skipped_and_flagged():
     clsa.clsa_topk(g.params, s, g.score_stride, g.idx, g.count, g.ws)
     assert g.status() & clsa.CLSA_DEV_BAD_SEQLEN
     assert (g.count.cpu().numpy() == 0).all() and torch.isnan(s).all()
+
+
+@pytest.mark.parametrize("block_size", [0, 16])
+def test_attention_alone_skips_sequences_outside_their_declared_bounds(block_size):
+    """clsa_sparse_attn accepts any caller-built index, so it cannot rely on the top-k to have refused a sequence
+    whose length lies outside [T, max_seq_len]: such a sequence is treated as count 0 (zeros, lse = -inf) and
+    flagged, and its index entries never become addresses -- contiguous and paged caches alike (with paging an
+    entry beyond max_blocks_per_seq * block_size would index past the sequence's row of the block table)."""
+    w = Workload(MID.replace(num_seqs=3, ctx=4000, top_k=128, num_layers=1, seed=77))
+    g = GpuProblem(w, block_size=block_size)
+    prob = _full_oracle(w)
+    gi, gc = g.topk(g.index_scores())
+    idx_np, cnt_np = gi.cpu().numpy().copy(), gc.cpu().numpy().copy()
+    base, base_lse = g.sparse_attn(0)
+    check_attention(prob, w, 0, base, base_lse, idx_np, cnt_np)
+    assert g.status() == 0
+    lens = g.t["seq_len"].clone()
+    g.t["seq_len"][1] = 10 ** 6            # far beyond max_seq_len (and beyond the block table's row)
+    big = idx_np.copy()
+    big[1, 0, :] = np.arange(128) * 7000   # positions that would be "valid" for such a length
+    out, lse = g.sparse_attn(0, idx=torch.from_numpy(big).to(g.dev))
+    torch.cuda.synchronize()
+    assert g.status() & clsa.CLSA_DEV_BAD_SEQLEN
+    assert (out[1].float() == 0).all() and torch.isneginf(lse[1]).all()
+    for b in (0, 2):
+        assert torch.equal(out[b].view(torch.int16), base[b].view(torch.int16))
+    clsa.clsa_clear_status(g.ws)
+    g.t["seq_len"][1] = 0                  # shorter than T
+    out, lse = g.sparse_attn(0)
+    assert g.status() & clsa.CLSA_DEV_BAD_SEQLEN
+    assert (out[1].float() == 0).all() and torch.isneginf(lse[1]).all()
+    clsa.clsa_clear_status(g.ws)
+    g.t["seq_len"].copy_(lens)
+    out, _ = g.sparse_attn(0)
+    assert g.status() == 0 and torch.equal(out.view(torch.int16), base.view(torch.int16))
 
 
 def test_non_finite_scores_never_fault_and_keep_the_index_contract():
@@ -341,8 +404,11 @@ def test_uncleared_workspace_header_is_flagged():
     want = torch.full((B, 1, n), float("nan"), dtype=torch.float32, device=dev)
     clsa.clsa_index_scores(p, q, want, n, good_ws)
     assert clsa.clsa_device_status(good_ws) == 0
-    ref = torch.einsum("bd,bnd->bn", q[:, 0].float(), kidx.view(B, n, 128).float())
-    assert (want[:, 0] - ref).abs().max().item() < 1e-3 * ref.abs().max().item()
+    ref = oracle.Problem(num_seqs=B, num_q_heads=32, num_kv_heads=8, head_dim=128, idx_dim=128, top_k=64, sm_scale=0.1,
+                         seq_start=seq_start.cpu().numpy(), seq_len=seq_len.cpu().numpy(),
+                         idx_k_cache=_bf16_bits(kidx)).index_scores(_bf16_bits(q), score_stride=n)
+    err = np.abs(want.cpu().numpy().astype(np.float64) - ref)
+    assert (err <= SCORE_RTOL * np.maximum(1.0, np.abs(ref))).all()
     assert good_ws[:256].count_nonzero().item() == 0                 # the counters are back at zero
     bad_ws = torch.zeros_like(good_ws)
     bad_ws[:256].view(torch.int32)[16] = 1 << 30                     # as if the header had never been cleared
@@ -360,7 +426,7 @@ def test_score_kernel_on_demand_tiles_cover_every_row_once(d_idx, paged):
     """Launches large enough for the on-demand part of the score kernel's schedule (ragged lengths, both indexer
     widths, contiguous and paged caches -- blocks shorter and longer than a warp's run of rows): every visible position gets its score, nothing beyond it is written, a
     second launch on the same workspace gives the same bits (the counters went back to zero), and the values match
-    a plain fp32 product."""
+    the oracle's fp64 scores within the score tolerance."""
     B, n_max = 24, 131072
     dev = torch.device("cuda:0")
     rng = np.random.default_rng(11 + d_idx)
@@ -402,15 +468,13 @@ def test_score_kernel_on_demand_tiles_cover_every_row_once(d_idx, paged):
     assert clsa.clsa_device_status(ws) == 0
     assert ws[:256].count_nonzero().item() == 0
     assert torch.equal(outs[0].nan_to_num(nan=-7.0), outs[1].nan_to_num(nan=-7.0))
-    got = outs[0][:, 0]
+    got = outs[0][:, 0].cpu().numpy().astype(np.float64)
+    ref = oracle.Problem(num_seqs=B, num_q_heads=32, num_kv_heads=8, head_dim=128, idx_dim=d_idx, top_k=64, sm_scale=0.1,
+                         seq_start=seq_start.cpu().numpy(), seq_len=lens, idx_k_cache=_bf16_bits(kidx),
+                         block_table=table.numpy() if paged else None,
+                         block_size=bs if paged else 0).index_scores(_bf16_bits(q), score_stride=n_max)[:, 0]
     for b in range(B):
         n = int(lens[b])
-        if paged:
-            pos = torch.arange(n, device=dev)
-            r = table_d[b, pos // bs].long() * bs + pos % bs
-        else:
-            r = int(seq_start[b]) + torch.arange(n, device=dev)
-        ref = kidx[r].float() @ q[b, 0].float()
-        assert not torch.isnan(got[b, :n]).any(), b
-        assert torch.isnan(got[b, n:]).all(), b
-        assert (got[b, :n] - ref).abs().max().item() <= 1e-3 * max(1.0, ref.abs().max().item()), b
+        assert not np.isnan(got[b, :n]).any(), b
+        assert np.isnan(got[b, n:]).all(), b
+        assert (np.abs(got[b, :n] - ref[b, :n]) <= SCORE_RTOL * np.maximum(1.0, np.abs(ref[b, :n]))).all(), b

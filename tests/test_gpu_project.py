@@ -35,7 +35,9 @@ def run_gpu(gp, proj, with_kv=True):
     c = gp.cfg
     q = torch.full((c.num_seqs, c.q_per_seq, c.idx_dim), float("nan"), dtype=torch.bfloat16, device=gp.dev)
     clsa.clsa_project_append(gp.params, c.d_model, proj["h"], proj["w_q_idx"], proj["w_k_idx"],
-                             proj["w_k"] if with_kv else None, proj["w_v"] if with_kv else None, q, gp.ws)
+                             proj["w_k"] if with_kv else None, proj["w_v"] if with_kv else None, q,
+                             gp.t["idx_k_cache"], gp.t["k_cache"] if with_kv else None,
+                             gp.t["v_cache"] if with_kv else None, gp.ws)
     torch.cuda.synchronize()
     return q
 
