@@ -261,7 +261,11 @@ CLSA_API clsa_status clsa_decode_step_static(const clsa_params* p, const void* q
  * shared-memory ring -- with the arithmetic, the queries and the outputs left out. Timing it on rows that are, or
  * are not, resident in L2 gives the rate the memory system delivers to this access pattern, the ceiling that the
  * attention kernel is measured against. T must be 1. hints as for clsa_sparse_attn_hinted (NULL = all zero;
- * shared_gpu and only_q_pending are ignored: the probe is the shape of a launch that has the GPU to itself). Writes only into the workspace (which must be the whole clsa_workspace_bytes). */
+ * shared_gpu and only_q_pending are ignored: the probe is the shape of a launch that has the GPU to itself). Writes
+ * only into the workspace (which must be the whole clsa_workspace_bytes). It leaves its own device-side duration in
+ * the workspace header, free of launch overheads: bytes 8..15 hold the bitwise complement of the earliest start of
+ * any of its warps and bytes 16..23 the latest end, both uint64 nanoseconds of the GPU's global timer; both words
+ * accumulate by maximum, so clear the header (clsa_clear_status) before a launch that is to be read. */
 CLSA_API clsa_status clsa_gather_probe(const clsa_params* p, const int32_t* idx, const int32_t* count,
                                        const clsa_attn_hints* hints, void* workspace, size_t workspace_bytes,
                                        clsa_stream stream);

@@ -120,6 +120,8 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_sk_kernel(const SkA
   const int s_begin = has_work ? span_begin(w, split) : 0;
   const int s_end = has_work ? (w + 1 < W ? span_begin(w + 1, split) : a.total_stages) : 0;
 
+  unsigned long long probe_t0 = 0;
+  if (PROBE) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(probe_t0));
   unsigned char* ring = smem + warp * kWarpRingBytes;
   const uint32_t ring_u32 = smem_u32(ring);
   uint32_t* stage_mask = reinterpret_cast<uint32_t*>(smem + WARPS * kWarpRingBytes) + warp * kAttnStages;
@@ -471,6 +473,15 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_sk_kernel(const SkA
   wait_now();  // a warp without work still takes part in the launch's dependency protocol
   if (PROBE) {
     if (has_work) reinterpret_cast<uint32_t*>(a.part)[(int64_t)w * 32 + lane] = probe_sum;
+    // The launch's own duration, for the caller to read: the earliest start (as its complement, so that both words
+    // accumulate by maximum from a cleared header) and the latest end over all warps, in globaltimer nanoseconds.
+    if (lane == 0 && a.status != nullptr) {
+      unsigned long long t1;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+      unsigned long long* clockwords = reinterpret_cast<unsigned long long*>(a.status);
+      atomicMax(clockwords + 1, ~probe_t0);
+      atomicMax(clockwords + 2, t1);
+    }
     return;
   }
   __syncthreads();  // every partial of this block is parked (shared-memory and global writes of the block are visible)

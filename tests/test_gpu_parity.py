@@ -478,3 +478,30 @@ def test_score_kernel_on_demand_tiles_cover_every_row_once(d_idx, paged):
         assert not np.isnan(got[b, :n]).any(), b
         assert np.isnan(got[b, n:]).all(), b
         assert (np.abs(got[b, :n] - ref[b, :n]) <= SCORE_RTOL * np.maximum(1.0, np.abs(ref[b, :n]))).all(), b
+
+
+def test_gather_probe_runs_the_access_pattern_and_reports_its_duration():
+    """The measurement aid: the attention launch's memory accesses without its arithmetic. It writes only into the
+    workspace, flags what the attention kernel would flag, and leaves its device-side duration in the header."""
+    w = Workload(MID.replace(num_seqs=5, ctx=30000, top_k=1024, num_layers=1, seed=3))
+    g = GpuProblem(w)
+    gi, gc = g.topk(g.index_scores())
+    before = [g.t[k].clone() for k in ("k_cache", "v_cache")]
+    clsa.clsa_clear_status(g.ws)
+    clsa.clsa_gather_probe(g.params, gi, gc, clsa.make_hints(reverse=1, keep_rows=1), g.ws)
+    torch.cuda.synchronize()
+    words = g.ws[:32].view(torch.int64).cpu().numpy().view(np.uint64)
+    assert int(words[0]) & 0xFFFFFFFF == 0, "no device flag"
+    start, end = int(~words[1]) & 0xFFFFFFFFFFFFFFFF, int(words[2])
+    assert 0 < end - start < 5_000_000, "duration in nanoseconds of the global timer"
+    for k, b in zip(("k_cache", "v_cache"), before):
+        assert torch.equal(g.t[k], b)
+    bad = gi.clone()
+    bad[2, 0, 17] = 10 ** 8
+    clsa.clsa_clear_status(g.ws)
+    clsa.clsa_gather_probe(g.params, bad, gc, None, g.ws)
+    assert g.status() & clsa.CLSA_DEV_BAD_INDEX
+    clsa.clsa_clear_status(g.ws)
+    # the attention kernel still works on the same workspace afterwards
+    out, lse = g.sparse_attn(0)
+    check_attention(_full_oracle(w), w, 0, out, lse, gi.cpu().numpy(), gc.cpu().numpy())
