@@ -352,7 +352,7 @@ class Problem:
         self.q_layers = [t["q_layers"][l] for l in range(L)]
         self.outs = [torch.empty((c.num_seqs, T, c.num_q_heads, c.head_dim), dtype=torch.bfloat16, device=dev) for _ in range(L)]
         self.stride = (w.max_seq_len + 63) // 64 * 64
-        self.scores = torch.empty((c.num_seqs, T, self.stride), dtype=torch.float32, device=dev)
+        self.scores = torch.empty((c.num_seqs, T, self.stride), dtype=torch.float32, device=dev) if T == 1 else None
         self.alg_bytes = w.algorithmic_bytes()
         self.key_bytes = int(w.seq_len.astype("int64").sum()) * c.idx_dim * 2
         self.gathered_per_layer = int(w.selected_counts().sum()) * c.num_kv_heads * c.head_dim * 4
@@ -363,8 +363,14 @@ class Problem:
         return self.clsa.make_hints(reverse=l & 1, keep_rows=l + 1 < self.L, only_q_pending=l > 0)
 
     def routing(self, q_idx=None):
+        """Eq. 3. Decoding: the two public calls (scores in a buffer of the caller's). A prefill chunk: clsa_index_topk,
+        which never materialises the T x n score matrix."""
         clsa = self.clsa
-        clsa.clsa_index_scores(self.p, self.t["q_idx"] if q_idx is None else q_idx, self.scores, self.stride, self.ws)
+        q_idx = self.t["q_idx"] if q_idx is None else q_idx
+        if self.T > 1:
+            clsa.clsa_index_topk(self.p, q_idx, self.idx, self.cnt, self.ws)
+            return
+        clsa.clsa_index_scores(self.p, q_idx, self.scores, self.stride, self.ws)
         clsa.clsa_topk(self.p, self.scores, self.stride, self.idx, self.cnt, self.ws)
 
     def layers_one_by_one(self, q_list=None, out_list=None, between=None):
@@ -514,25 +520,41 @@ def breakdown(clsa, torch, timer, pr, nb):
 
 
 def chunk_breakdown(clsa, torch, timer, pr, nb):
-    """Per-call microseconds of a prefill chunk's step."""
+    """Per-call microseconds of a prefill chunk's step: the fused routing (clsa_index_topk) and the L layers; and, for
+    comparison, the routing as the two materialising calls (a T x n fp32 score matrix written and read back)."""
     stream = timer.stream
-    acc = {"index_scores": [], "topk": [], "sparse_attn": []}
+    acc = {"index_topk_fused": [], "sparse_attn": []}
     for i in range(nb + 1):
         timer.flush()
-        m = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        m = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
         m[0].record(stream)
-        clsa.clsa_index_scores(pr.p, pr.t["q_idx"], pr.scores, pr.stride, pr.ws)
+        clsa.clsa_index_topk(pr.p, pr.t["q_idx"], pr.idx, pr.cnt, pr.ws)
         m[1].record(stream)
-        clsa.clsa_topk(pr.p, pr.scores, pr.stride, pr.idx, pr.cnt, pr.ws)
-        m[2].record(stream)
         clsa.clsa_sparse_attn_layers(pr.p, pr.q_layers, pr.idx, pr.cnt, pr.outs, pr.ws)
-        m[3].record(stream)
+        m[2].record(stream)
         torch.cuda.synchronize()
         if i >= 1:
             for j, k in enumerate(acc):
                 acc[k].append(m[j].elapsed_time(m[j + 1]) * 1e3)
     out = {k: statistics.median(v) for k, v in acc.items()}
     out["sparse_attn_per_layer"] = out["sparse_attn"] / pr.L
+    scores = torch.empty((pr.c.num_seqs, pr.T, pr.stride), dtype=torch.float32, device=pr.dev)
+    idx2, cnt2 = torch.empty_like(pr.idx), torch.empty_like(pr.cnt)
+    pair = {"index_scores": [], "topk": []}
+    for i in range(3):
+        timer.flush()
+        m = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        m[0].record(stream)
+        clsa.clsa_index_scores(pr.p, pr.t["q_idx"], scores, pr.stride, pr.ws)
+        m[1].record(stream)
+        clsa.clsa_topk(pr.p, scores, pr.stride, idx2, cnt2, pr.ws)
+        m[2].record(stream)
+        torch.cuda.synchronize()
+        if i >= 1:
+            for j, k in enumerate(pair):
+                pair[k].append(m[j].elapsed_time(m[j + 1]) * 1e3)
+    out["materialising_pair"] = {k: statistics.median(v) for k, v in pair.items()}
+    assert torch.equal(idx2, pr.idx) and torch.equal(cnt2, pr.cnt), "fused routing differs from the materialising pair"
     return out
 
 

@@ -70,6 +70,10 @@ typedef enum {
 #define CLSA_DEV_BAD_WORKSPACE 16u /* the workspace header was not zero before its first use (the score kernel found its
                                       scheduling counters out of range): results are invalid */
 
+#define CLSA_DEV_ROUTING_OVERFLOW 32u /* clsa_index_topk: more rows than its scratch holds had to be recomputed from the
+                                        full score row (long runs of equal scores, non-finite scores); the surplus rows
+                                        have count 0: route them with clsa_index_scores + clsa_topk */
+
 typedef void* clsa_stream; /* a cudaStream_t */
 
 typedef struct {
@@ -137,6 +141,21 @@ CLSA_API clsa_status clsa_index_scores(const clsa_params* p, const void* q_idx, 
  * Scores must be finite; a NaN is ordered by its bit pattern and never faults. */
 CLSA_API clsa_status clsa_topk(const clsa_params* p, const float* scores, int64_t score_stride, int32_t* idx,
                       int32_t* count, void* workspace, size_t workspace_bytes, clsa_stream stream);
+
+/* Eq. 3 in one call: S = TopK(Q_idx K_idx^T, k) per (b,t), the same idx and count as clsa_index_scores followed by
+ * clsa_topk, bit for bit. For a prefill chunk (T > 1) the T x n score matrix is never written to memory: the
+ * contraction runs on the tensor cores once over a sample of the keys, which gives every query row a pivot safely
+ * below its k-th largest score, and once over all keys with an epilogue that keeps only the scores not below the
+ * pivot as (score, position) candidates; an exact selection over the candidates gives the index. Rows whose
+ * candidates cannot give the exact answer (long runs of equal scores at the threshold, non-finite scores) are
+ * recomputed through a small scratch matrix; if more than 64 rows of one call need that, the surplus rows get
+ * count 0 and CLSA_DEV_ROUTING_OVERFLOW is set (see there). Shapes the fused route does not take (k so large, or rows
+ * so long, that its fixed-size lists or bitmaps would not hold them) and T == 1 run the two calls internally, with
+ * the scores in the workspace.
+ *   q_idx bf16 [B][T][d_idx], 16-byte aligned;  idx int32 [B][T][k], count int32 [B][T] as for clsa_topk
+ * Needs p->num_cache_rows when T > 1 and the whole workspace of clsa_workspace_bytes. */
+CLSA_API clsa_status clsa_index_topk(const clsa_params* p, const void* q_idx, int32_t* idx, int32_t* count, void* workspace,
+                                     size_t workspace_bytes, clsa_stream stream);
 
 /* Eq. 4 for ONE layer: for each (b,t) and query head h with KV head g = h / (Hq/Hkv),
  *   O = sum_{s in S} softmax_s(sm_scale * Q[b][t][h] . K[s][g]) V[s][g]   over the selected rows only.

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_PKG, "libclsa.so")
 
 CLSA_OK, CLSA_ERR_INVALID_ARG, CLSA_ERR_UNSUPPORTED, CLSA_ERR_WORKSPACE, CLSA_ERR_CUDA = range(5)
 CLSA_DEV_BAD_INDEX, CLSA_DEV_BAD_SEQLEN, CLSA_DEV_BAD_COUNT, CLSA_DEV_TIMEOUT, CLSA_DEV_BAD_WORKSPACE = 1, 2, 4, 8, 16
+CLSA_DEV_ROUTING_OVERFLOW = 32
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -54,6 +55,7 @@ _vp, _i64, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
 _lib.clsa_workspace_bytes.argtypes = [_P, ctypes.POINTER(_sz)]
 _lib.clsa_index_scores.argtypes = [_P, _vp, _vp, _i64, _vp, _sz, _vp]
 _lib.clsa_topk.argtypes = [_P, _vp, _i64, _vp, _vp, _vp, _sz, _vp]
+_lib.clsa_index_topk.argtypes = [_P, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_sparse_attn.argtypes = [_P, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.clsa_sparse_attn_hinted.argtypes = [_P, _vp, _vp, _vp, _vp, _vp, _H, _vp, _sz, _vp]
 _lib.clsa_gather_probe.argtypes = [_P, _vp, _vp, _H, _vp, _sz, _vp]
@@ -67,12 +69,12 @@ _lib.clsa_device_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32), _vp]
 _lib.clsa_status_string.argtypes = [ctypes.c_int]
 _lib.clsa_status_string.restype = ctypes.c_char_p
 _lib.clsa_version.restype = ctypes.c_int
-for _name in ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_sparse_attn_hinted",
+for _name in ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_index_topk", "clsa_sparse_attn", "clsa_sparse_attn_hinted",
               "clsa_gather_probe", "clsa_decode_step", "clsa_decode_step_static", "clsa_sparse_attn_layers",
               "clsa_project_append", "clsa_chain_plan", "clsa_clear_status", "clsa_device_status"):
     getattr(_lib, _name).restype = ctypes.c_int
 
-EXPORTS = ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_sparse_attn", "clsa_sparse_attn_hinted",
+EXPORTS = ("clsa_workspace_bytes", "clsa_index_scores", "clsa_topk", "clsa_index_topk", "clsa_sparse_attn", "clsa_sparse_attn_hinted",
            "clsa_gather_probe", "clsa_decode_step", "clsa_decode_step_static", "clsa_sparse_attn_layers",
            "clsa_project_append", "clsa_chain_plan", "clsa_clear_status", "clsa_device_status", "clsa_status_string",
            "clsa_version")
@@ -158,6 +160,12 @@ def clsa_index_scores(p, q_idx, scores, score_stride, workspace, workspace_bytes
 def clsa_topk(p, scores, score_stride, idx, count, workspace, workspace_bytes=None, stream=None) -> None:
     _check(_lib.clsa_topk(ctypes.byref(p), _ptr(scores), score_stride, _ptr(idx), _ptr(count), _ptr(workspace),
                           _nbytes(workspace, workspace_bytes), _stream(stream)), "clsa_topk")
+
+
+def clsa_index_topk(p, q_idx, idx, count, workspace, workspace_bytes=None, stream=None) -> None:
+    """Eq. 3 in one call (scores + TopK); for a prefill chunk the score matrix is never materialised."""
+    _check(_lib.clsa_index_topk(ctypes.byref(p), _ptr(q_idx), _ptr(idx), _ptr(count), _ptr(workspace),
+                                _nbytes(workspace, workspace_bytes), _stream(stream)), "clsa_index_topk")
 
 
 def clsa_sparse_attn(p, q, idx, count, out, lse, workspace, workspace_bytes=None, stream=None) -> None:

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libclsa.so")
-SOURCES = ["api.cu", "index_scores.cu", "index_gemm.cu", "topk.cu", "topk_filter.cu", "sparse_attn.cu", "sparse_attn_sk.cu", "project_append.cu"]
+SOURCES = ["api.cu", "index_scores.cu", "index_gemm.cu", "index_topk.cu", "topk.cu", "topk_filter.cu", "sparse_attn.cu", "sparse_attn_sk.cu", "project_append.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",

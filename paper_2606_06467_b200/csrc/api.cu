@@ -47,7 +47,9 @@ WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& de
   w.scores_off = w.attn_off + w.attn_bytes;
   w.score_stride = ((int64_t)p.max_seq_len + 63) / 64 * 64;
   w.scores_bytes = align((size_t)p.num_seqs * p.q_per_seq * w.score_stride * sizeof(float));
-  w.total = w.scores_off + w.scores_bytes;
+  // a prefill chunk's fused routing (clsa_index_topk) uses the same bytes for its own scratch instead
+  const size_t fused = p.q_per_seq > 1 ? index_topk_scratch_bytes(p) : 0;
+  w.total = w.scores_off + (w.scores_bytes > fused ? w.scores_bytes : fused);
   return w;
 }
 
@@ -221,6 +223,34 @@ clsa_status clsa_topk(const clsa_params* p, const float* scores, int64_t score_s
   if (!device_info(&dev)) return CLSA_ERR_CUDA;
   return from_cuda(launch_topk(*p, scores, score_stride, idx, count, static_cast<uint32_t*>(workspace), dev,
                                static_cast<cudaStream_t>(stream)));
+}
+
+clsa_status clsa_index_topk(const clsa_params* p, const void* q_idx, int32_t* idx, int32_t* count, void* workspace,
+                            size_t workspace_bytes, clsa_stream stream) {
+  CLSA_TRY(check_shape(p));
+  CLSA_TRY(check_seq(p));
+  CLSA_TRY(check_idx_cache(p));
+  if (q_idx == nullptr || idx == nullptr || count == nullptr) return CLSA_ERR_INVALID_ARG;
+  if (!aligned(q_idx, 16) || !aligned(idx, 4) || !aligned(count, 4)) return CLSA_ERR_INVALID_ARG;
+  if (p->q_per_seq > 1) {
+    if (p->num_cache_rows < 1 || p->num_cache_rows > 0x7fffffffLL) return CLSA_ERR_INVALID_ARG;
+    if ((int64_t)p->num_seqs * p->q_per_seq > 0x7fffffffLL) return CLSA_ERR_INVALID_ARG;
+  }
+  if (workspace == nullptr || !aligned(workspace, 256)) return CLSA_ERR_WORKSPACE;
+  DeviceInfo dev;
+  if (!device_info(&dev)) return CLSA_ERR_CUDA;
+  const WorkspaceLayout w = make_workspace_layout(*p, dev);
+  CLSA_TRY(check_workspace(workspace, workspace_bytes, w.total));
+  auto base = static_cast<unsigned char*>(workspace);
+  auto status = reinterpret_cast<uint32_t*>(base);
+  auto s = static_cast<cudaStream_t>(stream);
+  if (p->q_per_seq > 1 && index_topk_fits(*p, dev))
+    return from_cuda(launch_index_topk(*p, q_idx, idx, count, base + w.scores_off, status, dev, s));
+  auto scores = reinterpret_cast<float*>(base + w.scores_off);
+  cudaError_t err = p->q_per_seq > 1 ? launch_index_scores_gemm(*p, q_idx, scores, w.score_stride, status, dev, s)
+                                     : launch_index_scores_decode(*p, q_idx, scores, w.score_stride, status, status + kSchedWord, dev, s);
+  if (err != cudaSuccess) return CLSA_ERR_CUDA;
+  return from_cuda(launch_topk(*p, scores, w.score_stride, idx, count, status, dev, s));
 }
 
 clsa_status clsa_sparse_attn_hinted(const clsa_params* p, const void* q, const int32_t* idx, const int32_t* count,

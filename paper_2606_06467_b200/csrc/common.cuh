@@ -94,6 +94,39 @@ cudaError_t launch_index_scores_decode(const clsa_params& p, const void* q_idx, 
                                        uint32_t* status, uint32_t* sched, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
                                      uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+// Buffers of the fused chunk routing (clsa_index_topk, T > 1) that the GEMM's filtering and hand-back modes use.
+struct GemmFused {
+  const float* pivot;          // [rows] per query row: keys scoring below it cannot be among the row's k largest
+  uint2* cand;                 // [rows][cand_cap] (score bits, position) candidates
+  uint32_t* cand_count;        // [rows] candidates appended (may exceed cand_cap: the row overflowed)
+  int cand_cap;
+  const int32_t* slot_of_row;  // [rows] scratch row of a query row that was handed back, or -1
+  const uint32_t* qblock_flag; // [num_seqs * ceil(T / 128)] query blocks that hold a handed-back row
+  const uint32_t* nslots;      // rows handed back so far
+};
+cudaError_t launch_index_gemm_sample(const clsa_params& p, const void* q_idx, float* sample, int64_t sample_stride,
+                                     int sample_gs, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_index_gemm_filter(const clsa_params& p, const void* q_idx, const GemmFused& fx, uint32_t* status,
+                                     const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_index_gemm_handed_back(const clsa_params& p, const void* q_idx, float* scratch, int64_t score_stride,
+                                          const GemmFused& fx, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+// Scores and TopK of a prefill chunk in one go, the score matrix never materialised (index_topk.cu). `scratch` is
+// index_topk_scratch_bytes(p) bytes, 256-byte aligned; fits = false: the shape is outside what the fused route
+// handles (the caller materialises the scores instead).
+bool index_topk_fits(const clsa_params& p, const DeviceInfo& dev);
+size_t index_topk_scratch_bytes(const clsa_params& p);
+cudaError_t launch_index_topk(const clsa_params& p, const void* q_idx, int32_t* idx, int32_t* count, unsigned char* scratch,
+                              uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+// Exact TopK of every row from its candidate list (topk_filter.cu); rows that cannot be finished get count = -1.
+int topk_candidates_capacity();  // entries per row's list
+size_t topk_candidates_smem(int max_seq_len, const DeviceInfo& dev);
+cudaError_t launch_topk_candidates(const clsa_params& p, const uint2* cand, const uint32_t* cand_count, const float* pivot,
+                                   int32_t* idx, int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+// The general top-k kernel for the rows listed in row_of_slot[0 .. *nslots), row j reading row j of `scores`.
+cudaError_t launch_topk_slots(const clsa_params& p, const float* scores, int64_t score_stride, const int32_t* row_of_slot,
+                              const uint32_t* nslots, int max_slots, int32_t* idx, int32_t* count, uint32_t* status,
+                              const DeviceInfo& dev, cudaStream_t stream);
+
 cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx, int32_t* count,
                         uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 bool topk_prefilter_fits(const clsa_params& p, const float* scores, int64_t score_stride, const DeviceInfo& dev);

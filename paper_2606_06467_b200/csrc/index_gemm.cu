@@ -58,6 +58,26 @@ struct GemmArgs {
   // (block_size < 256), or as one box inside a block (block_size >= 256). Contiguous: one box, no table.
   const int32_t* block_table;
   int block_size, max_blocks_per_seq, box_rows, key_boxes;
+  // Sampling (sample_gs > 0): the "keys" of this launch are groups of 16 consecutive positions spaced sample_gs
+  // positions apart (a multiple of 16), column j of the output standing for position (j / 16) * sample_gs + j % 16;
+  // only groups that lie wholly inside a sequence count, and every query sees all of them (the caller applies the
+  // causal rule when it reads the sample). A key tile is then sixteen 16-row boxes, like a paged tile.
+  int sample_gs;
+  // Tile order. 0: query block fastest, tiles dealt round-robin (neighbouring SMs share a key tile in L2).
+  // 1: key tile fastest and every block takes one contiguous run of tiles, so that a block stays on the same 128
+  // queries for a long time (the filtering epilogue keeps per-query state between tiles).
+  int row_major;
+  // MODE 1 (filter): per query row, the score below which a key cannot be among the k largest; keys at or above it
+  // are appended as (score bits, position) pairs to the row's candidate list.
+  const float* pivot;
+  uint2* cand;
+  uint32_t* cand_count;
+  int cand_cap;
+  // MODE 2 (rows handed back): only query blocks with a set flag are computed, and only rows with a slot are stored,
+  // row `slot` of `scores`.
+  const int32_t* slot_of_row;
+  const uint32_t* qblock_flag;
+  const uint32_t* nslots;
 };
 
 // ---- PTX wrappers ----------------------------------------------------------------------------------
@@ -138,20 +158,33 @@ struct TileCoord {
 };
 // The same enumeration for every role: tile id -> (sequence, query block, key tile); valid == 0 for
 // tiles of a sequence with a bad length and for tiles wholly above the causal diagonal.
+template <int MODE>
 __device__ __forceinline__ TileCoord tile_coord(const GemmArgs& a, int64_t id) {
   TileCoord c;
   const int per_seq = a.m_blocks * a.n_tiles;
   c.b = (int)(id / per_seq);
   const int rem = (int)(id - (int64_t)c.b * per_seq);
-  c.nt = rem / a.m_blocks;
-  c.mb = rem - c.nt * a.m_blocks;
+  if (a.row_major) {
+    c.mb = rem / a.n_tiles;
+    c.nt = rem - c.mb * a.n_tiles;
+  } else {
+    c.nt = rem / a.m_blocks;
+    c.mb = rem - c.nt * a.m_blocks;
+  }
   c.n = a.seq_len[c.b];
+  const bool n_ok = c.n >= a.q_per_seq && c.n <= a.max_seq_len;
+  if (a.sample_gs > 0) c.n = n_ok ? (c.n / a.sample_gs) * 16 : 0;  // sampled columns: whole groups inside the sequence
   const int t_last = min(a.q_per_seq, (c.mb + 1) * kBM) - 1;
-  const int v_max = a.causal ? c.n - a.q_per_seq + t_last + 1 : c.n;
-  c.valid = (c.n >= a.q_per_seq && c.n <= a.max_seq_len && c.nt * kBN < v_max) ? 1 : 0;
+  const int v_max = (a.causal && a.sample_gs == 0) ? c.n - a.q_per_seq + t_last + 1 : c.n;
+  c.valid = (n_ok && c.nt * kBN < v_max) ? 1 : 0;
+  if (MODE == 2 && c.valid) c.valid = a.qblock_flag[c.b * a.m_blocks + c.mb] != 0u ? 1 : 0;
   return c;
 }
 
+// MODE 0: the scores are stored (clsa_index_scores; also the sampling pass of clsa_index_topk).
+// MODE 1: the scores are compared with a per-row pivot in registers and only candidates leave the SM (clsa_index_topk).
+// MODE 2: MODE 0 for the few rows that clsa_index_topk hands back, into a small scratch matrix.
+template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_s, const GemmArgs a) {
@@ -169,7 +202,14 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.idx_dim / kBK;  // 1 or 2
+  const bool causal = a.causal != 0 && a.sample_gs == 0;
   const int64_t total_tiles = (int64_t)a.num_seqs * a.m_blocks * a.n_tiles;
+  // this block's tiles: first, first + step, ... below last
+  const int64_t per_block = (total_tiles + gridDim.x - 1) / gridDim.x;
+  const int64_t tile_first = a.row_major ? (int64_t)blockIdx.x * per_block : (int64_t)blockIdx.x;
+  const int64_t tile_step = a.row_major ? 1 : (int64_t)gridDim.x;
+  const int64_t tile_last = a.row_major ? min(total_tiles, tile_first + per_block) : total_tiles;
+  if (MODE == 2 && *a.nslots == 0u) return;  // nothing was handed back (the usual case): before any barrier or TMEM use
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -191,14 +231,23 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // Lane 0 owns the barriers and the query tile; key boxes are spread over the lanes (lane i fetches box i),
     // so that a tile made of sixteen 16-row cache blocks does not queue 32 copies behind one thread.
     uint32_t it = 0;
-    for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
-      const TileCoord c = tile_coord(a, id);
+    for (int64_t id = tile_first; id < tile_last; id += tile_step) {
+      const TileCoord c = tile_coord<MODE>(a, id);
       if (!c.valid) continue;
       const int s = it % kStages;
       const uint32_t ph = (it / kStages) & 1u;
       // first cache row of this lane's key box (looked up before the wait, used after it)
       int krow = 0, boxes = 1;
-      if (a.block_table == nullptr) {
+      if (a.sample_gs > 0) {
+        // sixteen 16-row groups, sample_gs positions apart; groups past the sequence's last whole one are not fetched
+        const int group = c.nt * 16 + lane;
+        boxes = min(16, c.n / 16 - c.nt * 16);
+        if (lane < boxes) {
+          const int pos = group * a.sample_gs;
+          if (a.block_table == nullptr) krow = (int)(a.seq_start[c.b] + pos);
+          else krow = a.block_table[(int64_t)c.b * a.max_blocks_per_seq + pos / a.block_size] * a.block_size + pos % a.block_size;
+        }
+      } else if (a.block_table == nullptr) {
         krow = (int)(a.seq_start[c.b] + (int64_t)c.nt * kBN);
       } else {
         const int32_t* tab = a.block_table + (int64_t)c.b * a.max_blocks_per_seq;
@@ -233,8 +282,8 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_bf16(kBM, kBN);
       uint32_t it = 0;
-      for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
-        const TileCoord c = tile_coord(a, id);
+      for (int64_t id = tile_first; id < tile_last; id += tile_step) {
+        const TileCoord c = tile_coord<MODE>(a, id);
         if (!c.valid) continue;
         const int s = it % kStages, acc = it % kAccBufs;
         const uint32_t ph = (it / kStages) & 1u, aph = (it / kAccBufs) & 1u;
@@ -261,9 +310,40 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // ---------------- epilogue: TMEM -> registers -> global ----------------
     const int quad = warp & 3;          // TMEM lanes 32*quad .. 32*quad+31 (a warp may only touch its own quadrant)
     const int half = (warp - 4) >> 2;   // which 128 of the tile's 256 columns
+    // MODE 1: a lane appends its row's candidates straight to the row's list in global memory, into runs of kRun slots
+    // that it reserves with one atomic add each. A warp's scoreboard tracks a register for all lanes at once, so an
+    // atomic whose result any lane still waits for would stall every lane that touches the same register: the runs
+    // are therefore requested only at tile starts, by one convergent instruction into `f_pending`, which nothing reads
+    // before the next tile start (a whole tile later: the result has long arrived); there it becomes the lane's spare
+    // run, and a lane that fills its current run in the middle of a tile switches to the spare without touching an
+    // outstanding request. Only a lane that uses up both inside one tile reserves on the spot. When the block moves on
+    // to other queries, what is left of the runs is filled with holes (position = kHole), which the select skips.
+    // Entries past the list's capacity are dropped; the count keeps growing, which is how the select learns that the
+    // row overflowed.
+    constexpr uint32_t kRun = 16, kHole = 0xffffffffu;
+    int64_t f_row = -1;
+    float f_pivot = 0.f;
+    uint32_t f_base = 0, f_used = kRun, f_spare = 0, f_pending = 0;
+    bool f_has_spare = false, f_has_pending = false;
+    uint2* f_list = nullptr;
+    auto reserve_run = [&]() -> uint32_t { return atomicAdd(a.cand_count + f_row, kRun); };
+    auto put = [&](uint32_t slot, uint2 e) {
+      if (slot < (uint32_t)a.cand_cap) f_list[slot] = e;
+    };
+    auto close_runs = [&]() {  // the row is done for this lane: the unused slots become holes
+      if (MODE != 1 || f_list == nullptr) return;
+      for (uint32_t e = f_used; e < kRun; ++e) put(f_base + e, make_uint2(0u, kHole));
+      if (f_has_spare)
+        for (uint32_t e = 0; e < kRun; ++e) put(f_spare + e, make_uint2(0u, kHole));
+      if (f_has_pending)
+        for (uint32_t e = 0; e < kRun; ++e) put(f_pending + e, make_uint2(0u, kHole));
+      f_list = nullptr;
+      f_used = kRun;
+      f_has_spare = f_has_pending = false;
+    };
     uint32_t it = 0;
-    for (int64_t id = blockIdx.x; id < total_tiles; id += gridDim.x) {
-      const TileCoord c = tile_coord(a, id);
+    for (int64_t id = tile_first; id < tile_last; id += tile_step) {
+      const TileCoord c = tile_coord<MODE>(a, id);
       if (!c.valid) continue;
       const int acc = it % kAccBufs;
       const uint32_t aph = (it / kAccBufs) & 1u;
@@ -271,8 +351,98 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       tc_fence_after();
       const int t = c.mb * kBM + quad * 32 + lane;       // query of this thread's row
       const bool row_ok = t < a.q_per_seq;
-      const int v = row_ok ? (a.causal ? c.n - a.q_per_seq + t + 1 : c.n) : 0;  // visible keys of this query
+      const int v = row_ok ? (causal ? c.n - a.q_per_seq + t + 1 : c.n) : 0;  // visible keys of this query
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kBN);
+      // columns this warp has to drain: up to the last one any of its 32 queries can see (a multiple of 32)
+      const int v_warp = __reduce_max_sync(0xffffffffu, v) - c.nt * kBN;
+      const int c_begin = half * (kBN / 2);
+      const int c_end = min(c_begin + kBN / 2, (max(v_warp, 0) + 31) & ~31);
+      if (MODE == 1) {
+        // ---- filter: compare with the row's pivot in registers; only candidates leave the SM ----
+        const int64_t row = (int64_t)c.b * a.q_per_seq + t;
+        if (row != f_row) {           // the block moved on to other queries
+          close_runs();
+          f_row = row;
+          f_pivot = __int_as_float(0x7f800000);
+          if (row_ok) {
+            f_pivot = a.pivot[row];
+            // a row with +inf needs no candidates at all
+            if (f_pivot < __int_as_float(0x7f800000)) f_list = a.cand + row * a.cand_cap;
+          }
+        }
+        if (f_list != nullptr) {      // tile start: last tile's request becomes the spare run, and a new one goes out
+          if (f_has_pending && !f_has_spare) { f_spare = f_pending; f_has_spare = true; f_has_pending = false; }
+          if (!f_has_pending) { f_pending = reserve_run(); f_has_pending = true; }
+        }
+        uint32_t ra[32], rb[32];
+        // The warp's staging tile (32 rows x 128 bytes, 16-byte chunk c of row r at r * 128 + ((c ^ (r & 7)) << 4), free
+        // of bank conflicts for a row per lane) holds the chunk so that a lane can fetch the few columns that pass by
+        // index: a lane's pass mask costs one compare per column, and only its own set bits cost anything more.
+        unsigned char* tile = base_ptr + kStages * kStageBytes + (warp - 4) * 4096;
+        auto filter32 = [&](const uint32_t (&r)[32], int s0) {
+          // Two instructions per column: the sign of (score - pivot) is shifted into a mask by a funnel shift. Four
+          // chains of 8 columns, highest column first, so that column i ends up at bit i. The difference of a NaN is the
+          // canonical (positive) NaN: it passes, like everything that is not below the pivot.
+          uint32_t sg[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+          for (int j = 7; j >= 0; --j) {
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4)
+              sg[q4] = __funnelshift_l(__float_as_uint(__uint_as_float(r[q4 * 8 + j]) - f_pivot), sg[q4], 1);
+          }
+          uint32_t mask = ~((sg[0] & 0xffu) | ((sg[1] & 0xffu) << 8) | ((sg[2] & 0xffu) << 16) | (sg[3] << 24));
+          if (s0 + 32 > v) mask &= s0 >= v ? 0u : (0xffffffffu >> (32 - (v - s0)));
+          if (f_list == nullptr) mask = 0u;
+          if (__any_sync(0xffffffffu, mask != 0u) == 0) return;
+          __syncwarp();  // the previous chunk's reads of the tile are done
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch)
+            *reinterpret_cast<uint4*>(tile + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
+                make_uint4(r[4 * ch], r[4 * ch + 1], r[4 * ch + 2], r[4 * ch + 3]);
+          // a lane reads back only what it wrote: no barrier needed in between
+          while (mask != 0u) {
+            const int i = __ffs(mask) - 1;
+            mask &= mask - 1u;
+            const uint32_t bits = *reinterpret_cast<const uint32_t*>(tile + lane * 128 + (((i >> 2) ^ (lane & 7)) << 4) + (i & 3) * 4);
+            if (f_used == kRun) {  // the current run is full: take the spare, or (rarely) reserve on the spot
+              if (f_has_spare) { f_base = f_spare; f_has_spare = false; }
+              else f_base = reserve_run();
+              f_used = 0;
+            }
+            put(f_base + f_used, make_uint2(bits, (uint32_t)(s0 + i)));
+            ++f_used;
+          }
+        };
+        if (c_end > c_begin) tc_ld32(taddr + (uint32_t)c_begin, ra);
+#pragma unroll 1
+        for (int c0 = c_begin; c0 < c_end; c0 += 64) {
+          tc_ld_wait();
+          if (c0 + 32 < c_end) tc_ld32(taddr + (uint32_t)(c0 + 32), rb);
+          filter32(ra, c.nt * kBN + c0);
+          if (c0 + 32 < c_end) {
+            tc_ld_wait();
+            if (c0 + 64 < c_end) tc_ld32(taddr + (uint32_t)(c0 + 64), ra);
+            filter32(rb, c.nt * kBN + c0 + 32);
+          }
+        }
+      } else if (MODE == 2) {
+        // ---- rows handed back: a lane stores its own row (if it has a slot) as it comes from TMEM ----
+        const int64_t row = (int64_t)c.b * a.q_per_seq + t;
+        const int slot = row_ok ? a.slot_of_row[row] : -1;
+        float* dst_row = a.scores + (int64_t)max(slot, 0) * a.score_stride;
+        uint32_t ra[32];
+#pragma unroll 1
+        for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+          tc_ld32(taddr + (uint32_t)c0, ra);
+          tc_ld_wait();
+          const int s0 = c.nt * kBN + c0;
+          if (slot >= 0) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (s0 + i < v) dst_row[s0 + i] = __uint_as_float(ra[i]);
+          }
+        }
+      } else {
       // 32 columns at a time through two register buffers (the TMEM load of the next 32 columns is in flight
       // while the current 32 are stored). A TMEM load leaves a lane with 32 columns of ONE row; stored as they
       // come, a warp instruction would scatter 32-byte pieces over 32 rows. They go through a padded
@@ -287,7 +457,7 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       const uint32_t tile_u32 = smem_u32(tile);
       const int t0 = c.mb * kBM + quad * 32;  // first query row of this warp
       // every key below v_all is visible to all 32 rows (under the causal rule the first row sees the fewest)
-      const int v_all = (t0 + 31 < a.q_per_seq) ? (a.causal ? c.n - a.q_per_seq + t0 + 1 : c.n) : 0;
+      const int v_all = (t0 + 31 < a.q_per_seq) ? (causal ? c.n - a.q_per_seq + t0 + 1 : c.n) : 0;
       auto store32 = [&](const uint32_t (&r)[32], int s0) {
         // the copy engine must have finished reading the tile's previous contents; so must the other lanes
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -312,7 +482,7 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         for (int k = 0; k < 4; ++k) {
           const int row = k * 8 + (lane >> 2);
           const int tq = t0 + row;
-          const int vr = tq < a.q_per_seq ? (a.causal ? c.n - a.q_per_seq + tq + 1 : c.n) : 0;
+          const int vr = tq < a.q_per_seq ? (causal ? c.n - a.q_per_seq + tq + 1 : c.n) : 0;
           if (s >= vr) continue;
           const int ch = (lane & 3) * 2;
           const float4 w0 = *reinterpret_cast<const float4*>(tile + row * 128 + ((ch ^ (row & 7)) << 4));
@@ -330,10 +500,6 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
           }
         }
       };
-      // columns this warp has to drain: up to the last one any of its 32 queries can see (a multiple of 32)
-      const int v_warp = __reduce_max_sync(0xffffffffu, v) - c.nt * kBN;
-      const int c_begin = half * (kBN / 2);
-      const int c_end = min(c_begin + kBN / 2, (max(v_warp, 0) + 31) & ~31);
       uint32_t ra[32], rb[32];
       if (c_end > c_begin) tc_ld32(taddr + (uint32_t)c_begin, ra);
 #pragma unroll 1
@@ -347,12 +513,14 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
           store32(rb, c.nt * kBN + c0 + 32);
         }
       }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));        // one arrival per epilogue warp frees the accumulator
       ++it;
     }
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // this warp's bulk stores have landed
+    close_runs();
+    if (MODE == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // this warp's bulk stores have landed
   }
 
   tc_fence_before();
@@ -415,22 +583,26 @@ bool make_map_f32(CUtensorMap* map, void* ptr, uint64_t rows, uint64_t row_strid
 
 }  // namespace
 
-cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
-                                     uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
+namespace {
+
+// One launch of the chunk GEMM. mode 0: scores are stored into `scores` (sample_gs > 0: the sampled columns only);
+// mode 1: filtered against fx.pivot into fx.cand; mode 2: rows with a slot are stored into row `slot` of `scores`.
+cudaError_t launch_gemm(int mode, const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
+                        int sample_gs, const GemmFused* fx, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
   CUtensorMap map_q, map_k;
   const uint64_t q_rows = (uint64_t)p.num_seqs * p.q_per_seq;
   if (!make_map(&map_q, q_idx, q_rows, (uint64_t)p.idx_dim, (uint64_t)p.idx_dim, kBM)) return cudaErrorInvalidValue;
   const bool paged = p.block_table != nullptr;
-  const int box_rows = paged && p.block_size < kBN ? p.block_size : kBN;
+  const int box_rows = sample_gs > 0 ? 16 : (paged && p.block_size < kBN ? p.block_size : kBN);
   if (!make_map(&map_k, p.idx_k_cache, (uint64_t)p.num_cache_rows, (uint64_t)p.idx_dim, (uint64_t)p.idx_token_stride,
                 (uint32_t)box_rows))
     return cudaErrorInvalidValue;
-  // fp32 scores [B*T][score_stride], box = 32 columns x 32 rows, for the epilogue's tiled bulk stores (only when the
-  // rows are 32-byte aligned; otherwise the map is a valid dummy over the key cache and is never used)
-  const bool vec_ok = score_stride % 8 == 0 && reinterpret_cast<uintptr_t>(scores) % 32 == 0;
+  // fp32 scores [rows][score_stride], box = 32 columns x 32 rows, for the storing epilogue's tiled bulk stores (only
+  // when the rows are 32-byte aligned; otherwise the map is a valid dummy over the key cache and is never used)
+  const bool vec_ok = mode == 0 && score_stride % 8 == 0 && reinterpret_cast<uintptr_t>(scores) % 32 == 0;
   CUtensorMap map_s = map_k;
   if (vec_ok && !make_map_f32(&map_s, scores, q_rows, (uint64_t)score_stride)) return cudaErrorInvalidValue;
-  GemmArgs a;
+  GemmArgs a = {};
   a.block_table = p.block_table;
   a.block_size = paged ? p.block_size : 0;
   a.max_blocks_per_seq = p.max_blocks_per_seq;
@@ -447,14 +619,50 @@ cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, fl
   a.max_seq_len = p.max_seq_len;
   a.idx_dim = p.idx_dim;
   a.m_blocks = (p.q_per_seq + kBM - 1) / kBM;
-  a.n_tiles = (p.max_seq_len + kBN - 1) / kBN;
+  const int columns = sample_gs > 0 ? (p.max_seq_len / sample_gs) * 16 : p.max_seq_len;
+  a.n_tiles = (columns + kBN - 1) / kBN;
   a.vec_ok = vec_ok ? 1 : 0;
-  cudaError_t err = cudaFuncSetAttribute(index_scores_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-  if (err != cudaSuccess) return err;
+  a.sample_gs = sample_gs;
+  a.row_major = mode == 0 ? 0 : 1;
+  if (fx != nullptr) {
+    a.pivot = fx->pivot;
+    a.cand = fx->cand;
+    a.cand_count = fx->cand_count;
+    a.cand_cap = fx->cand_cap;
+    a.slot_of_row = fx->slot_of_row;
+    a.qblock_flag = fx->qblock_flag;
+    a.nslots = fx->nslots;
+  }
   const int64_t tiles = (int64_t)p.num_seqs * a.m_blocks * a.n_tiles;
+  if (tiles < 1) return cudaSuccess;
   const int grid = (int)(tiles < dev.sm_count ? tiles : dev.sm_count);
-  index_scores_gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_s, a);
+  auto kernel = mode == 0 ? index_scores_gemm_kernel<0> : mode == 1 ? index_scores_gemm_kernel<1> : index_scores_gemm_kernel<2>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (err != cudaSuccess) return err;
+  kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_s, a);
   return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
+                                     uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
+  return launch_gemm(0, p, q_idx, scores, score_stride, 0, nullptr, status, dev, stream);
+}
+
+cudaError_t launch_index_gemm_sample(const clsa_params& p, const void* q_idx, float* sample, int64_t sample_stride,
+                                     int sample_gs, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
+  return launch_gemm(0, p, q_idx, sample, sample_stride, sample_gs, nullptr, status, dev, stream);
+}
+
+cudaError_t launch_index_gemm_filter(const clsa_params& p, const void* q_idx, const GemmFused& fx, uint32_t* status,
+                                     const DeviceInfo& dev, cudaStream_t stream) {
+  return launch_gemm(1, p, q_idx, nullptr, 0, 0, &fx, status, dev, stream);
+}
+
+cudaError_t launch_index_gemm_handed_back(const clsa_params& p, const void* q_idx, float* scratch, int64_t score_stride,
+                                          const GemmFused& fx, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
+  return launch_gemm(2, p, q_idx, scratch, score_stride, 0, &fx, status, dev, stream);
 }
 
 }  // namespace clsa

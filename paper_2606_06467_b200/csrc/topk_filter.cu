@@ -370,6 +370,184 @@ topk_prefilter_kernel(const float* __restrict__ scores, int64_t score_stride, co
   for (int i = kk + tid; i < top_k; i += kThreads) out[i] = -1;
 }
 
+// ---------------------------------------------------------------------------------------------------------------------
+// Exact TopK of a row from a candidate list that somebody else filtered (the chunk GEMM's epilogue, clsa_index_topk):
+// unordered (score bits, position) pairs that contain every score not below the row's pivot. Steps 4 and 5 of the
+// kernel above on that list; the positions come out ascending through a position bitmap, since the list has no order.
+// A row that cannot be finished exactly from its list -- fewer than k candidates (pivot too high), more than the list
+// holds, a NaN below the pivot, more threshold-equal keys than can be ranked here -- gets count = -1 and is recomputed
+// by the caller.
+constexpr int kEqCap = 1024;  // threshold-equal candidates that are ranked by position here
+
+__global__ void __launch_bounds__(kThreads, 2)
+topk_candidates_kernel(const uint2* __restrict__ cand, const uint32_t* __restrict__ cand_count, int cand_cap,
+                       const float* __restrict__ pivot_of_row, const int32_t* __restrict__ seq_len, int q_per_seq, int causal,
+                       int top_k, int max_seq_len, int bitmap_words, int32_t* __restrict__ idx_out,
+                       int32_t* __restrict__ count_out, uint32_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  FShared& sh = *reinterpret_cast<FShared*>(smem_raw);
+  uint32_t* eq_pos = reinterpret_cast<uint32_t*>(smem_raw + sizeof(FShared));
+  uint32_t* bitmap = eq_pos + kEqCap;  // one bit per position of the row
+
+  const int row = blockIdx.x;
+  const int b = row / q_per_seq, t = row % q_per_seq;
+  const int tid = threadIdx.x, lane = tid & 31;
+  for (int i = tid; i < 4096; i += kThreads) sh.hist[i] = 0u;
+  for (int i = tid; i < 1024; i += kThreads) sh.hist10[i] = 0u;
+  if (tid == 0) { sh.cand_count = 0u; sh.cand_max = 0u; sh.small_count = 0u; sh.below_pivot = 0u; }
+  const int n = seq_len[b];
+  int v = causal ? n - q_per_seq + t + 1 : n;
+  if (n < q_per_seq || n > max_seq_len) {
+    v = 0;
+    if (tid == 0) flag_status(status, CLSA_DEV_BAD_SEQLEN);
+  }
+  const int kk = min(top_k, v);
+  int32_t* out = idx_out + (int64_t)row * top_k;
+  if (kk == v) {  // nothing to select: every visible position is taken, in order
+    if (tid == 0) count_out[row] = kk;
+    for (int i = tid; i < top_k; i += kThreads) out[i] = i < kk ? i : -1;
+    return;
+  }
+  const int words = (v + 31) >> 5;
+  for (int i = tid; i < words; i += kThreads) bitmap[i] = 0u;
+  const uint32_t slots = cand_count[row];  // slots handed out, holes included
+  if (slots > (uint32_t)cand_cap || words > bitmap_words) {
+    if (tid == 0) count_out[row] = -1;
+    return;
+  }
+  const uint32_t pivot = score_key(pivot_of_row[row]);
+  const uint2* list = cand + (int64_t)row * cand_cap;
+  __syncthreads();  // sh.cand_count is zero
+  {
+    // the list's entries without its holes (position = 0xffffffff: a slot that was reserved and not used), in no
+    // particular order
+    uint32_t my_max = 0u, bad = 0u;
+    constexpr int kPerThread = kCandCap / kThreads;  // all of a thread's loads are issued before the first is used
+    uint2 e[kPerThread];
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) {
+      const uint32_t i = (uint32_t)(u * kThreads + tid);
+      e[u] = i < slots ? list[i] : make_uint2(0u, 0xffffffffu);
+    }
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) {
+      if ((uint32_t)(u * kThreads) >= slots) break;  // uniform over the block
+      const bool real = e[u].y != 0xffffffffu;
+      const uint32_t ballot = __ballot_sync(kFull, real);
+      uint32_t at = 0;
+      if (lane == 0 && ballot != 0u) at = atomicAdd(&sh.cand_count, (uint32_t)__popc(ballot));
+      at = __shfl_sync(kFull, at, 0) + __popc(ballot & ((1u << lane) - 1u));
+      if (real) {
+        const uint32_t key = score_key(__uint_as_float(e[u].x));
+        sh.cand_key[at] = key;
+        sh.cand_pos[at] = e[u].y;
+        my_max = max(my_max, key);
+        bad |= (key < pivot || e[u].y >= (uint32_t)v) ? 1u : 0u;  // a NaN with the sign bit set passed the float compare
+      }
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) my_max = max(my_max, __shfl_xor_sync(kFull, my_max, d));
+    if (lane == 0) atomicMax(&sh.cand_max, my_max);
+    if (bad != 0u) sh.below_pivot = 1u;
+  }
+  __syncthreads();
+  const uint32_t C = sh.cand_count;
+  if (sh.below_pivot != 0u || C < (uint32_t)kk) {  // a NaN below the pivot, or the pivot came out above the k-th largest
+    if (tid == 0) count_out[row] = -1;
+    return;
+  }
+  // exact select over the candidates: first digit = top 12 bits of the candidates' actual spread
+  const uint32_t range = sh.cand_max - pivot;
+  const int s = max(0, 32 - __clz(range) - 12);  // range >> s < 4096
+  for (uint32_t i = tid; i < C; i += kThreads) atomicAdd(&sh.hist[(sh.cand_key[i] - pivot) >> s], 1u);
+  __syncthreads();
+  scan_from_top<4096>(sh, sh.hist, (uint32_t)kk);
+  const uint32_t b1 = sh.digit, k1 = sh.k_rem, cnt1 = sh.bin_count;
+  if (cnt1 <= (uint32_t)kSmallBin) {
+    for (uint32_t i = tid; i < C; i += kThreads) {
+      const uint32_t key = sh.cand_key[i];
+      if (((key - pivot) >> s) == b1) sh.small_key[atomicAdd(&sh.small_count, 1u)] = key;
+    }
+    __syncthreads();
+    if (tid < kSmallBin && tid < (int)cnt1) {
+      const uint32_t mine = sh.small_key[tid];
+      uint32_t greater = 0, equal = 0;
+      for (uint32_t j = 0; j < cnt1; ++j) {
+        const uint32_t other = sh.small_key[j];
+        greater += other > mine;
+        equal += other == mine;
+      }
+      if (greater < k1 && k1 <= greater + equal) {
+        sh.thr = mine;
+        sh.need_eq = k1 - greater;
+      }
+    }
+    __syncthreads();
+  } else {
+    uint32_t prefix = b1 << s, mask = s == 0 ? 0xffffffffu : ~((1u << s) - 1u), k_rem = k1;
+    int rest = s;
+#pragma unroll 1
+    while (rest > 0) {
+      const int wbits = min(10, rest), shift = rest - wbits;
+      for (uint32_t i = tid; i < C; i += kThreads) {
+        const uint32_t d = sh.cand_key[i] - pivot;
+        if ((d & mask) == prefix) atomicAdd(&sh.hist10[(d >> shift) & ((1u << wbits) - 1u)], 1u);
+      }
+      __syncthreads();
+      scan_from_top<1024>(sh, sh.hist10, k_rem);
+      prefix |= sh.digit << shift;
+      mask |= ((1u << wbits) - 1u) << shift;
+      k_rem = sh.k_rem;
+      rest = shift;
+    }
+    if (tid == 0) { sh.thr = pivot + prefix; sh.need_eq = k_rem; }
+    __syncthreads();
+  }
+  const uint32_t thr = sh.thr, need_eq = sh.need_eq;  // every key > thr, and the need_eq lowest positions with key == thr
+  // selected positions -> bitmap; threshold-equal ones are collected and, if not all are needed, ranked by position
+  if (tid == 0) sh.small_count = 0u;  // reused: number of threshold-equal candidates
+  __syncthreads();
+  for (uint32_t i = tid; i < C; i += kThreads) {
+    const uint32_t key = sh.cand_key[i], pos = sh.cand_pos[i];
+    if (key > thr) atomicOr(&bitmap[pos >> 5], 1u << (pos & 31u));
+    else if (key == thr) {
+      const uint32_t at = atomicAdd(&sh.small_count, 1u);
+      if (at < (uint32_t)kEqCap) eq_pos[at] = pos;
+    }
+  }
+  __syncthreads();
+  const uint32_t n_eq = sh.small_count;
+  if (n_eq > (uint32_t)kEqCap) {  // a long run of equal scores at the threshold
+    if (tid == 0) count_out[row] = -1;
+    return;
+  }
+  for (uint32_t i = tid; i < n_eq; i += kThreads) {
+    const uint32_t mine = eq_pos[i];
+    uint32_t lower = 0;
+    if (n_eq != need_eq)
+      for (uint32_t j = 0; j < n_eq; ++j) lower += eq_pos[j] < mine;
+    if (lower < need_eq) atomicOr(&bitmap[mine >> 5], 1u << (mine & 31u));
+  }
+  __syncthreads();
+  {
+    const int per = (words + kThreads - 1) / kThreads;  // consecutive bitmap words per thread
+    const int w_lo = min(words, tid * per), w_hi = min(words, w_lo + per);
+    uint32_t mine = 0;
+    for (int w = w_lo; w < w_hi; ++w) mine += __popc(bitmap[w]);
+    uint32_t off = block_excl_scan(sh, mine);
+    for (int w = w_lo; w < w_hi; ++w) {
+      uint32_t bits = bitmap[w];
+      while (bits != 0u) {
+        if (off < (uint32_t)kk) out[off] = (int32_t)(w * 32 + __ffs(bits) - 1);
+        ++off;
+        bits &= bits - 1u;
+      }
+    }
+  }
+  if (tid == 0) count_out[row] = kk;
+  for (int i = kk + tid; i < top_k; i += kThreads) out[i] = -1;
+}
+
 }  // namespace
 
 // Whether the one-sweep kernel can take this launch at all (the caller decides whether it should).
@@ -414,6 +592,35 @@ cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, topk_prefilter_kernel, scores, score_stride, p.seq_len, (int)p.q_per_seq, (int)p.causal,
                             (int)p.top_k, (int)p.max_seq_len, bitmap_words, idx, count, status);
+}
+
+}  // namespace clsa
+
+namespace clsa {
+
+int topk_candidates_capacity() { return kCandCap; }
+
+// Shared memory of topk_candidates_kernel for rows of up to max_seq_len positions (0 if it does not fit two blocks
+// per SM).
+size_t topk_candidates_smem(int max_seq_len, const DeviceInfo& dev) {
+  const int bitmap_words = ((max_seq_len + 31) / 32 + 3) & ~3;
+  const size_t smem = sizeof(FShared) + (size_t)kEqCap * sizeof(uint32_t) + (size_t)bitmap_words * sizeof(uint32_t);
+  const size_t half_sm = ((size_t)dev.max_smem_optin + 1024) / 2 - 1024;
+  return smem <= half_sm ? smem : 0;
+}
+
+cudaError_t launch_topk_candidates(const clsa_params& p, const uint2* cand, const uint32_t* cand_count, const float* pivot,
+                                   int32_t* idx, int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {
+  const size_t smem = topk_candidates_smem(p.max_seq_len, dev);
+  if (smem == 0) return cudaErrorInvalidValue;
+  const int bitmap_words = ((p.max_seq_len + 31) / 32 + 3) & ~3;
+  cudaError_t err = cudaFuncSetAttribute(topk_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
+  topk_candidates_kernel<<<(unsigned)rows, kThreads, smem, stream>>>(cand, cand_count, kCandCap, pivot, p.seq_len, p.q_per_seq,
+                                                                     p.causal, p.top_k, p.max_seq_len, bitmap_words, idx, count,
+                                                                     status);
+  return cudaGetLastError();
 }
 
 }  // namespace clsa

@@ -14,6 +14,7 @@ import __graft_entry__ as entry
 entry._load_build_module().build()
 
 import oracle
+import paper_2606_06467_b200 as clsa
 from _harness import (GpuProblem, check_attention, check_scores, check_topk_band, check_topk_exact_on_gpu_scores,
                       oracle_scores_and_topk)
 from workloads import HEADLINE, MID, RAGGED, Workload
@@ -79,6 +80,11 @@ def test_full_size_prefill_chunk():
     T, n, k = cfg.q_per_seq, cfg.ctx, cfg.top_k
     gs = g.index_scores()
     gi, gc = g.topk(gs)
+    # the fused routing (scores never materialised) gives the same index, bit for bit
+    fi, fc = torch.full_like(gi, -7), torch.full_like(gc, -7)
+    clsa.clsa_index_topk(g.params, g.t["q_idx"], fi, fc, g.ws)
+    torch.cuda.synchronize()
+    assert g.status() == 0 and torch.equal(fc, gc) and torch.equal(fi, gi)
     outs = [g.sparse_attn(l, reverse=l, lse=False)[0] for l in range(2)]
     torch.cuda.synchronize()
     assert g.status() == 0

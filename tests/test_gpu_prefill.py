@@ -19,6 +19,17 @@ from workloads import MID, TINY, Workload
 pytestmark = pytest.mark.gpu
 
 
+def _fused_equals_pair(g, gi, gc):
+    """clsa_index_topk against clsa_index_scores + clsa_topk on the same problem: the same index, bit for bit."""
+    idx = torch.full_like(gi, -7)
+    cnt = torch.full_like(gc, -7)
+    clsa.clsa_index_topk(g.params, g.t["q_idx"], idx, cnt, g.ws)
+    torch.cuda.synchronize()
+    assert g.status() == 0
+    assert torch.equal(cnt, gc)
+    assert torch.equal(idx, gi)
+
+
 def _full_oracle(w):
     kc, vc = w.host_kv_full()
     return oracle.problem_from_workload(w, k_cache=kc, v_cache=vc, idx_k_cache=w.host_kidx_cache())
@@ -44,6 +55,7 @@ def test_chunk_scores_topk_attention(B, T, n, d_idx, causal, ragged):
     check_topk_exact_on_gpu_scores(prob, gs, gi, gc, w)
     ref_idx, ref_cnt = prob.topk(ref_scores)
     check_topk_band(ref_scores, ref_idx, ref_cnt, gi, gc, w)
+    _fused_equals_pair(g, gi, gc)
     idx_np, cnt_np = gi.cpu().numpy().copy(), gc.cpu().numpy().copy()
     for l in range(2):
         out, lse = g.sparse_attn(l, reverse=l)
@@ -79,9 +91,74 @@ def test_chunk_on_paged_caches(B, T, n, d_idx, causal, ragged, bs):
     assert torch.equal(gs.nan_to_num(7.0), flat.index_scores().nan_to_num(7.0))
     gi, gc = g.topk(gs)
     check_topk_exact_on_gpu_scores(prob, gs, gi, gc, w)
+    _fused_equals_pair(g, gi, gc)
     out, lse = g.sparse_attn(0)
     check_attention(prob, w, 0, out, lse, gi.cpu().numpy().copy(), gc.cpu().numpy().copy())
     assert g.status() == 0
+
+
+@pytest.mark.parametrize("B,T,n,d_idx,k,causal,ragged,bs", [
+    (1, 300, 20000, 128, 512, 1, 0, 0), (2, 130, 9000, 64, 96, 1, 7000, 0), (1, 257, 40000, 128, 2048, 1, 0, 0),
+    (2, 140, 12000, 128, 300, 0, 0, 0), (1, 200, 20000, 128, 512, 1, 0, 16), (2, 129, 9000, 64, 200, 1, 6500, 64),
+    (1, 64, 70000, 128, 1024, 1, 0, 256)])
+def test_fused_chunk_routing_on_long_rows(B, T, n, d_idx, k, causal, ragged, bs):
+    """Rows longer than the candidate list: the pivot comes from a sample of the keys, the filter runs in the GEMM's
+    epilogue, the select works on the candidates alone. The index must equal the materialising pair's bit for bit
+    (same tensor-core scores, exact selection) and agree with the oracle under the usual rules; contiguous and paged."""
+    base = MID if d_idx == 128 else TINY
+    cfg = base.replace(num_seqs=B, ctx=n, q_per_seq=T, causal=causal, top_k=k, num_layers=1, seed=4000 + T + n + bs,
+                       ragged_min=ragged, num_short=0)
+    w = Workload(cfg)
+    g = GpuProblem(w, block_size=bs)
+    prob = oracle.problem_from_workload(w, idx_k_cache=w.host_kidx_cache())
+    ref_scores = prob.index_scores(w.q_idx_bits())
+    gs = g.index_scores()
+    gi, gc = g.topk(gs)
+    check_topk_exact_on_gpu_scores(prob, gs, gi, gc, w)
+    ref_idx, ref_cnt = prob.topk(ref_scores)
+    check_topk_band(ref_scores, ref_idx, ref_cnt, gi, gc, w)
+    _fused_equals_pair(g, gi, gc)
+
+
+def test_fused_chunk_routing_hands_back_rows_it_cannot_finish():
+    """Long runs of equal scores at the threshold defeat the candidate list (it would have to hold all of them). Such
+    rows are recomputed through the scratch matrix and still come out bit-identical to the materialising pair; when
+    more rows need that than the scratch holds (64), the surplus rows get count 0 and CLSA_DEV_ROUTING_OVERFLOW is
+    raised, and every other row is still right."""
+    n, T, k = 16000, 100, 256
+    w = Workload(MID.replace(num_seqs=1, ctx=n, q_per_seq=T, causal=1, top_k=k, num_layers=1, seed=77))
+    g = GpuProblem(w)
+    keys = g.t["idx_k_cache"]
+    # queries 0..39: their own key rows are far away; make 9000 cached keys copies of query-aligned directions so that
+    # for the first 40 queries thousands of scores tie exactly at the top
+    q = g.t["q_idx"][0]                                   # [T, d]
+    keys[1000:10000] = 0                                  # 9000 all-zero keys: score exactly 0 for every query
+    big = torch.zeros_like(keys[0]); big[0] = 1.0
+    # rows 0..39 get a negative component on dim 0 for all other keys -> zero-score keys rank at the top for them
+    g.t["q_idx"][0, :40, :] = 0
+    g.t["q_idx"][0, :40, 0] = -1.0
+    keys[:1000, 0] = keys[:1000, 0].abs() + 0.5           # positive dim 0 -> negative scores for queries 0..39
+    keys[10000:, 0] = keys[10000:, 0].abs() + 0.5
+    gs = g.index_scores()
+    gi, gc = g.topk(gs)
+    torch.cuda.synchronize()
+    assert (gs[0, :40, 1000:10000] == 0).all()
+    _fused_equals_pair(g, gi, gc)                         # 40 rows handed back: all fit the scratch
+    # now all 100 queries tie the same way: 100 rows need the scratch, 64 get it
+    g.t["q_idx"][0, :, :] = 0
+    g.t["q_idx"][0, :, 0] = -1.0
+    gs = g.index_scores()
+    gi, gc = g.topk(gs)
+    idx = torch.full_like(gi, -7)
+    cnt = torch.full_like(gc, -7)
+    clsa.clsa_index_topk(g.params, g.t["q_idx"], idx, cnt, g.ws)
+    torch.cuda.synchronize()
+    assert g.status() == clsa.CLSA_DEV_ROUTING_OVERFLOW
+    clsa.clsa_clear_status(g.ws)
+    done = cnt[0] > 0
+    assert int(done.sum()) == 64 and int((cnt[0] == 0).sum()) == T - 64
+    assert torch.equal(idx[0][done], gi[0][done]) and torch.equal(cnt[0][done], gc[0][done])
+    assert (idx[0][~done] == -1).all()
 
 
 def test_gemm_row_equals_decode_gemv():
