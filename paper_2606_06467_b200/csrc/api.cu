@@ -53,6 +53,22 @@ WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& de
   return w;
 }
 
+// L2 policy of a decode launch that has the GPU to itself and whose rows the next launch reads again (a decoder's
+// layers issued one by one). If the selected set of the batch fits in the part of L2 that such a gather can keep
+// (about half of it: rows are held on both sides of the chip), everything is fetched evict_last. If it does not, some
+// of it is evicted before the next layer arrives whatever the order; then of every 8 consecutive 16-token stages the
+// first few -- the share that fits -- are fetched evict_last and the others evict_first: every layer finds the same
+// rows in L2; hits and misses alternate inside every warp's pipeline, so that the L2 port and HBM are busy together
+// instead of one after the other (as they are when a launch first walks what its predecessor left behind and then
+// the rest); and the rows that will not be kept anyway do not push the kept ones out.
+int pinned_stages_of_eight(const clsa_params& p, const DeviceInfo& dev) {
+  const double k_eff = (double)(p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len);
+  const double gathered = (double)p.num_seqs * p.q_per_seq * k_eff * p.num_kv_heads * p.head_dim * 4.0;
+  const double keepable = 0.5 * (double)dev.l2_bytes;
+  const int pin = (int)(8.0 * keepable / gathered + 0.5);
+  return pin >= 8 ? -1 : (pin < 1 ? 1 : pin);
+}
+
 namespace {
 
 bool aligned(const void* ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) == 0; }
@@ -109,10 +125,9 @@ clsa_status check_workspace(const void* ws, size_t ws_bytes, size_t need) {
   return CLSA_OK;
 }
 
-// Below this occupancy of the whole-unit shape a launch with the GPU to itself takes the token-granular kernel
-// (measured on a B200, per layer at k = 2048, 32/8 heads: 1 sequence 10.9 against 12.5 us, 20 sequences 26.1 against
-// 30.4; where the whole-unit shape fills 65 % or more of its rounds it is as fast or faster, its merge staying inside
-// a block).
+// Below this occupancy of the whole-unit shape a launch with the GPU to itself takes the token-granular kernel. Where
+// the whole-unit shape fills about two thirds or more of its rounds it is as fast or faster (its merge stays inside a
+// block, and while the rows come from DRAM idle SMs cost nothing); well below that the idle SMs dominate.
 constexpr double kTokenGranularBelow = 0.6;
 
 #define CLSA_TRY(expr)                     \
@@ -145,7 +160,7 @@ cudaError_t launch_attention(const clsa_params& p, const void* q, const int32_t*
     auto arrive = reinterpret_cast<uint32_t*>(ws_base + w.attn_off);
     auto part = reinterpret_cast<float*>(ws_base + w.attn_part_off);
     return launch_sparse_attn_sk(p, plan, q, idx, count, out, lse, status, arrive, part, h.reverse, wait_prior,
-                                 h.only_q_pending, h.keep_rows, s);
+                                 h.only_q_pending, h.keep_rows, dev, s);
   }
   return launch_sparse_attn(p, q, idx, count, out, lse, status, h.reverse, wait_prior, h.only_q_pending, h.keep_rows,
                             h.shared_gpu, fine_rows, dev, s);
@@ -297,7 +312,7 @@ clsa_status clsa_gather_probe(const clsa_params* p, const int32_t* idx, const in
   auto base = static_cast<unsigned char*>(workspace);
   const SkPlan plan = make_sk_plan(*p, dev);
   return from_cuda(launch_gather_probe(*p, plan, idx, count, reinterpret_cast<uint32_t*>(base),
-                                       reinterpret_cast<float*>(base + w.attn_part_off), h.reverse, h.keep_rows,
+                                       reinterpret_cast<float*>(base + w.attn_part_off), h.reverse, h.keep_rows, dev,
                                        static_cast<cudaStream_t>(stream)));
 }
 

@@ -145,10 +145,14 @@ double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev);
 cudaError_t launch_sparse_attn_sk(const clsa_params& p, const SkPlan& plan, const void* q, const int32_t* idx,
                                   const int32_t* count, void* out, float* lse, uint32_t* status, uint32_t* arrive,
                                   float* part, int reverse, int wait_prior, int only_q_pending, int keep_rows,
-                                  cudaStream_t stream);
+                                  const DeviceInfo& dev, cudaStream_t stream);
 // The same gather without the arithmetic (measurement aid); part as above (used as a sink).
 cudaError_t launch_gather_probe(const clsa_params& p, const SkPlan& plan, const int32_t* idx, const int32_t* count,
-                                uint32_t* status, float* part, int reverse, int keep_rows, cudaStream_t stream);
+                                uint32_t* status, float* part, int reverse, int keep_rows, const DeviceInfo& dev,
+                                cudaStream_t stream);
+// Of every 8 consecutive 16-token stages of a row's selected set, how many a decode launch with the GPU to itself
+// fetches evict_last (the others evict_first) when the next launch reads the same rows again; -1: all of them.
+int pinned_stages_of_eight(const clsa_params& p, const DeviceInfo& dev);
 
 // idx_k_out / k_out / v_out: the caches of p, writable (k_out and v_out may be null together with w_k and w_v)
 cudaError_t launch_project_append(const clsa_params& p, int d_model, const void* h, const void* w_q_idx,

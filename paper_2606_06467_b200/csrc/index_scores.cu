@@ -3,9 +3,9 @@
 //
 // Work split: the (sequence, 128-or-256-row tile) space goes to a persistent grid of 4 blocks per
 // SM: the first three quarters of the tiles round-robin, the rest on demand from a ticket counter
-// (blocks do not all run at the same pace -- with a fixed deal the last of 592 blocks finished
-// 14 us after the first and 7 us after the median, time during which the memory system runs
-// below capacity and the kernel behind this one waits). Inside a tile each warp owns a contiguous run of rows; a key row (d_idx bf16)
+// (blocks do not all run at the same pace -- with a fixed deal the last blocks finish well after
+// the median one, time during which the memory system runs below capacity and the kernel behind
+// this one waits). Inside a tile each warp owns a contiguous run of rows; a key row (d_idx bf16)
 // is covered by d_idx/8 lanes holding 16 bytes each, and every thread keeps 8 independent 16-byte
 // loads in flight (128 KiB per SM at 1024 resident threads), which is what it takes to cover the
 // DRAM latency at full bandwidth. The per-row sum uses one fixed order (8 sequential FMAs per lane,
@@ -179,10 +179,10 @@ cudaError_t launch_index_scores_decode(const clsa_params& p, const void* q_idx, 
   const int64_t total = (int64_t)p.num_seqs * tiles_per_seq;
   int64_t grid = (int64_t)dev.sm_count * 4;
   if (grid > total) grid = total;
-  // three quarters of the tiles by a fixed deal (whole rounds of the grid), the rest on demand. Measured, headline /
-  // ragged step: all by the fixed deal 280 / 829 us, 87 % 274 / 821, 75 % 270 / 823, 50 % 269 / 834 (tiles past the end
-  // of a short sequence cost nothing in the fixed deal but a draw from the one counter on demand). Launches with
-  // only a few tiles per block are dealt whole.
+  // three quarters of the tiles by a fixed deal (whole rounds of the grid), the rest on demand: a larger on-demand
+  // share balances the end of the launch better, but tiles past the end of a short sequence cost nothing in the fixed
+  // deal and a draw from the one counter on demand, which a ragged batch notices. Launches with only a few tiles per
+  // block are dealt whole.
   int64_t static_tiles = total;
   if (total >= 8 * grid) static_tiles = (total * 3 / 4) / grid * grid;
   auto kidx = static_cast<const uint16_t*>(p.idx_k_cache);

@@ -66,6 +66,8 @@ struct AttnArgs {
   int coarse_blocks;  // -1: one block size, 2-D grid. >= 0: a 1-D grid of two block sizes (no cluster, one row per block):
                       // the first coarse_blocks blocks take heads_per_block KV heads each, row by row; the blocks behind
                       // them take half as many (twice the token ranges) and cover the remaining rows
+  int pin;            // -1: one L2 priority for every row (evict_last if keep). 0..8: of every 8 consecutive stages of a row's
+                      // selected set the first `pin` are fetched evict_last and the others evict_first
   int max_seq_len;    // sequences longer than this (or shorter than q_per_seq) are skipped and flagged
   float scale_log2;
 };
@@ -228,7 +230,8 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
     // apart, so what one layer fetches the next ones find in L2. Such launches fetch with the evict_last priority
     // (other traffic through L2 does not push the rows out in between); a launch on its own leaves the replacement
     // policy alone.
-    const uint64_t pol = a.keep ? l2_policy_evict_last() : l2_policy_evict_normal();
+    const uint64_t pol_keep = a.keep ? l2_policy_evict_last() : l2_policy_evict_normal();
+    const uint64_t pol_last = l2_policy_evict_last(), pol_first = l2_policy_evict_first();
     // Per-lane constants of the copies: where in a stage buffer this lane's 16-byte chunk of token j = 2*it + lane/16
     // goes (XOR swizzle), and the lane's byte offset inside a row.
     uint32_t sw[8];
@@ -244,6 +247,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
       if (i < nstages) {
         const int buf = i % kAttnStages;
         const uint32_t kdst = ring_u32 + buf * kStageBytes, vdst = kdst + kStageBytes / 2;
+        const uint64_t pol = a.pin < 0 ? pol_keep : (((stage_t0(i) >> 4) & 7) < a.pin ? pol_last : pol_first);
         // cache row relative to s0: the position itself, or its place inside its block
         const int my_idx = paged ? (blk << a.block_shift) + (raw & ((1 << a.block_shift) - 1)) : raw;
         const bool in_range = raw >= 0 && raw < n && (!a.off32 || (uint64_t)(s0 + my_idx) < (uint64_t)a.rows_max);
@@ -539,8 +543,7 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   plan.warps = p.num_q_heads / p.num_kv_heads <= 8 ? kAttnWarpsNarrow : kAttnWarpsWide;
   const int64_t rows_ = (int64_t)p.num_seqs * p.q_per_seq;
   // Side by side, 32 to 63 rows of 8 or more KV heads: 8 warps can take all 8 heads of a row (32 to 63 blocks per
-  // launch, the shape that works best), which 12 warps cannot (4 heads per block, twice the blocks). Measured at
-  // 32 rows: 631 against 736 us per step.
+  // launch, the shape that works best), which 12 warps cannot (4 heads per block, twice the blocks).
   if (throughput && p.num_kv_heads >= 8 && rows_ * ((p.num_kv_heads + 7) / 8) >= 32 && rows_ * ((p.num_kv_heads + 7) / 8) < 64)
     plan.warps = kAttnWarpsWide;
   plan.smem_bytes = (size_t)plan.warps * kWarpRingBytes + plan.warps * kAttnStages * sizeof(uint32_t);
@@ -801,6 +804,10 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   // fetches all of them with evict_last, so that scores, indices and outputs passing through L2 do not push them
   // out before the layers behind it arrive; a launch on its own leaves the replacement policy alone.
   a.keep = keep_for_next ? 1 : 0;
+  // A launch with the GPU to itself whose rows the next launch reads again keeps the share of them in L2 that fits
+  // there (pinned_stages_of_eight); chained launches trail one another over the same rows and fetch everything
+  // evict_last.
+  a.pin = (keep_for_next && throughput_plan == 0) ? pinned_stages_of_eight(p, dev) : -1;
   a.coarse_blocks = -1;
   a.max_seq_len = p.max_seq_len;
   a.scale_log2 = p.sm_scale * kLog2e;

@@ -35,7 +35,6 @@ namespace clsa {
 namespace {
 
 constexpr int kMergeBatch = 8;
-constexpr int kPinOfEight = 4;  // stages of every 8 that a launch with keep_rows holds in L2 (see the policy in the kernel)
 // Release/acquire fence at GPU scope (what the message-passing pattern of the merge needs; __threadfence() is the
 // sequentially consistent fence, several times as expensive with every block of the grid issuing it at once).
 __device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
@@ -629,7 +628,7 @@ namespace {
 template <bool PROBE>
 cudaError_t launch_sk(const clsa_params& p, const SkPlan& plan, const void* q, const int32_t* idx, const int32_t* count,
                       void* out, float* lse, uint32_t* status, uint32_t* arrive, float* part, int reverse, int wait_prior,
-                      int only_q_pending, int keep_rows, cudaStream_t stream) {
+                      int only_q_pending, int keep_rows, const DeviceInfo& dev, cudaStream_t stream) {
   SkArgs a;
   a.q = static_cast<const uint16_t*>(q);
   a.kc = static_cast<const uint16_t*>(p.k_cache);
@@ -657,13 +656,8 @@ cudaError_t launch_sk(const clsa_params& p, const SkPlan& plan, const void* q, c
   a.wait_prior = wait_prior ? 1 : 0;
   a.early = (wait_prior && only_q_pending) ? 1 : 0;
   a.keep = keep_rows ? 1 : 0;
-  // L2 policy. A launch that has the GPU to itself and whose rows the next launch reads again (a decoder's layers
-  // issued one by one) cannot keep the whole selected set in L2: about half of it stays, whatever the order. Half of
-  // the stages, interleaved with the others, are therefore fetched evict_last and the rest evict_first: the same half
-  // is found in L2 by every layer, hits and misses alternate inside every warp's pipeline (so the L2 port and HBM are
-  // busy together instead of one after the other, as they are when a launch first walks what its predecessor left
-  // behind and then the rest), and the rows that will not be kept anyway do not push the kept ones out.
-  a.pin = keep_rows ? kPinOfEight : -1;
+  // L2 policy of a launch whose rows the next launch reads again: see kPinOfEight.
+  a.pin = keep_rows ? pinned_stages_of_eight(p, dev) : -1;
   // With the extent of the row space known (num_cache_rows) and below 2^32 16-byte units, row offsets are 32-bit.
   a.rows_max = p.num_cache_rows;
   a.off32 = (a.rows_max > 0 && (double)a.rows_max * (double)(p.kv_token_stride >> 3) < 4294967296.0) ? 1 : 0;
@@ -702,15 +696,16 @@ cudaError_t launch_sk(const clsa_params& p, const SkPlan& plan, const void* q, c
 cudaError_t launch_sparse_attn_sk(const clsa_params& p, const SkPlan& plan, const void* q, const int32_t* idx,
                                   const int32_t* count, void* out, float* lse, uint32_t* status, uint32_t* arrive,
                                   float* part, int reverse, int wait_prior, int only_q_pending, int keep_rows,
-                                  cudaStream_t stream) {
+                                  const DeviceInfo& dev, cudaStream_t stream) {
   return launch_sk<false>(p, plan, q, idx, count, out, lse, status, arrive, part, reverse, wait_prior, only_q_pending,
-                          keep_rows, stream);
+                          keep_rows, dev, stream);
 }
 
 cudaError_t launch_gather_probe(const clsa_params& p, const SkPlan& plan, const int32_t* idx, const int32_t* count,
-                                uint32_t* status, float* part, int reverse, int keep_rows, cudaStream_t stream) {
+                                uint32_t* status, float* part, int reverse, int keep_rows, const DeviceInfo& dev,
+                                cudaStream_t stream) {
   return launch_sk<true>(p, plan, nullptr, idx, count, nullptr, nullptr, status, nullptr, part, reverse, 1, 0, keep_rows,
-                         stream);
+                         dev, stream);
 }
 
 }  // namespace clsa

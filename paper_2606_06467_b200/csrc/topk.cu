@@ -650,8 +650,8 @@ static int resident_clusters(int cluster, size_t smem_bytes, bool cached, const 
 }
 
 // Shared memory of a block whose slice of the row is `per` scores: the keys are kept there whenever they fit,
-// even if that leaves one block per SM and several waves (measured: 64 rows of 131072 in two waves of one block
-// per SM 41 us, in one wave of two blocks per SM that re-read their slices from L2 in every sweep 49 us).
+// even if that leaves one block per SM and several waves (two waves of one block per SM beat one wave of two blocks
+// per SM that re-read their slices from L2 in every sweep).
 static void size_blocks(TopkPlan& plan, int max_seq_len, const DeviceInfo& dev) {
   const int per = (((max_seq_len + plan.cluster - 1) / plan.cluster) + 3) & ~3;
   const size_t want = sizeof(Shared) + (size_t)per * sizeof(uint32_t);
@@ -680,8 +680,7 @@ TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev, bool one_sw
   plan.one_sweep = 0;
   size_blocks(plan, p.max_seq_len, dev);
   // In between (9 to about 22 rows): clusters of 6, if they are all resident at once (22 of them on a B200, against
-  // 15 of 7, 8 or 9) -- a third fewer scores per thread in the two sweeps: 1.6 us per step at 12, 16 and 20 rows of
-  // 131072 (the call on its own, with its launch, measures the same 22.5 us either way).
+  // 15 of 7, 8 or 9) -- a third fewer scores per thread in the two sweeps.
   if (pow2 == 4 && rows > 8 && p.max_seq_len / 6 >= 2048) {
     TopkPlan six = plan;
     six.cluster = 6;
@@ -691,9 +690,8 @@ TopkPlan make_topk_plan(const clsa_params& p, const DeviceInfo& dev, bool one_sw
   // Many rows. Far more rows than SMs (a prefill chunk): throughput matters, not the latency of one row; one block
   // per row needs no cluster barriers and keeps more rows in flight. And whenever the clusters of this launch would
   // not all be resident at once, the one-sweep kernel (one block per row, two blocks per SM, one pass over the
-  // scores) is faster than a second wave of clusters, if the shape fits it: 64 rows of 131072 scores 41 -> 34 us,
-  // 200 rows 150 -> 48 us, 400 rows of 32768 68 -> 42 us; 33 rows of 131072, the most that one wave of clusters of 4
-  // holds, 32 us either way.
+  // scores) is faster than a second wave of clusters, if the shape fits it (as fast at the largest launch that one
+  // wave of clusters still holds, and several times faster at a few hundred rows).
   bool many = rows >= 4 * (int64_t)dev.sm_count;
   if (!many && one_sweep_fits && rows > resident_clusters(plan.cluster, plan.smem_bytes, plan.slice_cap > 0, dev)) many = true;
   if (many) {
