@@ -10,6 +10,9 @@ constexpr int kStageBytes = kAttnStageTokens * 256 * 2;  // 16 K rows + 16 V row
 constexpr int kWarpRingBytes = kAttnStages * kStageBytes;
 constexpr int kPartialStride = 132;                      // floats per head of a partial: 128 outputs, max, sum, pad
 constexpr float kLog2e = 1.4426950408889634f;
+// Rank of stage s (mod 8) in the order in which stages are chosen for L2 residency: bit-reversed, so that the pinned
+// stages are spread as evenly as possible over every run of 8 (4 of 8: every other stage).
+__device__ __forceinline__ int pin_rank(int s) { return ((s & 1) << 2) | (s & 2) | ((s & 4) >> 2); }
 constexpr float kLn2 = 0.6931471805599453f;
 
 // 16-byte asynchronous copy global -> shared with an L2 eviction-priority hint.

@@ -235,7 +235,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_sk_kernel(const SkA
         if (i < nstages) {
           const int buf = i % kAttnStages;
           const uint32_t kdst = ring_u32 + buf * kStageBytes, vdst = kdst + kStageBytes / 2;
-          const uint64_t pol = a.pin < 0 ? pol_keep : (((stage_t0(i) >> 4) & 7) < a.pin ? pol_last : pol_first);
+          const uint64_t pol = a.pin < 0 ? pol_keep : (pin_rank((stage_t0(i) >> 4) & 7) < a.pin ? pol_last : pol_first);
           // cache row relative to s0: the position itself, or its place inside its block
           const int my_idx = paged ? (blk << a.block_shift) + (raw & ((1 << a.block_shift) - 1)) : raw;
           const bool in_range = raw >= 0 && raw < n && (!a.off32 || (uint64_t)(s0 + my_idx) < (uint64_t)a.rows_max);
