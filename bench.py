@@ -61,9 +61,12 @@ def parse():
                     help="also time the upstream step (Eq. 2 projections of the new tokens + cache append, "
                          "clsa_project_append) on the same workload; reported under \"projection\", not part of the step")
     ap.add_argument("--block-size", type=int, default=0, help="page the caches into scattered blocks of this many rows")
-    ap.add_argument("--e2e-out", default="mapped", choices=["mapped", "copy"],
-                    help="end-to-end legs: the layers store their outputs straight into pinned host memory (mapped) or "
-                         "into HBM followed by one device-to-host copy (copy)")
+    ap.add_argument("--e2e-group", type=int, default=4, help="--e2e-out streamed: layers per device-to-host copy")
+    ap.add_argument("--e2e-out", default="auto", choices=["auto", "mapped", "copy", "streamed"],
+                    help="end-to-end legs, how the L outputs reach the host: the layers store them straight into pinned "
+                         "host memory (mapped), into HBM followed by one device-to-host copy (copy), or into HBM with each "
+                         "layer's output copied on a second stream while the next layers run (streamed; layers one by one "
+                         "only). auto: streamed for the layers-one-by-one mode, mapped for clsa_decode_step")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-breakdown", action="store_true", help="skip the per-kernel instrumented loop and the gather ceilings")
     ap.add_argument("--no-other-configs", action="store_true",
@@ -760,8 +763,9 @@ def run_ours(args):
     # ---- end to end: per-step inputs from pinned host memory, per-step results back to the host --------
     # One pinned staging buffer each way: [q_idx | Q^(0) .. Q^(L-1)] up, [O^(0) .. O^(L-1)] down. q_idx goes up first
     # on the launch stream; the L query tensors follow on a second stream while the routing runs, and the launch
-    # stream waits for them just before the first layer; the layers store their 128 KB outputs straight into the
-    # pinned host buffer (any address the device can reach serves as an output).
+    # stream waits for them just before the first layer. The outputs come back in one of three ways (--e2e-out): the
+    # layers store them straight into the pinned host buffer (any address the device can reach serves as an output),
+    # one copy behind the last layer, or one copy per layer on a second stream while the layers behind it run.
     n_qidx = pr.t["q_idx"].numel()
     n_q = pr.q_layers[0].numel()
     h_in = torch.empty(n_qidx + L * n_q, dtype=torch.bfloat16).pin_memory()
@@ -773,18 +777,29 @@ def run_ours(args):
     d_q = [d_in[n_qidx + l * n_q: n_qidx + (l + 1) * n_q].view(pr.q_layers[l].shape) for l in range(L)]
     d_out = torch.empty((L,) + tuple(pr.outs[0].shape), dtype=torch.bfloat16, device=dev)
     h_out = torch.empty(d_out.shape, dtype=torch.bfloat16).pin_memory()
-    mapped_out = decode and args.e2e_out == "mapped"
-    e2e_outs = [(h_out if mapped_out else d_out)[l] for l in range(L)]
+    out_mode = {True: args.e2e_out, False: args.e2e_out}   # keyed by "layers one by one"
+    if args.e2e_out == "auto":
+        out_mode = {True: "streamed", False: "mapped"}
+    if out_mode[False] == "streamed":
+        out_mode[False] = "copy"
+    if not decode:
+        out_mode = {True: "copy", False: "copy"}
     copy_stream = torch.cuda.Stream(device=dev)
+    out_stream = torch.cuda.Stream(device=dev)
     q_ready = torch.cuda.Event()
     step_start = torch.cuda.Event()
+    layer_done = [torch.cuda.Event() for _ in range(L)]
+    outs_home = torch.cuda.Event()
+    kGroup = args.e2e_group
 
     def e2e_step(one_by_one):
         if not decode:  # a prefill chunk: one upload, the three calls, one download
             d_in.copy_(h_in, non_blocking=True)
-            pr.independent_step(d_qidx, d_q, e2e_outs)
+            pr.independent_step(d_qidx, d_q, [d_out[l] for l in range(L)])
             h_out.copy_(d_out, non_blocking=True)
             return
+        mode = out_mode[one_by_one]
+        targets = [(h_out if mode == "mapped" else d_out)[l] for l in range(L)]
         step_start.record(stream)
         d_in[:n_qidx].copy_(h_in[:n_qidx], non_blocking=True)
         with torch.cuda.stream(copy_stream):
@@ -793,11 +808,26 @@ def run_ours(args):
             q_ready.record(copy_stream)
         pr.routing(d_qidx)
         stream.wait_event(q_ready)
+        if one_by_one and mode == "streamed":
+            # a layer's output goes home on a second stream while the layers behind it run
+            # (in groups of kGroup layers: a copy per layer costs the host more than it saves the device)
+            for l in range(L):
+                clsa.clsa_sparse_attn_hinted(pr.p, d_q[l], pr.idx, pr.cnt, targets[l], None, pr.layer_hints(l), pr.ws)
+                if (l + 1) % kGroup == 0 or l == L - 1:
+                    first = l - l % kGroup
+                    layer_done[l].record(stream)
+                    with torch.cuda.stream(out_stream):
+                        out_stream.wait_event(layer_done[l])
+                        h_out[first:l + 1].copy_(d_out[first:l + 1], non_blocking=True)
+            with torch.cuda.stream(out_stream):
+                outs_home.record(out_stream)
+            stream.wait_event(outs_home)             # the step ends when the last output has reached the host
+            return
         if one_by_one:
-            pr.layers_one_by_one(d_q, e2e_outs)
+            pr.layers_one_by_one(d_q, targets)
         else:
-            clsa.clsa_sparse_attn_layers(pr.p, d_q, pr.idx, pr.cnt, e2e_outs, pr.ws)
-        if not mapped_out:
+            clsa.clsa_sparse_attn_layers(pr.p, d_q, pr.idx, pr.cnt, targets, pr.ws)
+        if mode != "mapped":
             h_out.copy_(d_out, non_blocking=True)
 
     sampler.resume()
@@ -931,7 +961,7 @@ def run_ours(args):
 
     other = None
     if solo and not args.no_other_configs and args.config == "headline128k" and not args.block_size:
-        del pr, d_in, d_q, d_qidx, d_out, e2e_outs
+        del pr, d_in, d_q, d_qidx, d_out
         torch.cuda.empty_cache()
         other = {}
         for name, graph in (("mid", False), ("ragged", False), ("tiny", False), ("tiny", True), ("prefill_chunk", False)):
@@ -955,7 +985,9 @@ def run_ours(args):
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_med,
                     "note": "the headline's mode with per-step inputs from pinned host memory (q_idx on the launch stream, the L "
                             "query tensors on a second stream while the routing runs) and all L outputs back ("
-                            + ("stored by the layers straight into pinned host memory" if mapped_out else "one copy") + "); the KV "
+                            + {"mapped": "stored by the layers straight into pinned host memory", "copy": "one copy behind the last layer",
+                               "streamed": f"the outputs of each {kGroup} layers copied on a second stream while the next layers run"}[out_mode[decode]]
+                            + "); the KV "
                             "and indexer-key caches are decoder state and stay resident"},
             "gpu_launches": K * (2 + L),
         }
