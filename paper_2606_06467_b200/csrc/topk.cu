@@ -178,7 +178,7 @@ __device__ __forceinline__ void radix_pass(Shared& sh, cg::cluster_group& cluste
 // `row`: the (sequence, query) row whose lengths apply and whose index is written; `score_row`: the row of `scores`
 // that holds its scores (the same, except for rows that another route handed back into a scratch matrix).
 template <bool CACHED>
-__device__ __forceinline__ void topk_row(const int row, const int64_t score_row, const float* __restrict__ scores, int64_t score_stride,
+__device__ __forceinline__ void topk_row(const int row, const int score_row, const float* __restrict__ scores, int64_t score_stride,
                                          const int32_t* __restrict__ seq_len, int q_per_seq, int causal, int top_k,
                                          int max_seq_len, int32_t* __restrict__ idx_out, int32_t* __restrict__ count_out,
                                          uint32_t* status, unsigned char* smem_raw) {
@@ -218,7 +218,7 @@ __device__ __forceinline__ void topk_row(const int row, const int64_t score_row,
     for (int i = tid; i < cnt; i += kThreads) out[lo + i] = lo + i;
     return;
   }
-  const float* src = scores + score_row * score_stride + lo;
+  const float* src = scores + (int64_t)score_row * score_stride + lo;
   auto key_at = [&](int i) -> uint32_t { return CACHED ? keys[i] : score_key(src[i]); };
 
   __syncthreads();
@@ -569,25 +569,15 @@ template <bool CACHED>
 __global__ void __launch_bounds__(kThreads, 1)
 topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const int32_t* __restrict__ seq_len,
                   int q_per_seq, int causal, int top_k, int max_seq_len, int pending_rows,
-                  const int32_t* __restrict__ row_of_slot, const uint32_t* __restrict__ nslots,
                   int32_t* __restrict__ idx_out, int32_t* __restrict__ count_out, uint32_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   // Programmatic dependent launch: this grid may have been scheduled before the kernel that writes the scores
   // has finished. The kernel after this one may be scheduled early in turn (it waits for this grid itself);
   // this grid's own wait sits in topk_row, after the shared-memory clears and before the first global access.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (row_of_slot != nullptr) {
-    // Rows that the fused chunk routing handed back: block j takes the row listed in slot j, whose scores are row j
-    // of the scratch matrix (no clusters; usually there is no such row and the block returns at once).
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (blockIdx.x >= *nslots) return;
-    topk_row<CACHED>(row_of_slot[blockIdx.x], (int64_t)blockIdx.x, scores, score_stride, seq_len, q_per_seq, causal, top_k,
-                     max_seq_len, idx_out, count_out, status, smem_raw);
-    return;
-  }
   if (pending_rows == 0) {
     const int nblk = (int)cg::this_cluster().num_blocks();
-    topk_row<CACHED>(blockIdx.x / nblk, (int64_t)(blockIdx.x / nblk), scores, score_stride, seq_len, q_per_seq, causal, top_k, max_seq_len, idx_out,
+    topk_row<CACHED>(blockIdx.x / nblk, blockIdx.x / nblk, scores, score_stride, seq_len, q_per_seq, causal, top_k, max_seq_len, idx_out,
                      count_out, status, smem_raw);
     return;
   }
@@ -606,11 +596,28 @@ topk_radix_kernel(const float* __restrict__ scores, int64_t score_stride, const 
   if (__syncthreads_or(mine) == 0) return;
   for (int j = 0; j < kPendingRowsPerBlock; ++j) {
     if (pending[j]) {
-      topk_row<CACHED>(first + j, (int64_t)(first + j), scores, score_stride, seq_len, q_per_seq, causal, top_k, max_seq_len, idx_out,
+      topk_row<CACHED>(first + j, first + j, scores, score_stride, seq_len, q_per_seq, causal, top_k, max_seq_len, idx_out,
                        count_out, status, smem_raw);
       __syncthreads();  // the next row reuses this block's shared memory
     }
   }
+}
+
+// Rows that the fused chunk routing handed back: block j takes the row listed in slot j, whose scores are row j of the
+// scratch matrix (no clusters; usually there is no such row and the block returns at once). A kernel of its own, so
+// that the decode kernel above is compiled exactly as it is without this route.
+template <bool CACHED>
+__global__ void __launch_bounds__(kThreads, 1)
+topk_radix_slots_kernel(const float* __restrict__ scores, int64_t score_stride, const int32_t* __restrict__ seq_len,
+                        int q_per_seq, int causal, int top_k, int max_seq_len,
+                        const int32_t* __restrict__ row_of_slot, const uint32_t* __restrict__ nslots,
+                        int32_t* __restrict__ idx_out, int32_t* __restrict__ count_out, uint32_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (blockIdx.x >= *nslots) return;
+  topk_row<CACHED>(row_of_slot[blockIdx.x], (int)blockIdx.x, scores, score_stride, seq_len, q_per_seq, causal, top_k,
+                   max_seq_len, idx_out, count_out, status, smem_raw);
 }
 
 }  // namespace
@@ -733,8 +740,7 @@ cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, scores, score_stride, p.seq_len, (int)p.q_per_seq, (int)p.causal,
-                            (int)p.top_k, (int)p.max_seq_len, pending_rows, (const int32_t*)nullptr, (const uint32_t*)nullptr,
-                            idx, count, status);
+                            (int)p.top_k, (int)p.max_seq_len, pending_rows, idx, count, status);
 }
 
 cudaError_t launch_topk_slots(const clsa_params& p, const float* scores, int64_t score_stride, const int32_t* row_of_slot,
@@ -744,7 +750,7 @@ cudaError_t launch_topk_slots(const clsa_params& p, const float* scores, int64_t
   plan.cluster = 1;
   plan.one_sweep = 0;
   size_blocks(plan, p.max_seq_len, dev);
-  auto kernel = plan.slice_cap > 0 ? topk_radix_kernel<true> : topk_radix_kernel<false>;
+  auto kernel = plan.slice_cap > 0 ? topk_radix_slots_kernel<true> : topk_radix_slots_kernel<false>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   cudaLaunchConfig_t cfg = {};
@@ -753,7 +759,7 @@ cudaError_t launch_topk_slots(const clsa_params& p, const float* scores, int64_t
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
   return cudaLaunchKernelEx(&cfg, kernel, scores, score_stride, p.seq_len, (int)p.q_per_seq, (int)p.causal, (int)p.top_k,
-                            (int)p.max_seq_len, 0, row_of_slot, nslots, idx, count, status);
+                            (int)p.max_seq_len, row_of_slot, nslots, idx, count, status);
 }
 
 }  // namespace clsa
