@@ -888,10 +888,13 @@ def run_ours(args):
             "achieved": rate(steady_us), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": rate(steady_us) / peak,
             "algorithmic_bytes_per_launch": gathered,
             "steady_layer": {"us": steady_us, "GBps": rate(steady_us), "frac_of_hbm_peak": rate(steady_us) / peak},
-            "cold_first_layer": {"us": cold_us, "GBps": rate(cold_us), "frac_of_hbm_peak": rate(cold_us) / peak},
+            "cold_first_layer": {"us": cold_us, "GBps": rate(cold_us), "frac_of_hbm_peak": rate(cold_us) / peak,
+                                 "traffic": profiled_traffic(c.name, "sparse_attn_kernel_cold")},
             "traffic": profiled_traffic(c.name, "sparse_attn_kernel"),
-            "traffic_note": "DRAM bytes of one launch on its own, from an ncu capture of the mid workload scaled to this "
-                            "workload by the units per launch; not measured in this run",
+            "traffic_note": "DRAM bytes read by one steady layer (cold_first_layer.traffic: by the first layer), from a "
+                            "one-pass ncu capture of this workload with the cache state carried from launch to launch "
+                            "(profiles/launch_list_headline128k.md; for other workloads one launch behind an L2 flush); "
+                            "recorded in profiles/traffic.txt, not measured in this run",
             "note": "achieved/frac: algorithmic (gathered) bytes of one layer over the steady layer's time (layers 2..L of the "
                     "dependent step, event-timed as a group). A steady layer finds part of its rows in L2, where its "
                     "predecessor left them, so this is a rate of algorithmic bytes and HBM traffic stays below it; the cold "
@@ -906,7 +909,7 @@ def run_ours(args):
             {"kernel": "index_scores_decode_kernel (one event-timed call)", "bound": "hbm",
              "algorithmic_bytes_per_launch": pr.key_bytes, "us": bd["index_scores"], "achieved": key_gbs, "frac": key_gbs / peak,
              "traffic": profiled_traffic(c.name, "index_scores_decode_kernel"),
-             "traffic_note": "scaled from an ncu capture of the mid workload; not measured in this run"},
+             "traffic_note": "scaled from an ncu capture of the mid workload by the keys streamed; not measured in this run"},
             {"kernel": "topk_radix_kernel", "bound": "latency", "us": bd["topk"],
              "note": "cluster barriers and dependent sweeps, not bytes"}]
 
