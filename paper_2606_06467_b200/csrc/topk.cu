@@ -301,6 +301,43 @@ __device__ __forceinline__ void topk_row(const int row, const int score_row, con
     // ---- short path: sweep 2 counts keys above the bin per warp and collects the bin's keys ----------
     uint2* cand = reinterpret_cast<uint2*>(sh.cluster_hist[1]);  // (key, slice position), unordered
     uint32_t gt = 0;
+    if (CACHED && use_bitmap) {
+      // One thread per bitmap word: it reads its 32 consecutive keys as eight 16-byte chunks (in an order rotated by
+      // its lane, so that the eight lanes of a quarter warp hit eight different bank groups), builds the word with
+      // bit operations instead of one ballot per 32 keys, and then appends the few keys of the threshold's bin.
+      const int words = (cnt + 31) >> 5;
+      for (int w = tid; w < words; w += kThreads) {
+        uint32_t above = 0, inbin = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int c = (j + lane) & 7;
+          const int i = 32 * w + 4 * c;
+          if (i < cnt) {  // the slice buffer is padded to a multiple of 4 keys
+            const uint4 k4 = *reinterpret_cast<const uint4*>(keys + i);
+            const uint32_t t0 = k4.x >> 20, t1 = k4.y >> 20, t2 = k4.z >> 20, t3 = k4.w >> 20;
+            const uint32_t a4 = (t0 > digit0 ? 1u : 0u) | (t1 > digit0 ? 2u : 0u) | (t2 > digit0 ? 4u : 0u) | (t3 > digit0 ? 8u : 0u);
+            const uint32_t e4 = (t0 == digit0 ? 1u : 0u) | (t1 == digit0 ? 2u : 0u) | (t2 == digit0 ? 4u : 0u) | (t3 == digit0 ? 8u : 0u);
+            above |= a4 << (4 * c);
+            inbin |= e4 << (4 * c);
+          }
+        }
+        const int left = cnt - 32 * w;  // >= 1
+        if (left < 32) {
+          const uint32_t valid = (1u << left) - 1u;
+          above &= valid;
+          inbin &= valid;
+        }
+        bitmap[w] = above;
+        gt += (uint32_t)__popc(above);
+        while (inbin != 0u) {
+          const int i = 32 * w + __ffs(inbin) - 1;
+          inbin &= inbin - 1u;
+          cand[atomicAdd(&sh.cand_count, 1u)] = make_uint2(keys[i], (uint32_t)i);
+        }
+      }
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) gt += __shfl_xor_sync(0xffffffffu, gt, d);
+    } else
     for (int i0 = c_lo; i0 < c_hi; i0 += 128) {
       uint32_t key[4];
 #pragma unroll
