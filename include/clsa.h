@@ -113,10 +113,8 @@ typedef struct {
 
 /* Bytes of workspace that any of the calls below may need for these params (the maximum over them:
  * the status header, the scratch through which a standalone decode clsa_sparse_attn merges the
- * partial results of its blocks -- arrival counters and partial slots --, the fp32 score matrix
- * that clsa_decode_step keeps there and, for paged caches (block_size > 0 or a block table), the index
- * of a step translated to cache rows once for all of its layers). Reads only the scalar fields and
- * whether block_table is set. *bytes is HOST memory. The workspace must be 256-byte aligned
+ * partial results of its blocks -- arrival counters and partial slots -- and the fp32 score matrix
+ * that clsa_decode_step keeps there). Reads only the scalar fields. *bytes is HOST memory. The workspace must be 256-byte aligned
  * and ALL of it zero before the first call (cudaMemset): its first 256 bytes hold the device status
  * word and the score kernel's scheduling counters, the attention scratch begins with arrival counters;
  * every launch leaves all of these counters at zero again, and clsa_clear_status zeroes the status word.

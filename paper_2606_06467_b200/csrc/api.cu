@@ -49,9 +49,7 @@ WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& de
   w.scores_bytes = align((size_t)p.num_seqs * p.q_per_seq * w.score_stride * sizeof(float));
   // a prefill chunk's fused routing (clsa_index_topk) uses the same bytes for its own scratch instead
   const size_t fused = p.q_per_seq > 1 ? index_topk_scratch_bytes(p) : 0;
-  w.rows_off = w.scores_off + (w.scores_bytes > fused ? w.scores_bytes : fused);
-  w.rows_bytes = (p.block_table != nullptr || p.block_size > 0) ? align((size_t)p.num_seqs * p.q_per_seq * p.top_k * sizeof(int32_t)) : 0;
-  w.total = w.rows_off + w.rows_bytes;
+  w.total = w.scores_off + (w.scores_bytes > fused ? w.scores_bytes : fused);
   return w;
 }
 
@@ -154,8 +152,7 @@ clsa_status check_hints(const clsa_attn_hints* h) {
 // whole (row, KV head) units to blocks.
 cudaError_t launch_attention(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                              float* lse, uint32_t* status, unsigned char* ws_base, const WorkspaceLayout& w,
-                             const clsa_attn_hints& h, int wait_prior, int fine_rows, const int32_t* cache_rows,
-                             const DeviceInfo& dev, cudaStream_t s) {
+                             const clsa_attn_hints& h, int wait_prior, int fine_rows, const DeviceInfo& dev, cudaStream_t s) {
   // With the GPU to itself, a decode launch whose (row, KV head) units would leave many SMs idle in the last round of
   // whole-unit blocks (20 rows x 8 heads: 160 units on 148 SMs) cuts its work at token granularity instead.
   if (p.q_per_seq == 1 && h.shared_gpu == 0 && attn_alone_occupancy(p, dev) < kTokenGranularBelow) {
@@ -166,7 +163,7 @@ cudaError_t launch_attention(const clsa_params& p, const void* q, const int32_t*
                                  h.only_q_pending, h.keep_rows, dev, s);
   }
   return launch_sparse_attn(p, q, idx, count, out, lse, status, h.reverse, wait_prior, h.only_q_pending, h.keep_rows,
-                            h.shared_gpu, fine_rows, cache_rows, dev, s);
+                            h.shared_gpu, fine_rows, dev, s);
 }
 
 // The L attention launches that share one index. Layer 0 follows whatever produced the index and must wait for it;
@@ -179,20 +176,12 @@ cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, voi
                           cudaStream_t s) {
   const WorkspaceLayout w = make_workspace_layout(p, dev);
   const ChainTail tail = chain_fine_tail(p, dev);
-  // Paged caches: every layer would look the same positions up in the block table; they are translated to cache rows
-  // once, into the workspace, and the layers read those (the same kernels as for contiguous caches).
-  int32_t* cache_rows = nullptr;
-  if (p.block_table != nullptr) {
-    cache_rows = reinterpret_cast<int32_t*>(ws_base + w.rows_off);
-    const cudaError_t err = launch_translate_index(p, idx, count, cache_rows, s);
-    if (err != cudaSuccess) return err;
-  }
   for (int l = 0; l < p.num_layers; ++l) {
     const bool fine = l >= p.num_layers - tail.layers;
     const int fine_rows = l == p.num_layers - tail.layers - 1 ? tail.rows : 0;  // the layer where the finer shape begins
     const clsa_attn_hints h = {0, fine ? 2 : 1, l + 1 < p.num_layers ? 1 : 0, 0};
     const cudaError_t err = launch_attention(p, q_layers[l], idx, count, out_layers[l], nullptr, status, ws_base, w, h,
-                                             l == 0 ? 1 : 0, fine_rows, cache_rows, dev, s);
+                                             l == 0 ? 1 : 0, fine_rows, dev, s);
     if (err != cudaSuccess) return err;
   }
   return cudaSuccess;
@@ -297,7 +286,7 @@ clsa_status clsa_sparse_attn_hinted(const clsa_params* p, const void* q, const i
   // a decode launch with the GPU to itself merges its split partials through the scratch behind the header
   CLSA_TRY(check_workspace(workspace, workspace_bytes, p->q_per_seq == 1 && h.shared_gpu == 0 ? w.scores_off : kStatusBytes));
   auto base = static_cast<unsigned char*>(workspace);
-  return from_cuda(launch_attention(*p, q, idx, count, out, lse, reinterpret_cast<uint32_t*>(base), base, w, h, 1, 0, nullptr, dev,
+  return from_cuda(launch_attention(*p, q, idx, count, out, lse, reinterpret_cast<uint32_t*>(base), base, w, h, 1, 0, dev,
                                     static_cast<cudaStream_t>(stream)));
 }
 

@@ -81,8 +81,6 @@ struct WorkspaceLayout {
   size_t attn_part_off;             // start of the partial slots
   size_t scores_off, scores_bytes;  // fp32 score matrix of clsa_decode_step
   int64_t score_stride;
-  // Paged caches only: the index of a step translated to physical cache rows once, for all of its layers.
-  size_t rows_off, rows_bytes;
   size_t total;
 };
 WorkspaceLayout make_workspace_layout(const clsa_params& p, const DeviceInfo& dev);
@@ -108,6 +106,7 @@ struct GemmFused {
 };
 cudaError_t launch_index_gemm_sample(const clsa_params& p, const void* q_idx, float* sample, int64_t sample_stride,
                                      int sample_gs, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+int index_gemm_filter_hole_slack(const clsa_params& p, const DeviceInfo& dev);
 cudaError_t launch_index_gemm_filter(const clsa_params& p, const void* q_idx, const GemmFused& fx, uint32_t* status,
                                      const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_index_gemm_handed_back(const clsa_params& p, const void* q_idx, float* scratch, int64_t score_stride,
@@ -134,16 +133,10 @@ cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score
 bool topk_prefilter_fits(const clsa_params& p, const float* scores, int64_t score_stride, const DeviceInfo& dev);
 cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx,
                                   int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
-// cache_rows: nullptr, or (paged caches) the index already translated to physical cache rows by
-// launch_translate_index; the launch then reads those instead of idx and does not touch the block table.
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
-                               int keep_for_next, int throughput_plan, int fine_rows, const int32_t* cache_rows,
-                               const DeviceInfo& dev, cudaStream_t stream);
-// Paged caches: cache_rows[r][j] = physical cache row of position idx[r][j] through the block table, -1 for entries that
-// are past the row's count, out of the sequence's range, or of a sequence whose length is out of bounds.
-cudaError_t launch_translate_index(const clsa_params& p, const int32_t* idx, const int32_t* count, int32_t* cache_rows,
-                                   cudaStream_t stream);
+                               int keep_for_next, int throughput_plan, int fine_rows, const DeviceInfo& dev,
+                               cudaStream_t stream);
 // Share of its rounds of one-block-per-SM that the whole-unit kernel's launch-on-its-own shape fills (0..1).
 double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev);
 

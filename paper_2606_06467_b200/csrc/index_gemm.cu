@@ -21,7 +21,8 @@
 //                      columns at a time (double-buffered) into a swizzled shared-memory tile; chunks that
 //                      every query of the warp may see leave as one tiled bulk store, the others (causal
 //                      diagonal, end of a sequence) as masked 32-byte stores, four lanes per row. The
-//                      epilogue of tile i overlaps the MMAs of tile i+1.
+//                      epilogue of tile i overlaps the MMAs of tile i+1. The filtering mode of clsa_index_topk
+//                      runs warps 4..19 instead: four per 32 TMEM lanes, 64 columns each, 16 at a time.
 // Tiles that lie entirely above the causal diagonal are skipped by every role alike.
 // Every mbarrier wait is bounded: on expiry the block raises CLSA_DEV_TIMEOUT in the status word,
 // all roles leave their loops, in-flight copies are given time to land, TMEM is freed, and the
@@ -35,15 +36,19 @@ namespace {
 
 constexpr int kBM = 128, kBN = 256, kBK = 64;  // tile; kBK bf16 = one 128-byte swizzle row
 constexpr int kStages = 2, kAccBufs = 2;
-constexpr int kEpiWarps = 8;                     // two per TMEM lane quadrant, 128 columns each
-constexpr int kThreads = (4 + kEpiWarps) * 32;
+// Epilogue warps: two per TMEM lane quadrant with 128 columns each where the scores are stored; four per quadrant with
+// 64 columns each in the filtering mode, whose epilogue is a chain of dependent instructions per warp (twice the warps
+// hide twice the latency; its 16-column register buffers keep 640 threads within the register file).
+__host__ __device__ constexpr int epi_warps(int mode) { return mode == 1 ? 16 : 8; }
+__host__ __device__ constexpr int gemm_threads(int mode) { return (4 + epi_warps(mode)) * 32; }
 constexpr int kABytes = kBM * kBK * 2;          // one k-block of the query tile (16 KiB)
 constexpr int kBBytes = kBN * kBK * 2;          // one k-block of the key tile (32 KiB)
 constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;  // up to two k-blocks each (96 KiB)
 constexpr int kBarrierBytes = 128;
-constexpr int kEpiTileBytes = kEpiWarps * 4096;  // one 32 x 32 fp32 tile (128-byte rows, 128-byte swizzle) per epilogue warp
+constexpr int kEpiTileBytes = 8 * 4096;          // a 32 x 32 fp32 tile per storing warp (128-byte rows, 128-byte swizzle) or a 32 x 16 one per filtering warp
 constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + kBarrierBytes + kEpiTileBytes + 1024;  // + alignment slack
 constexpr uint32_t kSpinLimit = 1u << 22;       // polls with back-off: a few seconds at most
+constexpr uint32_t kFilterRun = 8;              // slots of a candidate list that a lane reserves at a time
 
 struct GemmArgs {
   const int64_t* seq_start;
@@ -124,6 +129,15 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uin
       "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -185,7 +199,7 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmArgs& a, int64_t id) {
 // MODE 1: the scores are compared with a per-row pivot in registers and only candidates leave the SM (clsa_index_topk).
 // MODE 2: MODE 0 for the few rows that clsa_index_topk hands back, into a small scratch matrix.
 template <int MODE>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(gemm_threads(MODE), 1)
 index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_s, const GemmArgs a) {
   extern __shared__ unsigned char smem_dyn[];
@@ -201,6 +215,8 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kEpiTileBytes + 68);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int kEpi = epi_warps(MODE);
+  constexpr int kColsPerWarp = kBN / (kEpi / 4);  // columns of a tile that one epilogue warp drains
   const int kblocks = a.idx_dim / kBK;  // 1 or 2
   const bool causal = a.causal != 0 && a.sample_gs == 0;
   const int64_t total_tiles = (int64_t)a.num_seqs * a.m_blocks * a.n_tiles;
@@ -213,7 +229,7 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int i = 0; i < kAccBufs; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), kEpiWarps); }
+    for (int i = 0; i < kAccBufs; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), kEpi); }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -309,7 +325,7 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
   } else if (warp >= 4) {
     // ---------------- epilogue: TMEM -> registers -> global ----------------
     const int quad = warp & 3;          // TMEM lanes 32*quad .. 32*quad+31 (a warp may only touch its own quadrant)
-    const int half = (warp - 4) >> 2;   // which 128 of the tile's 256 columns
+    const int part = (warp - 4) >> 2;   // which kColsPerWarp of the tile's 256 columns
     // MODE 1: a lane appends its row's candidates straight to the row's list in global memory, into runs of kRun slots
     // that it reserves with one atomic add each. A warp's scoreboard tracks a register for all lanes at once, so an
     // atomic whose result any lane still waits for would stall every lane that touches the same register: the runs
@@ -320,7 +336,7 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // to other queries, what is left of the runs is filled with holes (position = kHole), which the select skips.
     // Entries past the list's capacity are dropped; the count keeps growing, which is how the select learns that the
     // row overflowed.
-    constexpr uint32_t kRun = 16, kHole = 0xffffffffu;
+    constexpr uint32_t kRun = kFilterRun, kHole = 0xffffffffu;
     int64_t f_row = -1;
     float f_pivot = 0.f;
     uint32_t f_base = 0, f_used = kRun, f_spare = 0, f_pending = 0;
@@ -355,8 +371,8 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kBN);
       // columns this warp has to drain: up to the last one any of its 32 queries can see (a multiple of 32)
       const int v_warp = __reduce_max_sync(0xffffffffu, v) - c.nt * kBN;
-      const int c_begin = half * (kBN / 2);
-      const int c_end = min(c_begin + kBN / 2, (max(v_warp, 0) + 31) & ~31);
+      const int c_begin = part * kColsPerWarp;
+      const int c_end = min(c_begin + kColsPerWarp, (max(v_warp, 0) + 31) & ~31);
       if (MODE == 1) {
         // ---- filter: compare with the row's pivot in registers; only candidates leave the SM ----
         const int64_t row = (int64_t)c.b * a.q_per_seq + t;
@@ -372,38 +388,47 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
         if (f_list != nullptr) {      // tile start: last tile's request becomes the spare run, and a new one goes out
           if (f_has_pending && !f_has_spare) { f_spare = f_pending; f_has_spare = true; f_has_pending = false; }
-          if (!f_has_pending) { f_pending = reserve_run(); f_has_pending = true; }
+          // ... unless this is the block's last tile on these queries: a run requested now would only become holes
+          bool more = false;
+          if (id + tile_step < tile_last) {
+            const TileCoord nx = tile_coord<MODE>(a, id + tile_step);
+            more = nx.valid && nx.b == c.b && nx.mb == c.mb;
+          }
+          // ... nor while the current run is less than half used and a spare is at hand
+          const bool soon = f_used * 2 >= kRun || !f_has_spare;
+          if (!f_has_pending && more && soon) { f_pending = reserve_run(); f_has_pending = true; }
         }
-        uint32_t ra[32], rb[32];
-        // The warp's staging tile (32 rows x 128 bytes, 16-byte chunk c of row r at r * 128 + ((c ^ (r & 7)) << 4), free
-        // of bank conflicts for a row per lane) holds the chunk so that a lane can fetch the few columns that pass by
-        // index: a lane's pass mask costs one compare per column, and only its own set bits cost anything more.
-        unsigned char* tile = base_ptr + kStages * kStageBytes + (warp - 4) * 4096;
-        auto filter32 = [&](const uint32_t (&r)[32], int s0) {
+        uint32_t ra[16], rb[16];
+        // The warp's staging tile (32 rows x 64 bytes, 16-byte chunk c of row r at r * 64 + ((c ^ ((r >> 1) & 3)) << 4),
+        // free of bank conflicts for a row per lane) holds the chunk so that a lane can fetch the few columns that pass
+        // by index: a lane's pass mask costs one compare per column, and only its own set bits cost anything more.
+        unsigned char* tile = base_ptr + kStages * kStageBytes + (warp - 4) * 2048;
+        const int swz = (lane >> 1) & 3;
+        auto filter16 = [&](const uint32_t (&r)[16], int s0) {
           // Two instructions per column: the sign of (score - pivot) is shifted into a mask by a funnel shift. Four
-          // chains of 8 columns, highest column first, so that column i ends up at bit i. The difference of a NaN is the
+          // chains of 4 columns, highest column first, so that column i ends up at bit i. The difference of a NaN is the
           // canonical (positive) NaN: it passes, like everything that is not below the pivot.
           uint32_t sg[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-          for (int j = 7; j >= 0; --j) {
+          for (int j = 3; j >= 0; --j) {
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4)
-              sg[q4] = __funnelshift_l(__float_as_uint(__uint_as_float(r[q4 * 8 + j]) - f_pivot), sg[q4], 1);
+              sg[q4] = __funnelshift_l(__float_as_uint(__uint_as_float(r[q4 * 4 + j]) - f_pivot), sg[q4], 1);
           }
-          uint32_t mask = ~((sg[0] & 0xffu) | ((sg[1] & 0xffu) << 8) | ((sg[2] & 0xffu) << 16) | (sg[3] << 24));
-          if (s0 + 32 > v) mask &= s0 >= v ? 0u : (0xffffffffu >> (32 - (v - s0)));
+          uint32_t mask = ~((sg[0] & 0xfu) | ((sg[1] & 0xfu) << 4) | ((sg[2] & 0xfu) << 8) | ((sg[3] & 0xfu) << 12)) & 0xffffu;
+          if (s0 + 16 > v) mask &= s0 >= v ? 0u : (0xffffu >> (16 - (v - s0)));
           if (f_list == nullptr) mask = 0u;
           if (__any_sync(0xffffffffu, mask != 0u) == 0) return;
           __syncwarp();  // the previous chunk's reads of the tile are done
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch)
-            *reinterpret_cast<uint4*>(tile + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
+          for (int ch = 0; ch < 4; ++ch)
+            *reinterpret_cast<uint4*>(tile + lane * 64 + ((ch ^ swz) << 4)) =
                 make_uint4(r[4 * ch], r[4 * ch + 1], r[4 * ch + 2], r[4 * ch + 3]);
           // a lane reads back only what it wrote: no barrier needed in between
           while (mask != 0u) {
             const int i = __ffs(mask) - 1;
             mask &= mask - 1u;
-            const uint32_t bits = *reinterpret_cast<const uint32_t*>(tile + lane * 128 + (((i >> 2) ^ (lane & 7)) << 4) + (i & 3) * 4);
+            const uint32_t bits = *reinterpret_cast<const uint32_t*>(tile + lane * 64 + (((i >> 2) ^ swz) << 4) + (i & 3) * 4);
             if (f_used == kRun) {  // the current run is full: take the spare, or (rarely) reserve on the spot
               if (f_has_spare) { f_base = f_spare; f_has_spare = false; }
               else f_base = reserve_run();
@@ -413,17 +438,15 @@ index_scores_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             ++f_used;
           }
         };
-        if (c_end > c_begin) tc_ld32(taddr + (uint32_t)c_begin, ra);
+        if (c_end > c_begin) tc_ld16(taddr + (uint32_t)c_begin, ra);
 #pragma unroll 1
-        for (int c0 = c_begin; c0 < c_end; c0 += 64) {
+        for (int c0 = c_begin; c0 < c_end; c0 += 32) {
           tc_ld_wait();
-          if (c0 + 32 < c_end) tc_ld32(taddr + (uint32_t)(c0 + 32), rb);
-          filter32(ra, c.nt * kBN + c0);
-          if (c0 + 32 < c_end) {
-            tc_ld_wait();
-            if (c0 + 64 < c_end) tc_ld32(taddr + (uint32_t)(c0 + 64), ra);
-            filter32(rb, c.nt * kBN + c0 + 32);
-          }
+          tc_ld16(taddr + (uint32_t)(c0 + 16), rb);   // c_end - c_begin is a multiple of 32
+          filter16(ra, c.nt * kBN + c0);
+          tc_ld_wait();
+          if (c0 + 32 < c_end) tc_ld16(taddr + (uint32_t)(c0 + 32), ra);
+          filter16(rb, c.nt * kBN + c0 + 16);
         }
       } else if (MODE == 2) {
         // ---- rows handed back: a lane stores its own row (if it has a slot) as it comes from TMEM ----
@@ -639,11 +662,24 @@ cudaError_t launch_gemm(int mode, const clsa_params& p, const void* q_idx, float
   auto kernel = mode == 0 ? index_scores_gemm_kernel<0> : mode == 1 ? index_scores_gemm_kernel<1> : index_scores_gemm_kernel<2>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (err != cudaSuccess) return err;
-  kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_s, a);
+  kernel<<<grid, gemm_threads(mode), kSmemBytes, stream>>>(map_q, map_k, map_s, a);
   return cudaGetLastError();
 }
 
 }  // namespace
+
+// Slots of a row's candidate list that the filtering launch may leave as holes, at most: every lane that appends to
+// the row (four per block: one per 64-column part of a tile) can end its stay on the row with a part-filled run and an
+// unused spare, and the row's key tiles are spread over the blocks that the tile order gives it.
+int index_gemm_filter_hole_slack(const clsa_params& p, const DeviceInfo& dev) {
+  const int64_t m_blocks = (p.q_per_seq + kBM - 1) / kBM, n_tiles = (p.max_seq_len + kBN - 1) / kBN;
+  const int64_t tiles = (int64_t)p.num_seqs * m_blocks * n_tiles;
+  const int64_t grid = tiles < dev.sm_count ? tiles : dev.sm_count;
+  const int64_t per_block = grid > 0 ? (tiles + grid - 1) / grid : 1;
+  int64_t blocks_per_row = n_tiles / per_block + 2;
+  if (blocks_per_row > n_tiles) blocks_per_row = n_tiles;
+  return (int)((epi_warps(1) / 4) * blocks_per_row * 2 * kFilterRun);
+}
 
 cudaError_t launch_index_scores_gemm(const clsa_params& p, const void* q_idx, float* scores, int64_t score_stride,
                                      uint32_t* status, const DeviceInfo& dev, cudaStream_t stream) {

@@ -42,7 +42,8 @@ __device__ __forceinline__ float key_score(uint32_t key) {  // inverse of score_
 // Step 2. One warp per (sequence, query) row. Column j of the sample stands for position (j / 16) * gs + j % 16.
 __global__ void __launch_bounds__(128)
 chunk_pivot_kernel(const float* __restrict__ sample, int64_t sample_stride, int sample_gs, const int32_t* __restrict__ seq_len,
-                   int q_per_seq, int causal, int top_k, int max_seq_len, int cand_cap, int64_t rows, float* __restrict__ pivot) {
+                   int q_per_seq, int causal, int top_k, int max_seq_len, int whole_row_cap, int64_t rows,
+                   float* __restrict__ pivot) {
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -59,7 +60,7 @@ chunk_pivot_kernel(const float* __restrict__ sample, int64_t sample_stride, int 
     if (lane == 0) pivot[row] = kInf;
     return;
   }
-  if (v <= cand_cap) {      // the whole row fits the candidate list
+  if (v <= whole_row_cap) {  // the whole row fits the candidate list, holes included
     if (lane == 0) pivot[row] = -kInf;
     return;
   }
@@ -172,11 +173,13 @@ bool index_topk_fits(const clsa_params& p, const DeviceInfo& dev) {
   // The candidate list must hold what the pivot is expected to let through on the longest row, give or take 2.5
   // standard deviations (the pivot sits at rank r of about kSampleTarget samples: about n r / samples scores pass).
   const double n = (double)p.max_seq_len, k = (double)(p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len);
-  if (n <= (double)topk_candidates_capacity()) return true;
+  // what the filter may leave of a list as holes comes off its capacity
+  const double cap = (double)topk_candidates_capacity() - (double)index_gemm_filter_hole_slack(p, dev);
+  if (n <= cap) return true;
   const double samples = n < kSampleTarget ? n : (double)kSampleTarget;
   const double expect = samples * k / n * 1.10;
   const double r = expect + 3.5 * sqrt(expect) + 4.0;
-  return n * (r + 2.5 * sqrt(r)) / samples <= (double)topk_candidates_capacity();
+  return n * (r + 2.5 * sqrt(r)) / samples <= cap;
 }
 
 cudaError_t launch_index_topk(const clsa_params& p, const void* q_idx, int32_t* idx, int32_t* count, unsigned char* scratch,
@@ -203,7 +206,8 @@ cudaError_t launch_index_topk(const clsa_params& p, const void* q_idx, int32_t* 
   err = launch_index_gemm_sample(p, q_idx, sample, l.sample_stride, l.sample_gs, status, dev, stream);
   if (err != cudaSuccess) return err;
   chunk_pivot_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, stream>>>(sample, l.sample_stride, l.sample_gs, p.seq_len, p.q_per_seq,
-                                                                     p.causal, p.top_k, p.max_seq_len, l.cand_cap, rows, pivot);
+                                                                     p.causal, p.top_k, p.max_seq_len,
+                                                                     l.cand_cap - index_gemm_filter_hole_slack(p, dev), rows, pivot);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   // 3. filter, 4. select
   GemmFused fx = {pivot, cand, cand_count, l.cand_cap, slot_of_row, qflags, nslots};

@@ -52,7 +52,6 @@ struct AttnArgs {
   const int32_t* count;
   const int32_t* block_table;  // paged caches: [B][max_blocks] physical block numbers, or nullptr
   int block_shift, max_blocks;
-  int phys;                    // idx holds physical cache rows already (paged caches, translated once per step)
   uint16_t* out;
   float* lse;
   uint32_t* status;
@@ -152,15 +151,14 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
   int cnt = a.count[r];
   const int b = (int)(r / a.q_per_seq);
   constexpr bool paged = PAGED;
-  // paged: positions are translated to cache rows when they are fetched, or (a.phys) have been already
-  const int64_t s0 = (paged || a.phys) ? 0 : a.seq_start[b];
+  const int64_t s0 = paged ? 0 : a.seq_start[b];  // paged: positions are translated to cache rows when they are fetched
   const int32_t* table = paged ? a.block_table + (int64_t)b * a.max_blocks : nullptr;
   // A sequence whose length lies outside its declared bounds is never read: with n = 0 no position passes the range
   // check, every stage is masked, and the row comes out as zeros with lse = -inf. (A select, not a branch: the length
   // is first needed when the first copies are issued, and the flag is raised behind the main loop.)
   const int n_raw = a.seq_len[b];
   const bool n_ok = n_raw >= a.q_per_seq && n_raw <= a.max_seq_len;
-  const int n = n_ok ? (a.phys ? 0x7fffffff : n_raw) : 0;  // physical rows were range-checked when they were translated
+  const int n = n_ok ? n_raw : 0;
   // Positions are fetched two pipeline steps before they are used and (paged caches) their block numbers one
   // step before, so that no load is consumed in the step that issued it. The first three steps' positions are
   // fetched here, speculatively for a range that lies entirely below the row's count (entries past the count
@@ -726,6 +724,7 @@ ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
   const ChainTail none = {0, 0};
   const int L = p.num_layers;
   if (L < 2) return none;
+  if (p.block_table != nullptr) return none;  // paged caches: the finer blocks cost more than the fuller last round returns
   // The block model above was measured on a B200 (148 SMs); on anything else the chain keeps one block size.
   if (dev.sm_count != 148 || dev.clock_khz <= 0) return none;
   const AttnPlan base = make_attn_plan(p, dev, 1), fine = make_attn_plan(p, dev, 2);
@@ -769,10 +768,9 @@ double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev) {
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
-                               int keep_for_next, int throughput_plan, int fine_rows, const int32_t* cache_rows,
-                               const DeviceInfo& dev, cudaStream_t stream) {
+                               int keep_for_next, int throughput_plan, int fine_rows, const DeviceInfo& dev,
+                               cudaStream_t stream) {
   const AttnPlan plan = make_attn_plan(p, dev, throughput_plan);
-  const bool translated = cache_rows != nullptr && p.block_table != nullptr;
   AttnArgs a;
   a.q = static_cast<const uint16_t*>(q);
   a.kc = static_cast<const uint16_t*>(p.k_cache);
@@ -781,12 +779,11 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.head_stride = p.kv_head_stride;
   a.seq_start = p.seq_start;
   a.seq_len = p.seq_len;
-  a.idx = translated ? cache_rows : idx;
+  a.idx = idx;
   a.count = count;
-  a.block_table = translated ? nullptr : p.block_table;
-  a.phys = translated ? 1 : 0;
+  a.block_table = p.block_table;
   a.block_shift = 0;
-  while (a.block_table != nullptr && (1 << a.block_shift) < p.block_size) ++a.block_shift;
+  while (p.block_table != nullptr && (1 << a.block_shift) < p.block_size) ++a.block_shift;
   a.max_blocks = p.max_blocks_per_seq;
   a.out = static_cast<uint16_t*>(out);
   a.lse = lse;
@@ -818,7 +815,7 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   a.rows_max = p.num_cache_rows;
   a.off32 = (a.rows_max > 0 && (double)a.rows_max * (double)(p.kv_token_stride >> 3) < 4294967296.0) ? 1 : 0;
   void (*kernel)(const AttnArgs);
-  const bool multi = plan.rows_per_block > 1, pg = a.block_table != nullptr;
+  const bool multi = plan.rows_per_block > 1, pg = p.block_table != nullptr;
 #define CLSA_ATTN_PICK(NT_, W_)                                                                      \
   (multi ? (pg ? sparse_attn_kernel<NT_, true, W_, true> : sparse_attn_kernel<NT_, false, W_, true>) \
          : (pg ? sparse_attn_kernel<NT_, true, W_, false> : sparse_attn_kernel<NT_, false, W_, false>))
@@ -859,51 +856,6 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, a);
-}
-
-namespace {
-
-__global__ void __launch_bounds__(256) translate_index_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ count,
-                                                              const int32_t* __restrict__ seq_len,
-                                                              const int32_t* __restrict__ table, int max_blocks, int shift,
-                                                              int q_per_seq, int top_k, int max_seq_len, int64_t entries,
-                                                              int32_t* __restrict__ cache_rows) {
-  // The index may come from the kernel just before this one (the top-k of a step); the layers behind this one wait
-  // for it in turn, or start only once a layer that waited has released them.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= entries) return;
-  const int64_t r = i / top_k;
-  const int j = (int)(i - r * top_k);
-  const int b = (int)(r / q_per_seq);
-  const int n = seq_len[b];
-  const int cnt = count[r];
-  const int raw = idx[i];
-  const bool ok = n >= q_per_seq && n <= max_seq_len && j < cnt && raw >= 0 && raw < n;
-  int32_t row = -1;
-  if (ok) row = (table[(int64_t)b * max_blocks + (raw >> shift)] << shift) + (raw & ((1 << shift) - 1));
-  cache_rows[i] = row;
-}
-
-}  // namespace
-
-cudaError_t launch_translate_index(const clsa_params& p, const int32_t* idx, const int32_t* count, int32_t* cache_rows,
-                                   cudaStream_t stream) {
-  int shift = 0;
-  while ((1 << shift) < p.block_size) ++shift;
-  const int64_t entries = (int64_t)p.num_seqs * p.q_per_seq * p.top_k;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((entries + 255) / 256), 1, 1);
-  cfg.blockDim = dim3(256, 1, 1);
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, translate_index_kernel, idx, count, p.seq_len, p.block_table, (int)p.max_blocks_per_seq, shift,
-                            (int)p.q_per_seq, (int)p.top_k, (int)p.max_seq_len, entries, cache_rows);
 }
 
 }  // namespace clsa

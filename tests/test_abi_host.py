@@ -166,9 +166,8 @@ def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
     fwd = subprocess.check_output([sys.executable, "-c", code, "f"])
     rev = subprocess.check_output([sys.executable, "-c", code, "r"])
     assert fwd == rev and len(fwd) > 500
-    # paged caches get the contiguous plan (their index is translated to cache rows once per step, so the chain runs
-    # the same kernels); prefill chunks and single layers keep one shape
-    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16, block_table=0x5000, block_size=16, max_blocks_per_seq=8192), 148, 1965000) == plan(num_seqs=16)
+    # paged caches, prefill chunks and single layers keep one shape
+    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16, block_table=0x5000, block_size=16, max_blocks_per_seq=8192), 148, 1965000) == (0, 0)
     assert plan(num_seqs=16, q_per_seq=4) == (0, 0) and clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=1, num_seqs=16), 148, 1965000) == (0, 0)
     n = ctypes.c_int32(0)
     assert clsa.raw().clsa_chain_plan(ctypes.byref(_good(clsa)), 0, 1965000, ctypes.byref(n), ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG

@@ -53,11 +53,11 @@ def test_paged_decode_matches_oracle_and_contiguous_run(cfg, bs):
     check_attention(prob, w, 0, out0, lse0, idx_np, cnt_np)
 
 
-def test_layers_call_on_paged_caches_translates_the_index_once_and_never_follows_a_bad_entry():
-    """clsa_sparse_attn_layers on paged caches turns the index into cache rows once, in the workspace, for all layers.
-    A caller-built index with corrupt entries, a count out of range and a sequence whose length lies outside its
-    bounds must come out as in the contiguous case: bad entries skipped and flagged (no block-table lookup, no row
-    fetched), every other row equal to the contiguous run byte for byte, the caller's index untouched."""
+def test_layers_call_on_paged_caches_never_follows_a_bad_entry():
+    """clsa_sparse_attn_layers on paged caches with a caller-built index that has corrupt entries, a shorter count and
+    a sequence whose length lies outside its bounds must come out as in the contiguous case: bad entries skipped and
+    flagged (no block-table lookup, no row fetched), every other row equal to the contiguous run byte for byte, the
+    caller's index untouched."""
     import numpy as np
     w = Workload(MID.replace(num_seqs=4, ctx=5000, top_k=256, num_layers=3, seed=123))
     kc, vc = w.host_kv_full()
