@@ -159,7 +159,9 @@ CLSA_API clsa_status clsa_index_topk(const clsa_params* p, const void* q_idx, in
 
 /* Eq. 4 for ONE layer: for each (b,t) and query head h with KV head g = h / (Hq/Hkv),
  *   O = sum_{s in S} softmax_s(sm_scale * Q[b][t][h] . K[s][g]) V[s][g]   over the selected rows only.
- * No positional rotation is applied (the cross-decoder's global attention is NoPE).
+ * No positional rotation is applied (the cross-decoder's global attention is NoPE). p->sm_scale must be finite and
+ * greater than zero (CLSA_ERR_INVALID_ARG otherwise): a restriction of this library, not of Eq. 4 -- the kernels take
+ * running maxima over the raw dot products and apply the scale afterwards.
  *   q   bf16 [B][T][Hq][D]           this layer's queries, 16-byte aligned
  *   out bf16 [B][T][Hq][D]           round-to-nearest-even from fp32 accumulators
  *   lse fp32 [B][T][Hq] or NULL      log-sum-exp of the scaled logits (natural log)
