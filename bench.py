@@ -61,7 +61,7 @@ def parse():
                     help="also time the upstream step (Eq. 2 projections of the new tokens + cache append, "
                          "clsa_project_append) on the same workload; reported under \"projection\", not part of the step")
     ap.add_argument("--block-size", type=int, default=0, help="page the caches into scattered blocks of this many rows")
-    ap.add_argument("--e2e-group", type=int, default=4, help="--e2e-out streamed: layers per device-to-host copy")
+    ap.add_argument("--e2e-group", type=int, default=2, help="--e2e-out streamed: layers per device-to-host copy")
     ap.add_argument("--e2e-out", default="auto", choices=["auto", "mapped", "copy", "streamed"],
                     help="end-to-end legs, how the L outputs reach the host: the layers store them straight into pinned "
                          "host memory (mapped), into HBM followed by one device-to-host copy (copy), or into HBM with each "
@@ -800,10 +800,13 @@ def run_ours(args):
             return
         mode = out_mode[one_by_one]
         targets = [(h_out if mode == "mapped" else d_out)[l] for l in range(L)]
-        step_start.record(stream)
         d_in[:n_qidx].copy_(h_in[:n_qidx], non_blocking=True)
+        step_start.record(stream)
         with torch.cuda.stream(copy_stream):
-            copy_stream.wait_event(step_start)       # the upload belongs to this step: it may not start earlier
+            # The upload belongs to this step, and it goes behind q_idx's: released at the same moment, the two copies
+            # are taken in either order by the copy engine, and every other step the 4 KB that the first kernel waits
+            # for queued behind the 2 MB that nobody needs yet.
+            copy_stream.wait_event(step_start)
             d_in[n_qidx:].copy_(h_in[n_qidx:], non_blocking=True)
             q_ready.record(copy_stream)
         pr.routing(d_qidx)
