@@ -38,13 +38,15 @@ struct AttnPlan {
 };
 // throughput: 0 = a launch on its own (whole-GPU shape); 1 = a few large blocks (the launch shares the GPU with its
 // neighbours on the stream); 2 = the same with half the KV heads per block, where that is possible (twice the
-// blocks: used for the last layers of a chain, see chain_fine_tail)
+// blocks: used for the last layers of a chain, see chain_fine_tail); 3 = the shape of a launch that computes two layers
+// at once (8 warps with two head tiles each), also available to a single layer so that a pair's results can be reproduced
 AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int throughput);
 // Which part of an L-layer chain should use the finer shape (throughput = 2) so that the chain's blocks fill the SMs
 // evenly to the end: the last `layers` layers entirely, and the last `rows` query rows of the layer before them.
 struct ChainTail {
   int layers;
   int rows;
+  int paired;  // leading layers of the chain that are computed two per launch (even; 0 = none)
 };
 ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev);
 
@@ -133,10 +135,12 @@ cudaError_t launch_topk(const clsa_params& p, const float* scores, int64_t score
 bool topk_prefilter_fits(const clsa_params& p, const float* scores, int64_t score_stride, const DeviceInfo& dev);
 cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx,
                                   int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
+// q2 / out2: nullptr, or the queries and outputs of a second layer that the same launch computes over the same staged
+// rows (throughput_plan 3, decode, groups of up to 8 query heads).
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
-                               int keep_for_next, int throughput_plan, int fine_rows, const DeviceInfo& dev,
-                               cudaStream_t stream);
+                               int keep_for_next, int throughput_plan, int fine_rows, const void* q2, void* out2,
+                               const DeviceInfo& dev, cudaStream_t stream);
 // Share of its rounds of one-block-per-SM that the whole-unit kernel's launch-on-its-own shape fills (0..1).
 double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev);
 

@@ -43,6 +43,7 @@ constexpr int kMergeBatch = 8;
 
 struct AttnArgs {
   const uint16_t* q;
+  const uint16_t* q2;   // PAIR: the second layer's queries
   const uint16_t* kc;
   const uint16_t* vc;
   int64_t tok_stride, head_stride;
@@ -53,6 +54,7 @@ struct AttnArgs {
   const int32_t* block_table;  // paged caches: [B][max_blocks] physical block numbers, or nullptr
   int block_shift, max_blocks;
   uint16_t* out;
+  uint16_t* out2;       // PAIR: the second layer's outputs
   float* lse;
   uint32_t* status;
   int q_per_seq, num_q_heads, num_kv_heads, group, top_k;
@@ -78,8 +80,13 @@ struct AttnArgs {
 // over the block.
 // MIXED = the launch has two block sizes (AttnArgs::coarse_blocks); a variant of its own so that launches of one
 // size keep their block shape in kernel parameters, not registers.
-template <int NT, bool PAGED, int WARPS, bool MULTI, bool MIXED = false>
+// PAIR = two layers in one launch (NT == 2, groups of up to 8 query heads): head tile 0 holds the first layer's query
+// heads, tile 1 the second layer's, both over the same staged K/V rows -- the rows of a step are the same for every
+// layer, so a pair of layers whose queries are both at hand copies them from L2 once instead of twice. Per layer the
+// arithmetic is that of a single-layer launch of the same block shape, bit for bit.
+template <int NT, bool PAGED, int WARPS, bool MULTI, bool MIXED = false, bool PAIR = false>
 __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnArgs a) {
+  static_assert(!PAIR || (NT == 2 && !MULTI && !MIXED), "a pair of layers takes the two head tiles");
   extern __shared__ __align__(128) unsigned char smem[];
   cg::cluster_group cluster = cg::this_cluster();
   const int C = (int)cluster.num_blocks();
@@ -194,10 +201,10 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
     // Q^T fragments (B operand, 128 x 8 per head tile): head = rowq, two consecutive d per register.
     uint32_t qb[NT][8][2];
     auto load_q = [&]() {
-      const uint16_t* qbase = a.q + (r * a.num_q_heads + h0) * 128;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        const int head = nt * 8 + rowq;
+        const uint16_t* qbase = ((PAIR && nt == 1) ? a.q2 : a.q) + (r * a.num_q_heads + h0) * 128;
+        const int head = PAIR ? rowq : nt * 8 + rowq;
         const bool hv = head < G;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
@@ -418,16 +425,18 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
     __syncwarp();
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      const int headA = nt * 8 + hcol, headB = headA + 1;
+      // slot of a head in the warp's partial: the head itself, or (PAIR) layer * G + head of the layer
+      const int headA = PAIR ? nt * G + hcol : nt * 8 + hcol, headB = headA + 1;
+      const bool okA = PAIR ? hcol < G : headA < G, okB = PAIR ? hcol + 1 < G : headB < G;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int d = 16 * j + rowq;
-        if (headA < G) { mypart[headA * kPartialStride + d] = o[nt][j][0]; mypart[headA * kPartialStride + d + 8] = o[nt][j][2]; }
-        if (headB < G) { mypart[headB * kPartialStride + d] = o[nt][j][1]; mypart[headB * kPartialStride + d + 8] = o[nt][j][3]; }
+        if (okA) { mypart[headA * kPartialStride + d] = o[nt][j][0]; mypart[headA * kPartialStride + d + 8] = o[nt][j][2]; }
+        if (okB) { mypart[headB * kPartialStride + d] = o[nt][j][1]; mypart[headB * kPartialStride + d + 8] = o[nt][j][3]; }
       }
       if (rowq == 0) {
-        if (headA < G) *reinterpret_cast<float2*>(mypart + headA * kPartialStride + 128) = make_float2(mA[nt], lA[nt]);
-        if (headB < G) *reinterpret_cast<float2*>(mypart + headB * kPartialStride + 128) = make_float2(mB[nt], lB[nt]);
+        if (okA) *reinterpret_cast<float2*>(mypart + headA * kPartialStride + 128) = make_float2(mA[nt], lA[nt]);
+        if (okB) *reinterpret_cast<float2*>(mypart + headB * kPartialStride + 128) = make_float2(mB[nt], lB[nt]);
       }
     }
   }
@@ -435,15 +444,19 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
 
   // Output jobs (KV head of this block's group, query head of the group) dealt over the cluster's warps.
   const int heads_here = min(HC, a.num_kv_heads - (int)by * HC);
-  const int jobs_per_row = heads_here * G;
+  const int jobs_per_layer = heads_here * G;
+  const int jobs_per_row = jobs_per_layer * (PAIR ? 2 : 1);
   const int njobs = RB * jobs_per_row;
   const uint32_t smem_base = smem_u32(smem);
   for (int job = crank + C * warp; job < njobs; job += C * WARPS) {
     const int rl = MULTI ? job / jobs_per_row : 0;  // which of the block's rows
     const int64_t r_job = (int64_t)(bx / C) * RB + rl;
     if (MULTI && r_job >= a.num_rows) continue;
-    const int jrow = job - rl * jobs_per_row;
+    const int jrow_all = job - rl * jobs_per_row;
+    const int lyr = PAIR ? jrow_all / jobs_per_layer : 0;   // which layer of the pair
+    const int jrow = jrow_all - lyr * jobs_per_layer;
     const int jg = jrow / G, hh = jrow - jg * G;   // local KV head, query head within the group
+    const int hslot = PAIR ? lyr * G + hh : hh;    // the head's slot in a warp's partial
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f, M = -INFINITY;
     // Partial p = (block p / S, range p % S) of row rl was left by warp (rl * S + p % S) * HC + jg of block p / S. Lane p of each
@@ -454,7 +467,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
       float2 ml = make_float2(-INFINITY, 0.f);
       if (p < nsplit) {
         const int c2 = p / S, sub2 = p - c2 * S;
-        const uint32_t local = smem_base + (uint32_t)(((rl * S + sub2) * HC + jg) * kWarpRingBytes + hh * kPartialStride * 4);
+        const uint32_t local = smem_base + (uint32_t)(((rl * S + sub2) * HC + jg) * kWarpRingBytes + hslot * kPartialStride * 4);
         asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(src) : "r"(local), "r"(c2));
         asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(ml.x), "=f"(ml.y) : "r"(src + 512u) : "memory");
       }
@@ -498,7 +511,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnAr
     uint2 packed;
     packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
     packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
-    *reinterpret_cast<uint2*>(a.out + item * 128 + lane * 4) = packed;
+    *reinterpret_cast<uint2*>(((PAIR && lyr == 1) ? a.out2 : a.out) + item * 128 + lane * 4) = packed;
     if (a.lse != nullptr && lane == 0) a.lse[item] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
   }
   if (C > 1) cluster.sync();  // no block may exit while a neighbour can still read its shared memory
@@ -541,6 +554,7 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   // main loop is a dependent chain per warp, so warps per SM, not bytes in flight, set the pace once the rows come
   // from L2.
   plan.warps = p.num_q_heads / p.num_kv_heads <= 8 ? kAttnWarpsNarrow : kAttnWarpsWide;
+  if (throughput == 3) plan.warps = kAttnWarpsWide;  // two layers per launch: two head tiles per warp, as for wide groups
   const int64_t rows_ = (int64_t)p.num_seqs * p.q_per_seq;
   // Side by side, 32 to 63 rows of 8 or more KV heads: 8 warps can take all 8 heads of a row (32 to 63 blocks per
   // launch, the shape that works best), which 12 warps cannot (4 heads per block, twice the blocks).
@@ -672,7 +686,7 @@ struct TailKey {
 };
 
 ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fine, int hg_base, int hg_fine) {
-  const ChainTail none = {0, 0};
+  const ChainTail none = {0, 0, 0};
   const double rate = kPortBytesPerClock * (double)key.clock_khz * 1e3 / 1e6;  // bytes per microsecond per SM
   auto duration = [&](int heads_per_block) { return kBlockFixedUs + (double)heads_per_block * key.k_eff * 512.0 / rate; };
   const double d_base = duration(key.hb), d_fine = duration(key.hf);
@@ -712,7 +726,7 @@ ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fin
         gt = h.place(nb_base, d_base, gt, en);
       }
       for (int l = 0; l < tail; ++l) gt = h.place(nb_fine, d_fine, gt, en);
-      if (en < best - 1e-9) { best = en; best_tail = ChainTail{tail, (int)part}; }
+      if (en < best - 1e-9) { best = en; best_tail = ChainTail{tail, (int)part, 0}; }
     }
   if (best > 0.98 * plain) best_tail = none;
   return best_tail;
@@ -721,9 +735,11 @@ ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fin
 }  // namespace
 
 ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
-  const ChainTail none = {0, 0};
+  const ChainTail none = {0, 0, 0};
   const int L = p.num_layers;
   if (L < 2) return none;
+  // Decode chains of query-head groups up to 8: the layers go two per launch (an odd last layer on its own).
+  if (p.q_per_seq == 1 && p.num_q_heads / p.num_kv_heads <= 8) return ChainTail{0, 0, L & ~1};
   if (p.block_table != nullptr) return none;  // paged caches: the finer blocks cost more than the fuller last round returns
   // The block model above was measured on a B200 (148 SMs); on anything else the chain keeps one block size.
   if (dev.sm_count != 148 || dev.clock_khz <= 0) return none;
@@ -768,11 +784,14 @@ double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev) {
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
-                               int keep_for_next, int throughput_plan, int fine_rows, const DeviceInfo& dev,
-                               cudaStream_t stream) {
+                               int keep_for_next, int throughput_plan, int fine_rows, const void* q2, void* out2,
+                               const DeviceInfo& dev, cudaStream_t stream) {
   const AttnPlan plan = make_attn_plan(p, dev, throughput_plan);
+  const bool pair = q2 != nullptr && out2 != nullptr;
   AttnArgs a;
   a.q = static_cast<const uint16_t*>(q);
+  a.q2 = static_cast<const uint16_t*>(q2);
+  a.out2 = static_cast<uint16_t*>(out2);
   a.kc = static_cast<const uint16_t*>(p.k_cache);
   a.vc = static_cast<const uint16_t*>(p.v_cache);
   a.tok_stride = p.kv_token_stride;
@@ -823,7 +842,9 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   else if (plan.warps == kAttnWarpsNarrow) kernel = CLSA_ATTN_PICK(1, kAttnWarpsNarrow);
   else kernel = CLSA_ATTN_PICK(1, kAttnWarpsWide);
 #undef CLSA_ATTN_PICK
-  const bool can_mix = a.group <= 8 && !multi && !pg;  // the shapes a chain's partly finer layer can have
+  if (pair) kernel = pg ? sparse_attn_kernel<2, true, kAttnWarpsWide, false, false, true>
+                        : sparse_attn_kernel<2, false, kAttnWarpsWide, false, false, true>;
+  const bool can_mix = a.group <= 8 && !multi && !pg && !pair;  // the shapes a chain's partly finer layer can have
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
