@@ -464,13 +464,15 @@ clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, con
 }
 
 clsa_status clsa_chain_plan(const clsa_params* p, int32_t sm_count, int32_t clock_khz, int32_t* fine_layers,
-                            int32_t* fine_rows) {
-  if (fine_layers == nullptr || fine_rows == nullptr || sm_count < 1 || clock_khz < 1) return CLSA_ERR_INVALID_ARG;
+                            int32_t* fine_rows, int32_t* paired_layers) {
+  if (fine_layers == nullptr || fine_rows == nullptr || paired_layers == nullptr || sm_count < 1 || clock_khz < 1)
+    return CLSA_ERR_INVALID_ARG;
   CLSA_TRY(check_shape(p));
   DeviceInfo dev = {sm_count, 227 * 1024, 0, clock_khz};
   const ChainTail t = p->q_per_seq == 1 ? chain_fine_tail(*p, dev) : ChainTail{0, 0, 0};
   *fine_layers = t.layers;
   *fine_rows = t.rows;
+  *paired_layers = t.paired;
   return CLSA_OK;
 }
 

@@ -573,8 +573,10 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
     // work per block, not how many SMs one launch covers: as many KV heads per block as leave about 32 blocks
     // per launch, no clusters. Four or five layers are then in flight at once and keep every SM busy
     // (measured: 32 blocks per layer beat 16, 64 and 128 at every batch size tried).
+    // Two layers per launch (3): blocks run twice as long, and about 16 per launch did best (at 16 rows of 8 KV heads a
+    // block then takes a whole row, one KV head per warp: nothing is split and nothing merged).
     hc = hc_max;
-    while (hc > 1 && rows * ((hkv + hc - 1) / hc) < 32) hc /= 2;
+    while (hc > 1 && rows * ((hkv + hc - 1) / hc) < (throughput == 3 ? 16 : 32)) hc /= 2;
     if (throughput == 2 && hc > 1) hc /= 2;
   } else {
     // Heads per block: as few as it takes for all blocks to be resident at once (more blocks, and the
@@ -599,7 +601,7 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   {
     const int per_block = plan.warps / hc;  // (row, range) slots of a block
     const int64_t want_blocks = throughput ? (throughput == 2 ? 64 : 32) : 2 * (int64_t)dev.sm_count;
-    for (int rb = per_block; rb > 1; --rb) {
+    for (int rb = per_block; rb > 1 && throughput != 3; --rb) {  // (the two-layer kernel takes one row per block)
       if (per_block % rb != 0) continue;
       if ((rows + rb - 1) / rb * plan.head_groups >= want_blocks) { plan.rows_per_block = rb; break; }
     }
@@ -709,7 +711,9 @@ ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fin
   double best = plain;
   ChainTail best_tail = none;
   const int64_t rows = key.rows;
-  const int64_t step = rows >= 8 ? rows / 8 : 1;  // partial layers in eighths of the rows
+  // Whole layers only: the chains that still take this route (groups of 9 to 16 query heads; narrower groups go two
+  // layers per launch) have no launch of two block sizes.
+  const int64_t step = rows;
   for (int tail = 0; tail <= max_tail; ++tail)
     for (int64_t part = 0; part < rows; part += step) {
       if (tail == 0 && part == 0) continue;

@@ -97,7 +97,7 @@ def test_bad_arguments_are_refused_on_the_host(clsa):
     # decode launches need their merge scratch, whose size depends on the device: without one the call stops at the device query
     too_small = (clsa.CLSA_ERR_WORKSPACE, clsa.CLSA_ERR_CUDA)
     assert raw.clsa_sparse_attn(P(good), 0x50000, 0x60000, 0x70000, 0x80000, None, ws, 256, st) in too_small
-    for bad in (clsa.make_hints(reverse=2), clsa.make_hints(shared_gpu=-1), clsa.make_hints(shared_gpu=3), clsa.make_hints(keep_rows=7), clsa.make_hints(only_q_pending=2)):
+    for bad in (clsa.make_hints(reverse=2), clsa.make_hints(shared_gpu=-1), clsa.make_hints(shared_gpu=4), clsa.make_hints(keep_rows=7), clsa.make_hints(only_q_pending=2)):
         assert raw.clsa_sparse_attn_hinted(P(good), 0x50000, 0x60000, 0x70000, 0x80000, None, P(bad), ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
         assert raw.clsa_gather_probe(P(good), 0x60000, 0x70000, P(bad), ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
     assert raw.clsa_sparse_attn_hinted(P(good), None, 0x60000, 0x70000, 0x80000, None, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
@@ -130,25 +130,40 @@ def test_bad_arguments_are_refused_on_the_host(clsa):
 
 
 def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
-    """clsa_chain_plan (the host-side model behind the chained layers' launch shapes) needs no GPU. A shape that has
-    not been seen must cost microseconds, not milliseconds -- a server whose batch size keeps changing pays it on the
-    step that first sees a shape -- and shapes are remembered beyond a handful; two models that differ only in the
-    number of KV heads must not share an entry."""
+    """clsa_chain_plan (the host-side choice of the chained layers' launch shapes) needs no GPU. Decode chains of groups
+    of up to 8 query heads go two layers per launch. Wider groups keep one layer per launch and may end in a finer
+    tail, chosen by a model of how the blocks fill the SMs: a shape that has not been seen must cost microseconds, not
+    milliseconds -- a server whose batch size keeps changing pays it on the step that first sees a shape -- and shapes
+    are remembered beyond a handful; two models that differ only in the number of KV heads must not share an entry."""
     import time
 
-    def plan(**kw):
-        return clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, **kw), 148, 1965000)
+    def narrow(**kw):
+        return clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, **{"num_layers": 16, **kw}), 148, 1965000)
 
-    assert plan(num_seqs=16) in ((2, 2), (2, 4), (3, 0), (2, 6), (2, 8))      # the headline: a short finer tail
-    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16), 132, 1755000) == (0, 0)  # a device the model was not measured on
+    def wide(**kw):   # 16 query heads per KV head: one layer per launch
+        kw = {"num_layers": 16, "num_q_heads": 128, "num_kv_heads": 8, "max_seq_len": 131072, **kw}
+        return clsa.clsa_chain_plan(_good(clsa, **kw), 148, 1965000)
+
+    # two layers per launch: all of them, all but an odd last one, none for a single layer or a prefill chunk;
+    # paged caches and unknown devices alike
+    assert narrow(num_seqs=16) == (0, 0, 16) and narrow(num_seqs=16, num_layers=15) == (0, 0, 14)
+    assert narrow(num_seqs=16, num_layers=1) == (0, 0, 0) and narrow(num_seqs=16, q_per_seq=4) == (0, 0, 0)
+    assert narrow(num_seqs=3, block_table=0x5000, block_size=16, max_blocks_per_seq=8192) == (0, 0, 16)
+    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16), 132, 1755000) == (0, 0, 16)
+    # wide groups: a short finer tail at most, never pairs; a device the block model was not measured on keeps one shape
+    fl, fr, pl = wide(num_seqs=16, top_k=2048)
+    assert 0 <= fl <= 3 and fr >= 0 and pl == 0
+    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16, num_q_heads=128,
+                                      num_kv_heads=8), 132, 1755000) == (0, 0, 0)
     shapes = [dict(num_seqs=b, top_k=k) for b in range(1, 51) for k in (1024, 2048)]
     t0 = time.perf_counter()
-    first = [clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, num_layers=16, **sh), 148, 1965000) for sh in shapes]
+    first = [wide(**sh) for sh in shapes]
     cold = (time.perf_counter() - t0) / len(shapes)
     t0 = time.perf_counter()
-    again = [clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, num_layers=16, **sh), 148, 1965000) for sh in shapes[-60:]]
+    again = [wide(**sh) for sh in shapes[-60:]]
     warm = (time.perf_counter() - t0) / 60
     assert again == first[-60:]
+    assert any(f[0] > 0 for f in first), "the model never chose a finer tail"
     assert cold < 100e-6, f"{cold * 1e6:.1f} us per unseen shape (ctypes call included)"
     assert warm < 30e-6, f"{warm * 1e6:.1f} us per remembered shape"
     # The memo may never hand one model's answer to another (models that share heads per block and rows but differ in
@@ -156,7 +171,7 @@ def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
     # fresh processes ask the same 72 models in opposite orders and must agree on every one.
     code = (
         "import sys, json; sys.path.insert(0, %r); import paper_2606_06467_b200 as c\n"
-        "cfgs = [(b, hq, hkv, k) for b in (4, 8, 12, 16, 20, 32) for hq, hkv in ((32, 8), (64, 16), (16, 4), (20, 4)) for k in (1024, 2048, 4096)]\n"
+        "cfgs = [(b, hq, hkv, k) for b in (4, 8, 12, 16, 20, 32) for hq, hkv in ((128, 8), (256, 16), (64, 4), (48, 4)) for k in (1024, 2048, 4096)]\n"
         "cfgs = cfgs[::-1] if sys.argv[1] == 'r' else cfgs\n"
         "out = {}\n"
         "for b, hq, hkv, k in cfgs:\n"
@@ -167,11 +182,13 @@ def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
     rev = subprocess.check_output([sys.executable, "-c", code, "r"])
     assert fwd == rev and len(fwd) > 500
     # paged caches, prefill chunks and single layers keep one shape
-    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16, block_table=0x5000, block_size=16, max_blocks_per_seq=8192), 148, 1965000) == (0, 0)
-    assert plan(num_seqs=16, q_per_seq=4) == (0, 0) and clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=1, num_seqs=16), 148, 1965000) == (0, 0)
+    assert wide(num_seqs=16, block_table=0x5000, block_size=16, max_blocks_per_seq=8192) == (0, 0, 0)
+    assert wide(num_seqs=16, q_per_seq=4) == (0, 0, 0) and wide(num_seqs=16, num_layers=1) == (0, 0, 0)
     n = ctypes.c_int32(0)
-    assert clsa.raw().clsa_chain_plan(ctypes.byref(_good(clsa)), 0, 1965000, ctypes.byref(n), ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
-    assert clsa.raw().clsa_chain_plan(ctypes.byref(_good(clsa)), 148, 1965000, None, ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
+    raw = clsa.raw().clsa_chain_plan
+    assert raw(ctypes.byref(_good(clsa)), 0, 1965000, ctypes.byref(n), ctypes.byref(n), ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw(ctypes.byref(_good(clsa)), 148, 1965000, None, ctypes.byref(n), ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw(ctypes.byref(_good(clsa)), 148, 1965000, ctypes.byref(n), ctypes.byref(n), None) == clsa.CLSA_ERR_INVALID_ARG
 
 
 def test_binding_raises_with_the_status(clsa):

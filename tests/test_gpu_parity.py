@@ -60,7 +60,10 @@ def _run_all(w, layers=None, check_lse=True):
         # ... and its finer variant, which a chain may use for its last layers
         out2, lse2 = g.sparse_attn(l, shared_gpu=2, keep_rows=keep)
         check_attention(prob, w, l, out2, lse2 if check_lse else None, idx_np, cnt_np)
-        singles.append((out1, out2))
+        # ... and the block shape of the launches that compute two layers at once
+        out3, lse3 = g.sparse_attn(l, shared_gpu=3, keep_rows=keep)
+        check_attention(prob, w, l, out3, lse3 if check_lse else None, idx_np, cnt_np)
+        singles.append((out1, out2, out3))
     # the chain: same index for all layers, byte-identical to the separate calls in the chain's launch shapes
     g.idx.fill_(-7); g.count.fill_(-7)
     outs = g.decode_step()
@@ -68,15 +71,18 @@ def _run_all(w, layers=None, check_lse=True):
     np.testing.assert_array_equal(g.idx.cpu().numpy(), idx_np)
     np.testing.assert_array_equal(g.count.cpu().numpy(), cnt_np)
     props = torch.cuda.get_device_properties(0)
-    fine_layers, fine_rows = clsa.clsa_chain_plan(g.params, props.multi_processor_count, props.clock_rate)
+    fine_layers, fine_rows, paired_layers = clsa.clsa_chain_plan(g.params, props.multi_processor_count, props.clock_rate)
     rows = w.cfg.num_seqs * w.cfg.q_per_seq
     for l in range(g.L):
         # which shape each query row of this layer takes, as clsa_chain_plan reports it
+        a, b1, b2, b3 = (x.reshape(rows, -1).view(torch.int16) for x in (outs[l],) + singles[l])
+        if l < paired_layers:   # computed together with its neighbour: the single-layer launch of that block shape
+            assert torch.equal(a, b3), f"layer {l}: chain != separate call (shape 3)"
+            continue
         n_fine = rows if l >= g.L - fine_layers else (fine_rows if l == g.L - fine_layers - 1 else 0)
-        a, b1, b2 = (x.reshape(rows, -1).view(torch.int16) for x in (outs[l], singles[l][0], singles[l][1]))
         assert torch.equal(a[: rows - n_fine], b1[: rows - n_fine]), f"layer {l}: chain != separate call (shape 1)"
         assert torch.equal(a[rows - n_fine:], b2[rows - n_fine:]), f"layer {l}: chain != separate call (shape 2)"
-    g.fine_layers = fine_layers
+    g.fine_layers, g.paired_layers = fine_layers, paired_layers
     # the attention half of the chain on its own, fed the index that is already there
     layer_outs = [g.new_out() for _ in range(g.L)]
     clsa.clsa_sparse_attn_layers(g.params, [g.t["q_layers"][l] for l in range(g.L)], g.idx, g.count, layer_outs, g.ws)
@@ -113,13 +119,24 @@ def test_ragged_with_duplicates_and_short_sequences():
     np.testing.assert_array_equal(gs[b, 0, dup].view(np.uint32), gs[b, 0, local[dup]].view(np.uint32))
 
 
-def test_chain_with_finer_last_layers():
-    """The headline's launch geometry at a context the oracle handles in seconds: 16 layers of 32 blocks do not fill
-    148 SMs evenly, so the chain gives its last layers the finer shape; every layer still equals the separate call of
-    its shape bit for bit, and the oracle within tolerance. The launches with the GPU to themselves cut 128 (row, KV
-    head) units over 148 blocks: spans that end inside a unit, partials merged across blocks."""
+def test_chain_at_the_headline_geometry():
+    """The headline's launch geometry at a context the oracle handles in seconds. Groups of 4 query heads: the chain
+    computes its 16 layers two per launch, and every layer equals the single-layer launch of that block shape bit for
+    bit, and the oracle within tolerance. With an odd number of layers the last one goes alone."""
     w = Workload(MID.replace(num_seqs=16, ctx=4096, top_k=2048, num_layers=16, seed=31))
     g, _ = _run_all(w, check_lse=False)
+    assert g.paired_layers == 16 and g.fine_layers == 0
+    g, _ = _run_all(Workload(MID.replace(num_seqs=5, ctx=3000, top_k=700, num_layers=3, seed=32)), check_lse=False)
+    assert g.paired_layers == 2
+
+
+def test_chain_of_wide_groups_with_finer_last_layers():
+    """16 query heads per KV head: one layer per launch (a warp's two head tiles are taken by the group), 16 layers of
+    32 blocks do not fill 148 SMs evenly, so the chain gives its last layers the finer shape; every layer still equals
+    the separate call of its shape bit for bit, and the oracle within tolerance."""
+    w = Workload(MID.replace(num_seqs=16, ctx=4096, top_k=2048, num_layers=16, num_q_heads=128, num_kv_heads=8, seed=33))
+    g, _ = _run_all(w, check_lse=False)
+    assert g.paired_layers == 0
     if torch.cuda.get_device_properties(0).multi_processor_count == 148:
         assert 1 <= g.fine_layers <= 3, g.fine_layers
 
