@@ -63,8 +63,7 @@ _lib.clsa_decode_step.argtypes = [_P, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_
 _lib.clsa_decode_step_static.argtypes = [_P, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _vp, _vp, _vp]
 _lib.clsa_sparse_attn_layers.argtypes = [_P, ctypes.POINTER(_vp), _vp, _vp, ctypes.POINTER(_vp), _vp, _sz, _vp]
 _lib.clsa_project_append.argtypes = [_P, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
-_lib.clsa_chain_plan.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
-                                 ctypes.POINTER(ctypes.c_int32)]
+_lib.clsa_chain_plan.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
 _lib.clsa_clear_status.argtypes = [_vp, _sz, _vp]
 _lib.clsa_device_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32), _vp]
 _lib.clsa_status_string.argtypes = [ctypes.c_int]
@@ -240,12 +239,11 @@ def clsa_project_append(p, d_model, h, w_q_idx, w_k_idx, w_k, w_v, q_idx_out, id
 
 
 def clsa_chain_plan(p, sm_count, clock_khz):
-    """(fine_layers, fine_rows, paired_layers): the tail of an L-layer chain that uses the finer launch shape, and the
-    number of leading layers that are computed two per launch. Host only."""
-    a, b, c = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
-    _check(_lib.clsa_chain_plan(ctypes.byref(p), int(sm_count), int(clock_khz), ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
-           "clsa_chain_plan")
-    return int(a.value), int(b.value), int(c.value)
+    """(fine_layers, paired_layers): the trailing layers of an L-layer chain that use the finer launch shape, and the
+    leading layers that are computed two per launch. Host only."""
+    a, b = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(_lib.clsa_chain_plan(ctypes.byref(p), int(sm_count), int(clock_khz), ctypes.byref(a), ctypes.byref(b)), "clsa_chain_plan")
+    return int(a.value), int(b.value)
 
 
 def clsa_clear_status(workspace, workspace_bytes=None, stream=None) -> None:

@@ -152,7 +152,7 @@ clsa_status check_hints(const clsa_attn_hints* h) {
 // whole (row, KV head) units to blocks.
 cudaError_t launch_attention(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                              float* lse, uint32_t* status, unsigned char* ws_base, const WorkspaceLayout& w,
-                             const clsa_attn_hints& h, int wait_prior, int fine_rows, const void* q2, void* out2,
+                             const clsa_attn_hints& h, int wait_prior, const void* q2, void* out2,
                              const DeviceInfo& dev, cudaStream_t s) {
   // With the GPU to itself, a decode launch whose (row, KV head) units would leave many SMs idle in the last round of
   // whole-unit blocks (20 rows x 8 heads: 160 units on 148 SMs) cuts its work at token granularity instead.
@@ -164,7 +164,7 @@ cudaError_t launch_attention(const clsa_params& p, const void* q, const int32_t*
                                  h.only_q_pending, h.keep_rows, dev, s);
   }
   return launch_sparse_attn(p, q, idx, count, out, lse, status, h.reverse, wait_prior, h.only_q_pending, h.keep_rows,
-                            h.shared_gpu, fine_rows, q2, out2, dev, s);
+                            h.shared_gpu, q2, out2, dev, s);
 }
 
 // The L attention launches that share one index. Layer 0 follows whatever produced the index and must wait for it;
@@ -181,15 +181,14 @@ cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, voi
   for (int l = 0; l + 1 < tail.paired; l += 2) {
     const clsa_attn_hints h = {0, 3, l + 2 < p.num_layers ? 1 : 0, 0};
     const cudaError_t err = launch_attention(p, q_layers[l], idx, count, out_layers[l], nullptr, status, ws_base, w, h,
-                                             l == 0 ? 1 : 0, 0, q_layers[l + 1], out_layers[l + 1], dev, s);
+                                             l == 0 ? 1 : 0, q_layers[l + 1], out_layers[l + 1], dev, s);
     if (err != cudaSuccess) return err;
   }
   for (int l = tail.paired; l < p.num_layers; ++l) {
     const bool fine = l >= p.num_layers - tail.layers;
-    const int fine_rows = l == p.num_layers - tail.layers - 1 ? tail.rows : 0;  // the layer where the finer shape begins
     const clsa_attn_hints h = {0, fine ? 2 : 1, l + 1 < p.num_layers ? 1 : 0, 0};
     const cudaError_t err = launch_attention(p, q_layers[l], idx, count, out_layers[l], nullptr, status, ws_base, w, h,
-                                             l == 0 ? 1 : 0, fine_rows, nullptr, nullptr, dev, s);
+                                             l == 0 ? 1 : 0, nullptr, nullptr, dev, s);
     if (err != cudaSuccess) return err;
   }
   return cudaSuccess;
@@ -294,7 +293,7 @@ clsa_status clsa_sparse_attn_hinted(const clsa_params* p, const void* q, const i
   // a decode launch with the GPU to itself merges its split partials through the scratch behind the header
   CLSA_TRY(check_workspace(workspace, workspace_bytes, p->q_per_seq == 1 && h.shared_gpu == 0 ? w.scores_off : kStatusBytes));
   auto base = static_cast<unsigned char*>(workspace);
-  return from_cuda(launch_attention(*p, q, idx, count, out, lse, reinterpret_cast<uint32_t*>(base), base, w, h, 1, 0, nullptr, nullptr, dev,
+  return from_cuda(launch_attention(*p, q, idx, count, out, lse, reinterpret_cast<uint32_t*>(base), base, w, h, 1, nullptr, nullptr, dev,
                                     static_cast<cudaStream_t>(stream)));
 }
 
@@ -464,14 +463,12 @@ clsa_status clsa_decode_step_static(const clsa_params* p, const void* q_idx, con
 }
 
 clsa_status clsa_chain_plan(const clsa_params* p, int32_t sm_count, int32_t clock_khz, int32_t* fine_layers,
-                            int32_t* fine_rows, int32_t* paired_layers) {
-  if (fine_layers == nullptr || fine_rows == nullptr || paired_layers == nullptr || sm_count < 1 || clock_khz < 1)
-    return CLSA_ERR_INVALID_ARG;
+                            int32_t* paired_layers) {
+  if (fine_layers == nullptr || paired_layers == nullptr || sm_count < 1 || clock_khz < 1) return CLSA_ERR_INVALID_ARG;
   CLSA_TRY(check_shape(p));
   DeviceInfo dev = {sm_count, 227 * 1024, 0, clock_khz};
-  const ChainTail t = p->q_per_seq == 1 ? chain_fine_tail(*p, dev) : ChainTail{0, 0, 0};
+  const ChainTail t = p->q_per_seq == 1 ? chain_fine_tail(*p, dev) : ChainTail{0, 0};
   *fine_layers = t.layers;
-  *fine_rows = t.rows;
   *paired_layers = t.paired;
   return CLSA_OK;
 }

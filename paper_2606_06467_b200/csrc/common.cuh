@@ -44,8 +44,7 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
 // Which part of an L-layer chain should use the finer shape (throughput = 2) so that the chain's blocks fill the SMs
 // evenly to the end: the last `layers` layers entirely, and the last `rows` query rows of the layer before them.
 struct ChainTail {
-  int layers;
-  int rows;
+  int layers;  // trailing layers that use the finer shape
   int paired;  // leading layers of the chain that are computed two per launch (even; 0 = none)
 };
 ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev);
@@ -139,7 +138,7 @@ cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int
 // rows (throughput_plan 3, decode, groups of up to 8 query heads).
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
-                               int keep_for_next, int throughput_plan, int fine_rows, const void* q2, void* out2,
+                               int keep_for_next, int throughput_plan, const void* q2, void* out2,
                                const DeviceInfo& dev, cudaStream_t stream);
 // Share of its rounds of one-block-per-SM that the whole-unit kernel's launch-on-its-own shape fills (0..1).
 double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev);

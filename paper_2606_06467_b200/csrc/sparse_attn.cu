@@ -65,9 +65,6 @@ struct AttnArgs {
   int off32;          // every row offset of the caches fits 32 bits when counted in 16-byte units
   int64_t rows_max;   // extent of the cache row space (off32 only): rows at or beyond it are refused like bad indices
   int keep;           // 1: the rows are fetched with the L2 evict_last priority (launches behind this one read them again)
-  int coarse_blocks;  // -1: one block size, 2-D grid. >= 0: a 1-D grid of two block sizes (no cluster, one row per block):
-                      // the first coarse_blocks blocks take heads_per_block KV heads each, row by row; the blocks behind
-                      // them take half as many (twice the token ranges) and cover the remaining rows
   int pin;            // -1: one L2 priority for every row (evict_last if keep). 0..8: of every 8 consecutive stages of a row's
                       // selected set the first `pin` are fetched evict_last and the others evict_first
   int max_seq_len;    // sequences longer than this (or shorter than q_per_seq) are skipped and flagged
@@ -78,37 +75,20 @@ struct AttnArgs {
 // WARPS = warps per block: 12 for NT = 1 (about 165 registers per thread), 8 for NT = 2.
 // MULTI: a block serves several query rows (rows_per_block > 1); the single-row instances keep the row uniform
 // over the block.
-// MIXED = the launch has two block sizes (AttnArgs::coarse_blocks); a variant of its own so that launches of one
-// size keep their block shape in kernel parameters, not registers.
 // PAIR = two layers in one launch (NT == 2, groups of up to 8 query heads): head tile 0 holds the first layer's query
 // heads, tile 1 the second layer's, both over the same staged K/V rows -- the rows of a step are the same for every
 // layer, so a pair of layers whose queries are both at hand copies them from L2 once instead of twice. Per layer the
 // arithmetic is that of a single-layer launch of the same block shape, bit for bit.
-template <int NT, bool PAGED, int WARPS, bool MULTI, bool MIXED = false, bool PAIR = false>
+template <int NT, bool PAGED, int WARPS, bool MULTI, bool PAIR = false>
 __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnArgs a) {
-  static_assert(!PAIR || (NT == 2 && !MULTI && !MIXED), "a pair of layers takes the two head tiles");
+  static_assert(!PAIR || (NT == 2 && !MULTI), "a pair of layers takes the two head tiles");
   extern __shared__ __align__(128) unsigned char smem[];
   cg::cluster_group cluster = cg::this_cluster();
   const int C = (int)cluster.num_blocks();
   const int crank = (int)cluster.block_rank();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int HC_ = a.heads_per_block, S_ = a.subs;
-  unsigned bx = blockIdx.x, by = blockIdx.y;
-  if (MIXED) {
-    const int hgc = (a.num_kv_heads + HC_ - 1) / HC_;  // coarse blocks per row
-    if ((int)blockIdx.x < a.coarse_blocks) {
-      bx = blockIdx.x / hgc;
-      by = blockIdx.x % hgc;
-    } else {
-      const int j = (int)blockIdx.x - a.coarse_blocks;
-      HC_ >>= 1;
-      S_ <<= 1;
-      const int hgf = (a.num_kv_heads + HC_ - 1) / HC_;  // fine blocks per row
-      bx = a.coarse_blocks / hgc + j / hgf;
-      by = j % hgf;
-    }
-  }
-  const int HC = HC_, S = S_, G = a.group;
+  const unsigned bx = blockIdx.x, by = blockIdx.y;
+  const int HC = a.heads_per_block, S = a.subs, G = a.group;
   const int g_local = warp % HC;
   const int RB = MULTI ? a.rows_per_block : 1;
   const int row_local = MULTI ? (warp / HC) / S : 0;  // which of the block's rows
@@ -688,7 +668,7 @@ struct TailKey {
 };
 
 ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fine, int hg_base, int hg_fine) {
-  const ChainTail none = {0, 0, 0};
+  const ChainTail none = {0, 0};
   const double rate = kPortBytesPerClock * (double)key.clock_khz * 1e3 / 1e6;  // bytes per microsecond per SM
   auto duration = [&](int heads_per_block) { return kBlockFixedUs + (double)heads_per_block * key.k_eff * 512.0 / rate; };
   const double d_base = duration(key.hb), d_fine = duration(key.hf);
@@ -730,7 +710,7 @@ ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fin
         gt = h.place(nb_base, d_base, gt, en);
       }
       for (int l = 0; l < tail; ++l) gt = h.place(nb_fine, d_fine, gt, en);
-      if (en < best - 1e-9) { best = en; best_tail = ChainTail{tail, (int)part, 0}; }
+      if (en < best - 1e-9) { best = en; best_tail = ChainTail{tail, 0}; }
     }
   if (best > 0.98 * plain) best_tail = none;
   return best_tail;
@@ -739,11 +719,11 @@ ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fin
 }  // namespace
 
 ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
-  const ChainTail none = {0, 0, 0};
+  const ChainTail none = {0, 0};
   const int L = p.num_layers;
   if (L < 2) return none;
   // Decode chains of query-head groups up to 8: the layers go two per launch (an odd last layer on its own).
-  if (p.q_per_seq == 1 && p.num_q_heads / p.num_kv_heads <= 8) return ChainTail{0, 0, L & ~1};
+  if (p.q_per_seq == 1 && p.num_q_heads / p.num_kv_heads <= 8) return ChainTail{0, L & ~1};
   if (p.block_table != nullptr) return none;  // paged caches: the finer blocks cost more than the fuller last round returns
   // The block model above was measured on a B200 (148 SMs); on anything else the chain keeps one block size.
   if (dev.sm_count != 148 || dev.clock_khz <= 0) return none;
@@ -788,7 +768,7 @@ double attn_alone_occupancy(const clsa_params& p, const DeviceInfo& dev) {
 
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
-                               int keep_for_next, int throughput_plan, int fine_rows, const void* q2, void* out2,
+                               int keep_for_next, int throughput_plan, const void* q2, void* out2,
                                const DeviceInfo& dev, cudaStream_t stream) {
   const AttnPlan plan = make_attn_plan(p, dev, throughput_plan);
   const bool pair = q2 != nullptr && out2 != nullptr;
@@ -831,7 +811,6 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   // there (pinned_stages_of_eight); chained launches trail one another over the same rows and fetch everything
   // evict_last.
   a.pin = (keep_for_next && throughput_plan == 0) ? pinned_stages_of_eight(p, dev) : -1;
-  a.coarse_blocks = -1;
   a.max_seq_len = p.max_seq_len;
   a.scale_log2 = p.sm_scale * kLog2e;
   // With the extent of the row space known (num_cache_rows) and below 2^32 16-byte units, row offsets are 32-bit.
@@ -846,28 +825,13 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   else if (plan.warps == kAttnWarpsNarrow) kernel = CLSA_ATTN_PICK(1, kAttnWarpsNarrow);
   else kernel = CLSA_ATTN_PICK(1, kAttnWarpsWide);
 #undef CLSA_ATTN_PICK
-  if (pair) kernel = pg ? sparse_attn_kernel<2, true, kAttnWarpsWide, false, false, true>
-                        : sparse_attn_kernel<2, false, kAttnWarpsWide, false, false, true>;
-  const bool can_mix = a.group <= 8 && !multi && !pg && !pair;  // the shapes a chain's partly finer layer can have
+  if (pair) kernel = pg ? sparse_attn_kernel<2, true, kAttnWarpsWide, false, true>
+                        : sparse_attn_kernel<2, false, kAttnWarpsWide, false, true>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((rows + plan.rows_per_block - 1) / plan.rows_per_block * plan.cluster), (unsigned)plan.head_groups, 1);
-  // Two block sizes in one launch (the layer of a chain where the finer shape begins, see chain_fine_tail): the
-  // last fine_rows rows get blocks of half the KV heads. Only where the plan allows it; otherwise one size.
-  if (can_mix && throughput_plan == 1 && fine_rows > 0 && fine_rows < rows && plan.cluster == 1 &&
-      plan.rows_per_block == 1 && plan.heads_per_block > 1) {
-    kernel = plan.warps == kAttnWarpsNarrow ? sparse_attn_kernel<1, false, kAttnWarpsNarrow, false, true>
-                                            : sparse_attn_kernel<1, false, kAttnWarpsWide, false, true>;
-    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
-    if (err != cudaSuccess) return err;
-    const int hc_fine = plan.heads_per_block / 2;
-    const int64_t coarse = (rows - fine_rows) * plan.head_groups;
-    const int64_t fine = (int64_t)fine_rows * ((p.num_kv_heads + hc_fine - 1) / hc_fine);
-    a.coarse_blocks = (int)coarse;
-    cfg.gridDim = dim3((unsigned)(coarse + fine), 1, 1);
-  }
   cfg.blockDim = dim3((unsigned)plan.warps * 32, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;

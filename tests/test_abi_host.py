@@ -146,15 +146,15 @@ def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
 
     # two layers per launch: all of them, all but an odd last one, none for a single layer or a prefill chunk;
     # paged caches and unknown devices alike
-    assert narrow(num_seqs=16) == (0, 0, 16) and narrow(num_seqs=16, num_layers=15) == (0, 0, 14)
-    assert narrow(num_seqs=16, num_layers=1) == (0, 0, 0) and narrow(num_seqs=16, q_per_seq=4) == (0, 0, 0)
-    assert narrow(num_seqs=3, block_table=0x5000, block_size=16, max_blocks_per_seq=8192) == (0, 0, 16)
-    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16), 132, 1755000) == (0, 0, 16)
+    assert narrow(num_seqs=16) == (0, 16) and narrow(num_seqs=16, num_layers=15) == (0, 14)
+    assert narrow(num_seqs=16, num_layers=1) == (0, 0) and narrow(num_seqs=16, q_per_seq=4) == (0, 0)
+    assert narrow(num_seqs=3, block_table=0x5000, block_size=16, max_blocks_per_seq=8192) == (0, 16)
+    assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16), 132, 1755000) == (0, 16)
     # wide groups: a short finer tail at most, never pairs; a device the block model was not measured on keeps one shape
-    fl, fr, pl = wide(num_seqs=16, top_k=2048)
-    assert 0 <= fl <= 3 and fr >= 0 and pl == 0
+    fl, pl = wide(num_seqs=16, top_k=2048)
+    assert 0 <= fl <= 3 and pl == 0
     assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16, num_q_heads=128,
-                                      num_kv_heads=8), 132, 1755000) == (0, 0, 0)
+                                      num_kv_heads=8), 132, 1755000) == (0, 0)
     shapes = [dict(num_seqs=b, top_k=k) for b in range(1, 51) for k in (1024, 2048)]
     t0 = time.perf_counter()
     first = [wide(**sh) for sh in shapes]
@@ -182,13 +182,13 @@ def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
     rev = subprocess.check_output([sys.executable, "-c", code, "r"])
     assert fwd == rev and len(fwd) > 500
     # paged caches, prefill chunks and single layers keep one shape
-    assert wide(num_seqs=16, block_table=0x5000, block_size=16, max_blocks_per_seq=8192) == (0, 0, 0)
-    assert wide(num_seqs=16, q_per_seq=4) == (0, 0, 0) and wide(num_seqs=16, num_layers=1) == (0, 0, 0)
+    assert wide(num_seqs=16, block_table=0x5000, block_size=16, max_blocks_per_seq=8192) == (0, 0)
+    assert wide(num_seqs=16, q_per_seq=4) == (0, 0) and wide(num_seqs=16, num_layers=1) == (0, 0)
     n = ctypes.c_int32(0)
     raw = clsa.raw().clsa_chain_plan
-    assert raw(ctypes.byref(_good(clsa)), 0, 1965000, ctypes.byref(n), ctypes.byref(n), ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
-    assert raw(ctypes.byref(_good(clsa)), 148, 1965000, None, ctypes.byref(n), ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
-    assert raw(ctypes.byref(_good(clsa)), 148, 1965000, ctypes.byref(n), ctypes.byref(n), None) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw(ctypes.byref(_good(clsa)), 0, 1965000, ctypes.byref(n), ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw(ctypes.byref(_good(clsa)), 148, 1965000, None, ctypes.byref(n)) == clsa.CLSA_ERR_INVALID_ARG
+    assert raw(ctypes.byref(_good(clsa)), 148, 1965000, ctypes.byref(n), None) == clsa.CLSA_ERR_INVALID_ARG
 
 
 def test_binding_raises_with_the_status(clsa):

@@ -71,7 +71,7 @@ def _run_all(w, layers=None, check_lse=True):
     np.testing.assert_array_equal(g.idx.cpu().numpy(), idx_np)
     np.testing.assert_array_equal(g.count.cpu().numpy(), cnt_np)
     props = torch.cuda.get_device_properties(0)
-    fine_layers, fine_rows, paired_layers = clsa.clsa_chain_plan(g.params, props.multi_processor_count, props.clock_rate)
+    fine_layers, paired_layers = clsa.clsa_chain_plan(g.params, props.multi_processor_count, props.clock_rate)
     rows = w.cfg.num_seqs * w.cfg.q_per_seq
     for l in range(g.L):
         # which shape each query row of this layer takes, as clsa_chain_plan reports it
@@ -79,9 +79,8 @@ def _run_all(w, layers=None, check_lse=True):
         if l < paired_layers:   # computed together with its neighbour: the single-layer launch of that block shape
             assert torch.equal(a, b3), f"layer {l}: chain != separate call (shape 3)"
             continue
-        n_fine = rows if l >= g.L - fine_layers else (fine_rows if l == g.L - fine_layers - 1 else 0)
-        assert torch.equal(a[: rows - n_fine], b1[: rows - n_fine]), f"layer {l}: chain != separate call (shape 1)"
-        assert torch.equal(a[rows - n_fine:], b2[rows - n_fine:]), f"layer {l}: chain != separate call (shape 2)"
+        fine = l >= g.L - fine_layers
+        assert torch.equal(a, b2 if fine else b1), f"layer {l}: chain != separate call (shape {2 if fine else 1})"
     g.fine_layers, g.paired_layers = fine_layers, paired_layers
     # the attention half of the chain on its own, fed the index that is already there
     layer_outs = [g.new_out() for _ in range(g.L)]
