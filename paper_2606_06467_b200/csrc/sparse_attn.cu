@@ -26,7 +26,9 @@
 // (a prefill chunk) puts several rows in a block, up to one warp per (row, KV head) with nothing to merge. The layers of one decode step, which do not wait for one another,
 // are launched side by side instead: about 32 large blocks per layer (as many KV heads per block as that
 // allows), so that four or five layers are in flight at once: every SM stays busy and the per-block
-// fixed costs are paid 32 instead of 128 times per layer.
+// fixed costs are paid 32 instead of 128 times per layer. And where a warp has a head tile to spare (groups of up to
+// 8 query heads), such layers go two per launch: every layer of a step gathers the same rows, so the second tile
+// takes the next layer's query heads over the same staged rows (about 16 blocks per launch of two layers).
 // `reverse` flips the order in which a warp walks its range (a locality hint for callers that issue
 // dependent layers one by one; the chained layers of a step all walk the same way).
 #include <cooperative_groups.h>
