@@ -932,13 +932,17 @@ def run_ours(args):
             modes["dependent_with_ffn_reads"] = dep_ffn
     modes["independent"] = mode(ind_ms, ind_med, e2e_ind_ms)
     modes["independent"]["what"] = ("clsa_decode_step: every layer's queries are handed over up front, the layers do not wait for "
-                                    "one another and share the selected rows through L2 -- a rate of algorithmic bytes above the "
-                                    "HBM peak is L2 reuse, not HBM bandwidth" if decode else
+                                    "one another, go two per launch (the rows are copied from L2 once for both) and share the "
+                                    "selected rows through L2 -- a rate of algorithmic bytes above the HBM peak is L2 reuse, not "
+                                    "HBM bandwidth" if decode else
                                     "a prefill chunk: clsa_index_scores (tensor-core GEMM), clsa_topk, clsa_sparse_attn_layers")
     if decode and bd is not None and ceilings is not None:
         per_layer = (ind_med * 1e3 - bd["index_scores"] - bd["topk"]) / L
         modes["independent"]["attention_per_layer_us"] = per_layer
         modes["independent"]["attention_frac_of_l2_gather_ceiling"] = (gathered / (per_layer * 1e-6) / 1e9) / ceilings["l2_gather_ceiling"]["GBps"]
+        modes["independent"]["attention_note"] = ("gathered bytes per layer over the step's attention time per layer, against the rate at "
+                                                  "which one launch copies that many bytes from L2; above 1 where two layers share a "
+                                                  "launch, because the pair copies its rows once")
 
     cpu_baseline = None
     if solo and not args.no_cpu_baseline:
