@@ -467,7 +467,7 @@ clsa_status clsa_chain_plan(const clsa_params* p, int32_t sm_count, int32_t cloc
   if (fine_layers == nullptr || paired_layers == nullptr || sm_count < 1 || clock_khz < 1) return CLSA_ERR_INVALID_ARG;
   CLSA_TRY(check_shape(p));
   DeviceInfo dev = {sm_count, 227 * 1024, 0, clock_khz};
-  const ChainTail t = p->q_per_seq == 1 ? chain_fine_tail(*p, dev) : ChainTail{0, 0};
+  const ChainTail t = chain_fine_tail(*p, dev);
   *fine_layers = t.layers;
   *paired_layers = t.paired;
   return CLSA_OK;

@@ -83,7 +83,7 @@ struct AttnArgs {
 // arithmetic is that of a single-layer launch of the same block shape, bit for bit.
 template <int NT, bool PAGED, int WARPS, bool MULTI, bool PAIR = false>
 __global__ void __launch_bounds__(WARPS * 32, 1) sparse_attn_kernel(const AttnArgs a) {
-  static_assert(!PAIR || (NT == 2 && !MULTI), "a pair of layers takes the two head tiles");
+  static_assert(!PAIR || NT == 2, "a pair of layers takes the two head tiles");
   extern __shared__ __align__(128) unsigned char smem[];
   cg::cluster_group cluster = cg::this_cluster();
   const int C = (int)cluster.num_blocks();
@@ -583,7 +583,7 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   {
     const int per_block = plan.warps / hc;  // (row, range) slots of a block
     const int64_t want_blocks = throughput ? (throughput == 2 ? 64 : 32) : 2 * (int64_t)dev.sm_count;
-    for (int rb = per_block; rb > 1 && throughput != 3; --rb) {  // (the two-layer kernel takes one row per block)
+    for (int rb = per_block; rb > 1; --rb) {
       if (per_block % rb != 0) continue;
       if ((rows + rb - 1) / rb * plan.head_groups >= want_blocks) { plan.rows_per_block = rb; break; }
     }
@@ -724,8 +724,8 @@ ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
   const ChainTail none = {0, 0};
   const int L = p.num_layers;
   if (L < 2) return none;
-  // Decode chains of query-head groups up to 8: the layers go two per launch (an odd last layer on its own).
-  if (p.q_per_seq == 1 && p.num_q_heads / p.num_kv_heads <= 8) return ChainTail{0, L & ~1};
+  // Chains of query-head groups up to 8: the layers go two per launch (an odd last layer on its own).
+  if (p.num_q_heads / p.num_kv_heads <= 8) return ChainTail{0, L & ~1};
   if (p.block_table != nullptr) return none;  // paged caches: the finer blocks cost more than the fuller last round returns
   // The block model above was measured on a B200 (148 SMs); on anything else the chain keeps one block size.
   if (dev.sm_count != 148 || dev.clock_khz <= 0) return none;
@@ -827,8 +827,10 @@ cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_
   else if (plan.warps == kAttnWarpsNarrow) kernel = CLSA_ATTN_PICK(1, kAttnWarpsNarrow);
   else kernel = CLSA_ATTN_PICK(1, kAttnWarpsWide);
 #undef CLSA_ATTN_PICK
-  if (pair) kernel = pg ? sparse_attn_kernel<2, true, kAttnWarpsWide, false, true>
-                        : sparse_attn_kernel<2, false, kAttnWarpsWide, false, true>;
+  if (pair) kernel = multi ? (pg ? sparse_attn_kernel<2, true, kAttnWarpsWide, true, true>
+                                 : sparse_attn_kernel<2, false, kAttnWarpsWide, true, true>)
+                           : (pg ? sparse_attn_kernel<2, true, kAttnWarpsWide, false, true>
+                                 : sparse_attn_kernel<2, false, kAttnWarpsWide, false, true>);
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (err != cudaSuccess) return err;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;

@@ -144,10 +144,10 @@ def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
         kw = {"num_layers": 16, "num_q_heads": 128, "num_kv_heads": 8, "max_seq_len": 131072, **kw}
         return clsa.clsa_chain_plan(_good(clsa, **kw), 148, 1965000)
 
-    # two layers per launch: all of them, all but an odd last one, none for a single layer or a prefill chunk;
+    # two layers per launch: all of them, all but an odd last one, none for a single layer; prefill chunks,
     # paged caches and unknown devices alike
     assert narrow(num_seqs=16) == (0, 16) and narrow(num_seqs=16, num_layers=15) == (0, 14)
-    assert narrow(num_seqs=16, num_layers=1) == (0, 0) and narrow(num_seqs=16, q_per_seq=4) == (0, 0)
+    assert narrow(num_seqs=16, num_layers=1) == (0, 0) and narrow(num_seqs=16, q_per_seq=4) == (0, 16)   # chunks pair too
     assert narrow(num_seqs=3, block_table=0x5000, block_size=16, max_blocks_per_seq=8192) == (0, 16)
     assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16), 132, 1755000) == (0, 16)
     # wide groups: a short finer tail at most, never pairs; a device the block model was not measured on keeps one shape
