@@ -187,7 +187,10 @@ typedef struct {
                              chained calls use it for their last layers so that the chain's blocks keep every SM
                              busy to the end (see clsa_chain_plan).
                              3: the block shape of the launches in which the chained calls compute two layers at once
-                             (see clsa_chain_plan), for one layer: a few larger blocks, about 16 per launch. */
+                             (see clsa_chain_plan), for one layer: a few larger blocks, about 16 per launch; which
+                             shape that is depends on p->num_layers too (how many such launches share the GPU).
+                             4: as 3 with half the KV heads per block where the chain's plan allows it; the chained
+                             calls use it for their last pairs of layers. */
   int32_t keep_rows;      /* 1: another launch that reads the same selected rows follows (the next layer): fetch them
                              with the L2 evict_last priority so that other traffic does not push them out in between. */
   int32_t only_q_pending; /* 1: idx, count, seq_len, the block table and the caches were all complete before the kernel
@@ -207,8 +210,8 @@ CLSA_API clsa_status clsa_sparse_attn_hinted(const clsa_params* p, const void* q
  *   q_layers   HOST array of L device pointers, each bf16 [B][T][Hq][D]
  *   out_layers HOST array of L device pointers, each bf16 [B][T][Hq][D]
  * Equivalent, bit for bit, to clsa_index_scores, clsa_topk and L calls of clsa_sparse_attn_hinted made one after
- * another with hints {reverse 0, shared_gpu 3 for the layers that clsa_chain_plan reports as computed two per launch,
- * else 1 or -- for the last layers that it reports -- 2, keep_rows 1 except for the last layer}. Two layers per launch (decoding, groups of
+ * another with hints {reverse 0, shared_gpu 3 (or 4) for the layers that clsa_chain_plan reports as computed two per
+ * launch (in the finer shape), else 1 (or 2), keep_rows 1 except for the last layer}. Two layers per launch (decoding, groups of
  * up to 8 query heads per KV head): every layer gathers the same rows, so a launch that has two layers' queries copies
  * the rows from L2 once for both. The layers do not wait for one another (each reads only the index, the caches and its own queries, all of which the caller
  * hands over up front), so several of them are in flight at once and share the selected rows through L2. A decoder
@@ -296,11 +299,12 @@ CLSA_API clsa_status clsa_gather_probe(const clsa_params* p, const int32_t* idx,
 
 /* Host only, no CUDA call: the launch shapes of an L-layer chain (clsa_decode_step, clsa_sparse_attn_layers) on a device
  * with `sm_count` SMs and a peak SM clock of `clock_khz`. The first *paired_layers layers (an even number) are computed
- * two per launch (shared_gpu = 3; decoding with groups of up to 8 query heads: all but an odd last layer). Of the
- * others, the last *fine_layers layers use the finer shape (shared_gpu = 2), the rest shape 1 (0: one shape; always so
- * for T > 1, for paged caches and for devices the block model was not measured on). The finer tail comes from a model of
- * how the chain's blocks fill the SMs; it costs a few microseconds the first time a shape is seen and is remembered
- * afterwards. Outputs are HOST pointers. */
+ * two per launch (groups of up to 8 query heads: all but an odd last layer), the last *fine_layers of them in the finer
+ * shape (shared_gpu = 4), the rest in shape 3. With *paired_layers = 0 (wider groups) the last *fine_layers layers use
+ * the finer one-layer shape (shared_gpu = 2), the rest shape 1. *fine_layers = 0: one shape throughout; always so for
+ * T > 1 and for devices the block model was not measured on. The finer tail comes from a model of how the chain's blocks
+ * fill the SMs; it costs a few microseconds the first time a shape is seen and is remembered afterwards. Outputs are
+ * HOST pointers. */
 CLSA_API clsa_status clsa_chain_plan(const clsa_params* p, int32_t sm_count, int32_t clock_khz, int32_t* fine_layers,
                                      int32_t* paired_layers);
 

@@ -142,7 +142,7 @@ clsa_status check_hints(const clsa_attn_hints* h) {
   if (h == nullptr) return CLSA_OK;
   for (int32_t v : {h->reverse, h->keep_rows, h->only_q_pending})
     if (v != 0 && v != 1) return CLSA_ERR_INVALID_ARG;
-  if (h->shared_gpu < 0 || h->shared_gpu > 3) return CLSA_ERR_INVALID_ARG;
+  if (h->shared_gpu < 0 || h->shared_gpu > 4) return CLSA_ERR_INVALID_ARG;
   return CLSA_OK;
 }
 
@@ -179,13 +179,14 @@ cudaError_t launch_layers(const clsa_params& p, const void* const* q_layers, voi
   const ChainTail tail = chain_fine_tail(p, dev);
   // The leading layers two per launch: both read the same rows, which are then copied from L2 once for the two.
   for (int l = 0; l + 1 < tail.paired; l += 2) {
-    const clsa_attn_hints h = {0, 3, l + 2 < p.num_layers ? 1 : 0, 0};
+    const bool fine = l >= tail.paired - tail.layers;  // the last pairs of the chain in the finer shape
+    const clsa_attn_hints h = {0, fine ? 4 : 3, l + 2 < p.num_layers ? 1 : 0, 0};
     const cudaError_t err = launch_attention(p, q_layers[l], idx, count, out_layers[l], nullptr, status, ws_base, w, h,
                                              l == 0 ? 1 : 0, q_layers[l + 1], out_layers[l + 1], dev, s);
     if (err != cudaSuccess) return err;
   }
   for (int l = tail.paired; l < p.num_layers; ++l) {
-    const bool fine = l >= p.num_layers - tail.layers;
+    const bool fine = tail.paired == 0 && l >= p.num_layers - tail.layers;
     const clsa_attn_hints h = {0, fine ? 2 : 1, l + 1 < p.num_layers ? 1 : 0, 0};
     const cudaError_t err = launch_attention(p, q_layers[l], idx, count, out_layers[l], nullptr, status, ws_base, w, h,
                                              l == 0 ? 1 : 0, nullptr, nullptr, dev, s);

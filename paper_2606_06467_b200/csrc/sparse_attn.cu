@@ -530,13 +530,19 @@ static int max_resident_blocks(int cluster, size_t smem_bytes, int warps) {
 
 }  // namespace
 
+// Block model of the two-layer decode launches (measured on a B200 at the headline: a block of 8 KV heads x 2048 tokens
+// x 2 layers takes about 125 us).
+constexpr double kPairBytesPerUs = 64.0e3;   // bytes of K/V rows a block copies per microsecond
+constexpr double kPairBlockFixedUs = 9.5;    // launch gap + pipeline ramp + merge of one block
+
 AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int throughput) {
   AttnPlan plan;
   // 12 warps per block where the registers allow it (query-head groups up to 8: one 8-column tile per warp); the
   // main loop is a dependent chain per warp, so warps per SM, not bytes in flight, set the pace once the rows come
   // from L2.
   plan.warps = p.num_q_heads / p.num_kv_heads <= 8 ? kAttnWarpsNarrow : kAttnWarpsWide;
-  if (throughput == 3) plan.warps = kAttnWarpsWide;  // two layers per launch: two head tiles per warp, as for wide groups
+  const bool pair_shape = throughput == 3 || throughput == 4;
+  if (pair_shape) plan.warps = kAttnWarpsWide;  // two layers per launch: two head tiles per warp, as for wide groups
   const int64_t rows_ = (int64_t)p.num_seqs * p.q_per_seq;
   // Side by side, 32 to 63 rows of 8 or more KV heads: 8 warps can take all 8 heads of a row (32 to 63 blocks per
   // launch, the shape that works best), which 12 warps cannot (4 heads per block, twice the blocks).
@@ -549,16 +555,40 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   int hc_max = 1;
   while (hc_max * 2 <= hkv && plan.warps % (hc_max * 2) == 0) hc_max *= 2;
   int hc, c = 1;
+  bool pair_fine_grain = false;
   if (throughput) {
     // The launch shares the GPU with the launches next to it on the stream (the layers of one step: each reads
     // only the index, the caches and its own queries, so none waits for its predecessor). What counts then is the
     // work per block, not how many SMs one launch covers: as many KV heads per block as leave about 32 blocks
     // per launch, no clusters. Four or five layers are then in flight at once and keep every SM busy
     // (measured: 32 blocks per layer beat 16, 64 and 128 at every batch size tried).
-    // Two layers per launch (3): blocks run twice as long, and about 16 per launch did best (at 16 rows of 8 KV heads a
-    // block then takes a whole row, one KV head per warp: nothing is split and nothing merged).
     hc = hc_max;
-    while (hc > 1 && rows * ((hkv + hc - 1) / hc) < (throughput == 3 ? 16 : 32)) hc /= 2;
+    while (hc > 1 && rows * ((hkv + hc - 1) / hc) < (pair_shape ? 16 : 32)) hc /= 2;
+    // ... as long as the step has at most about two and a half rounds of blocks; beyond that the finer blocks lose more
+    // (split rows, rows of a step no longer walked together by its launches) than the fuller last round returns.
+    pair_fine_grain = pair_shape && p.q_per_seq == 1 &&
+                      (p.num_layers >= 2 ? p.num_layers / 2 : 1) * rows * ((hkv + hc - 1) / hc) * 2 <= 5 * (int64_t)dev.sm_count;
+    if (pair_fine_grain) {
+      // Two layers per launch, decoding: blocks run twice as long, and about 16 per launch do best while all launches
+      // of the step are resident at once (16 rows of 8 KV heads: a block takes a whole row, one KV head per warp,
+      // nothing split and nothing merged; 8 launches x 16 blocks on 148 SMs). One row more and the step's blocks no
+      // longer fit one round: then fewer heads per block fill the last round at a finer grain. The same block model as
+      // for the finer tail of one-layer chains: a fixed part plus the block's bytes at the rate a block of this kernel
+      // copies them; the step's blocks are placed in rounds of one per SM.
+      const double k_eff = (double)(p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len);
+      const double us_per_head = k_eff * 512.0 / kPairBytesPerUs;
+      const int64_t launches = p.num_layers >= 2 ? p.num_layers / 2 : 1;
+      double best = 0.0;
+      int best_hc = hc;
+      for (int cand = hc; cand >= 1; cand /= 2) {
+        const int64_t blocks = launches * rows * ((hkv + cand - 1) / cand);
+        const int64_t rounds = (blocks + dev.sm_count - 1) / dev.sm_count;
+        const double cost = (double)rounds * (kPairBlockFixedUs + cand * us_per_head);
+        if (cand == hc || cost < 0.97 * best) { best = cost; best_hc = cand; }
+      }
+      hc = best_hc;
+    }
+    if (throughput == 4 && hc > 1 && pair_fine_grain) hc /= 2;
     if (throughput == 2 && hc > 1) hc /= 2;
   } else {
     // Heads per block: as few as it takes for all blocks to be resident at once (more blocks, and the
@@ -583,7 +613,8 @@ AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int through
   {
     const int per_block = plan.warps / hc;  // (row, range) slots of a block
     const int64_t want_blocks = throughput ? (throughput == 2 ? 64 : 32) : 2 * (int64_t)dev.sm_count;
-    for (int rb = per_block; rb > 1; --rb) {
+    // (not for the two-layer decode launches: their heads per block were chosen for the number of blocks they give)
+    for (int rb = per_block; rb > 1 && !pair_fine_grain; --rb) {
       if (per_block % rb != 0) continue;
       if ((rows + rb - 1) / rb * plan.head_groups >= want_blocks) { plan.rows_per_block = rb; break; }
     }
@@ -661,18 +692,21 @@ struct SmGroups {
 };
 
 struct TailKey {
-  int L, sms, clock_khz, k_eff, hb, hf, hkv;
+  int L, sms, clock_khz, k_eff, hb, hf, hkv;  // L: launches of the chain
   int64_t rows;
+  int pair;                                   // launches of two layers each (their own block model)
   bool operator==(const TailKey& o) const {
     return L == o.L && sms == o.sms && clock_khz == o.clock_khz && k_eff == o.k_eff && hb == o.hb && hf == o.hf &&
-           hkv == o.hkv && rows == o.rows;
+           hkv == o.hkv && rows == o.rows && pair == o.pair;
   }
 };
 
 ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fine, int hg_base, int hg_fine) {
   const ChainTail none = {0, 0};
-  const double rate = kPortBytesPerClock * (double)key.clock_khz * 1e3 / 1e6;  // bytes per microsecond per SM
-  auto duration = [&](int heads_per_block) { return kBlockFixedUs + (double)heads_per_block * key.k_eff * 512.0 / rate; };
+  // bytes per microsecond that a block copies: the L2-to-SM port for one-layer blocks, what the two-layer kernel reaches
+  const double rate = key.pair ? kPairBytesPerUs : kPortBytesPerClock * (double)key.clock_khz * 1e3 / 1e6;
+  const double fixed = key.pair ? kPairBlockFixedUs : kBlockFixedUs;
+  auto duration = [&](int heads_per_block) { return fixed + (double)heads_per_block * key.k_eff * 512.0 / rate; };
   const double d_base = duration(key.hb), d_fine = duration(key.hf);
   const int L = key.L;
   const int max_tail = L - 1 < kTailMaxLayers ? L - 1 : kTailMaxLayers;
@@ -721,23 +755,27 @@ ChainTail simulate_fine_tail(const TailKey& key, int64_t nb_base, int64_t nb_fin
 }  // namespace
 
 ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
-  const ChainTail none = {0, 0};
   const int L = p.num_layers;
-  if (L < 2) return none;
-  // Chains of query-head groups up to 8: the layers go two per launch (an odd last layer on its own).
-  if (p.num_q_heads / p.num_kv_heads <= 8) return ChainTail{0, L & ~1};
-  if (p.block_table != nullptr) return none;  // paged caches: the finer blocks cost more than the fuller last round returns
-  // The block model above was measured on a B200 (148 SMs); on anything else the chain keeps one block size.
-  if (dev.sm_count != 148 || dev.clock_khz <= 0) return none;
-  const AttnPlan base = make_attn_plan(p, dev, 1), fine = make_attn_plan(p, dev, 2);
+  if (L < 2) return ChainTail{0, 0};
+  // Chains of query-head groups up to 8: the layers go two per launch (an odd last layer on its own); the last of
+  // those launches may take the finer shape too.
+  const bool pair = p.num_q_heads / p.num_kv_heads <= 8;
+  const ChainTail plain = {0, pair ? (L & ~1) : 0};
+  if (!pair && p.block_table != nullptr) return plain;  // paged caches: the finer blocks cost more than the fuller last round returns
+  // The block models were measured on a B200 (148 SMs); on anything else the chain keeps one block size.
+  if (dev.sm_count != 148 || dev.clock_khz <= 0) return plain;
+  if (pair && p.q_per_seq != 1) return plain;
+  const AttnPlan base = make_attn_plan(p, dev, pair ? 3 : 1), fine = make_attn_plan(p, dev, pair ? 4 : 2);
   if (base.cluster != 1 || fine.cluster != 1 || fine.heads_per_block == base.heads_per_block ||
       base.rows_per_block != 1 || fine.rows_per_block != 1)
-    return none;
+    return plain;
   const int64_t rows = (int64_t)p.num_seqs * p.q_per_seq;
   const int64_t nb_base = rows * base.head_groups, nb_fine = rows * fine.head_groups;
-  if (nb_base > 4096 || nb_fine > 8192) return none;  // far more blocks than SMs: the last round is a small part of the whole
-  const TailKey key = {L, dev.sm_count, dev.clock_khz, p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len,
-                       base.heads_per_block, fine.heads_per_block, p.num_kv_heads, rows};
+  if (nb_base > 4096 || nb_fine > 8192) return plain;  // far more blocks than SMs: the last round is a small part of the whole
+  const int launches = pair ? L / 2 : L;
+  if (launches < 2) return plain;
+  const TailKey key = {launches, dev.sm_count, dev.clock_khz, p.top_k < p.max_seq_len ? p.top_k : p.max_seq_len,
+                       base.heads_per_block, fine.heads_per_block, p.num_kv_heads, rows, pair ? 1 : 0};
   struct Entry { TailKey key; ChainTail tail; uint64_t used; };
   constexpr int kMemo = 64;
   static std::mutex mu;
@@ -749,7 +787,8 @@ ChainTail chain_fine_tail(const clsa_params& p, const DeviceInfo& dev) {
     for (int i = 0; i < filled; ++i)
       if (memo[i].key == key) { memo[i].used = ++tick; return memo[i].tail; }
   }
-  const ChainTail tail = simulate_fine_tail(key, nb_base, nb_fine, base.head_groups, fine.head_groups);  // outside the lock
+  ChainTail tail = simulate_fine_tail(key, nb_base, nb_fine, base.head_groups, fine.head_groups);  // outside the lock
+  if (pair) tail = ChainTail{2 * tail.layers, L & ~1};  // the model counts launches; the plan counts layers
   {
     std::lock_guard<std::mutex> lock(mu);
     int slot = 0;

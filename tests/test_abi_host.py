@@ -97,7 +97,7 @@ def test_bad_arguments_are_refused_on_the_host(clsa):
     # decode launches need their merge scratch, whose size depends on the device: without one the call stops at the device query
     too_small = (clsa.CLSA_ERR_WORKSPACE, clsa.CLSA_ERR_CUDA)
     assert raw.clsa_sparse_attn(P(good), 0x50000, 0x60000, 0x70000, 0x80000, None, ws, 256, st) in too_small
-    for bad in (clsa.make_hints(reverse=2), clsa.make_hints(shared_gpu=-1), clsa.make_hints(shared_gpu=4), clsa.make_hints(keep_rows=7), clsa.make_hints(only_q_pending=2)):
+    for bad in (clsa.make_hints(reverse=2), clsa.make_hints(shared_gpu=-1), clsa.make_hints(shared_gpu=5), clsa.make_hints(keep_rows=7), clsa.make_hints(only_q_pending=2)):
         assert raw.clsa_sparse_attn_hinted(P(good), 0x50000, 0x60000, 0x70000, 0x80000, None, P(bad), ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
         assert raw.clsa_gather_probe(P(good), 0x60000, 0x70000, P(bad), ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
     assert raw.clsa_sparse_attn_hinted(P(good), None, 0x60000, 0x70000, 0x80000, None, None, ws, wsb, st) == clsa.CLSA_ERR_INVALID_ARG
@@ -148,6 +148,7 @@ def test_chain_planner_is_cheap_and_keyed_on_every_input(clsa):
     # paged caches and unknown devices alike
     assert narrow(num_seqs=16) == (0, 16) and narrow(num_seqs=16, num_layers=15) == (0, 14)
     assert narrow(num_seqs=16, num_layers=1) == (0, 0) and narrow(num_seqs=16, q_per_seq=4) == (0, 16)   # chunks pair too
+    assert narrow(num_seqs=20) in ((2, 16), (4, 16), (6, 16))   # more blocks than one round of SMs holds: a finer tail of pairs
     assert narrow(num_seqs=3, block_table=0x5000, block_size=16, max_blocks_per_seq=8192) == (0, 16)
     assert clsa.clsa_chain_plan(_good(clsa, max_seq_len=131072, top_k=2048, num_layers=16, num_seqs=16), 132, 1755000) == (0, 16)
     # wide groups: a short finer tail at most, never pairs; a device the block model was not measured on keeps one shape

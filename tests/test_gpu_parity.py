@@ -63,7 +63,9 @@ def _run_all(w, layers=None, check_lse=True):
         # ... and the block shape of the launches that compute two layers at once
         out3, lse3 = g.sparse_attn(l, shared_gpu=3, keep_rows=keep)
         check_attention(prob, w, l, out3, lse3 if check_lse else None, idx_np, cnt_np)
-        singles.append((out1, out2, out3))
+        out4, lse4 = g.sparse_attn(l, shared_gpu=4, keep_rows=keep)
+        check_attention(prob, w, l, out4, lse4 if check_lse else None, idx_np, cnt_np)
+        singles.append((out1, out2, out3, out4))
     # the chain: same index for all layers, byte-identical to the separate calls in the chain's launch shapes
     g.idx.fill_(-7); g.count.fill_(-7)
     outs = g.decode_step()
@@ -75,9 +77,10 @@ def _run_all(w, layers=None, check_lse=True):
     rows = w.cfg.num_seqs * w.cfg.q_per_seq
     for l in range(g.L):
         # which shape each query row of this layer takes, as clsa_chain_plan reports it
-        a, b1, b2, b3 = (x.reshape(rows, -1).view(torch.int16) for x in (outs[l],) + singles[l])
+        a, b1, b2, b3, b4 = (x.reshape(rows, -1).view(torch.int16) for x in (outs[l],) + singles[l])
         if l < paired_layers:   # computed together with its neighbour: the single-layer launch of that block shape
-            assert torch.equal(a, b3), f"layer {l}: chain != separate call (shape 3)"
+            fine = l >= paired_layers - fine_layers
+            assert torch.equal(a, b4 if fine else b3), f"layer {l}: chain != separate call (shape {4 if fine else 3})"
             continue
         fine = l >= g.L - fine_layers
         assert torch.equal(a, b2 if fine else b1), f"layer {l}: chain != separate call (shape {2 if fine else 1})"
@@ -127,6 +130,10 @@ def test_chain_at_the_headline_geometry():
     assert g.paired_layers == 16 and g.fine_layers == 0
     g, _ = _run_all(Workload(MID.replace(num_seqs=5, ctx=3000, top_k=700, num_layers=3, seed=32)), check_lse=False)
     assert g.paired_layers == 2
+    # 20 rows: the step's blocks no longer fit one round of one per SM, and the last pairs take the finer shape
+    g, _ = _run_all(Workload(MID.replace(num_seqs=20, ctx=2500, top_k=2048, num_layers=16, seed=34)), check_lse=False)
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert g.paired_layers == 16 and g.fine_layers in (2, 4, 6), g.fine_layers
 
 
 def test_chain_of_wide_groups_with_finer_last_layers():

@@ -66,7 +66,7 @@ def test_chunk_scores_topk_attention(B, T, n, d_idx, causal, ragged):
     clsa.clsa_sparse_attn_layers(g.params, [g.t["q_layers"][l] for l in range(2)], g.idx, g.count, outs, g.ws)
     for l in range(2):
         check_attention(prob, w, l, outs[l], None, idx_np, cnt_np)
-        singles = [g.sparse_attn(l, shared_gpu=sg, keep_rows=1 if l == 0 else 0, lse=False)[0] for sg in (1, 2, 3)]
+        singles = [g.sparse_attn(l, shared_gpu=sg, keep_rows=1 if l == 0 else 0, lse=False)[0] for sg in (1, 2, 3, 4)]
         assert any(torch.equal(outs[l].view(torch.int16), x.view(torch.int16)) for x in singles), l
     assert g.status() == 0
 

@@ -69,7 +69,7 @@ def test_random_shape(seed):
         out, lse = g.sparse_attn(l, reverse=l & 1, keep_rows=1, only_q_pending=int(l > 0))
         check_attention(prob, w, l, out, lse, idx_np, cnt_np)
         pair = []
-        for shape in (1, 2, 3):
+        for shape in (1, 2, 3, 4):
             o, s = g.sparse_attn(l, shared_gpu=shape)
             check_attention(prob, w, l, o, s, idx_np, cnt_np)
             pair.append(o)
@@ -79,7 +79,7 @@ def test_random_shape(seed):
         torch.cuda.synchronize()
         for l in range(L):
             rows = outs[l].shape[0] * outs[l].shape[1]
-            a, b1, b2, b3 = (x.reshape(rows, -1).view(torch.int16) for x in [outs[l]] + singles[l])
-            same = (a == b1).all(dim=1) | (a == b2).all(dim=1) | (a == b3).all(dim=1)
+            a, b1, b2, b3, b4 = (x.reshape(rows, -1).view(torch.int16) for x in [outs[l]] + singles[l])
+            same = (a == b1).all(dim=1) | (a == b2).all(dim=1) | (a == b3).all(dim=1) | (a == b4).all(dim=1)
             assert bool(same.all()), "chain differs from the separate calls"
     assert g.status() == 0
