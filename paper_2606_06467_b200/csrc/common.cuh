@@ -39,10 +39,12 @@ struct AttnPlan {
 // throughput: 0 = a launch on its own (whole-GPU shape); 1 = a few large blocks (the launch shares the GPU with its
 // neighbours on the stream); 2 = the same with half the KV heads per block, where that is possible (twice the
 // blocks: used for the last layers of a chain, see chain_fine_tail); 3 = the shape of a launch that computes two layers
-// at once (8 warps with two head tiles each), also available to a single layer so that a pair's results can be reproduced
+// at once (8 warps with two head tiles each), also available to a single layer so that a pair's results can be
+// reproduced; 4 = as 3 with half the KV heads per block where the plan cuts the step's blocks finely
 AttnPlan make_attn_plan(const clsa_params& p, const DeviceInfo& dev, int throughput);
-// Which part of an L-layer chain should use the finer shape (throughput = 2) so that the chain's blocks fill the SMs
-// evenly to the end: the last `layers` layers entirely, and the last `rows` query rows of the layer before them.
+// The launch shapes of an L-layer chain: how many leading layers go two per launch, and how many trailing layers (of
+// those, or of all when none are paired) use the finer shape (throughput = 4 or 2) so that the chain's blocks fill the
+// SMs evenly to the end.
 struct ChainTail {
   int layers;  // trailing layers that use the finer shape
   int paired;  // leading layers of the chain that are computed two per launch (even; 0 = none)
@@ -135,7 +137,7 @@ bool topk_prefilter_fits(const clsa_params& p, const float* scores, int64_t scor
 cudaError_t launch_topk_prefilter(const clsa_params& p, const float* scores, int64_t score_stride, int32_t* idx,
                                   int32_t* count, uint32_t* status, const DeviceInfo& dev, cudaStream_t stream);
 // q2 / out2: nullptr, or the queries and outputs of a second layer that the same launch computes over the same staged
-// rows (throughput_plan 3, decode, groups of up to 8 query heads).
+// rows (throughput_plan 3 or 4, groups of up to 8 query heads).
 cudaError_t launch_sparse_attn(const clsa_params& p, const void* q, const int32_t* idx, const int32_t* count, void* out,
                                float* lse, uint32_t* status, int reverse, int wait_prior, int only_q_pending,
                                int keep_for_next, int throughput_plan, const void* q2, void* out2,
