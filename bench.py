@@ -903,6 +903,12 @@ def run_ours(args):
                     "predecessor left them, so this is a rate of algorithmic bytes and HBM traffic stays below it; the cold "
                     "first layer reads every row from DRAM",
         }
+        for key, name in (("steady_layer", "sparse_attn_kernel"), ("cold_first_layer", "sparse_attn_kernel_cold")):
+            t = profiled_traffic(c.name, name)   # DRAM bytes of that launch as recorded from the one-pass ncu capture
+            if t is not None:
+                roofline[key]["traffic"] = t
+                roofline[key]["dram_GBps"] = t / (roofline[key]["us"] * 1e-6) / 1e9
+                roofline[key]["dram_frac_of_hbm_peak"] = roofline[key]["dram_GBps"] / peak
         if ceilings is not None:
             roofline.update(ceilings)
             for key in ("steady_layer", "cold_first_layer"):
